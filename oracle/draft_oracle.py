@@ -1,0 +1,188 @@
+"""Longest-suffix match and draft-tree construction by brute force (test infrastructure).
+
+What is computed (paper, Section 3: SuffixDecoding "stores the historical trajectories and matches the
+current token pattern against them to generate draft tokens"; Section 3.2: it "caches token-sequence
+patterns from previously generated trajectories" and predicts likely next tokens from them):
+
+  match   the largest l <= min(P, tail_len) such that the last l context tokens occur contiguously inside
+          ONE stored trajectory (occurrences never straddle two trajectories);
+  tree    slot 0 is the root (the last context token).  Every other slot is one continuation token of the
+          matched string; count = number of occurrences (with multiplicity, overlaps included, over all
+          trajectories) of matched string + root path.  Each node offers its k most frequent continuations
+          (count descending, then token id ascending); slots are created best-first from the pool of
+          offered continuations (count descending, then parent slot ascending, then token id ascending)
+          until N slots exist or nothing is offered.
+
+The paper fixes none of the tie rules or the node budget convention; the rules above are this build's
+reading and are listed in the design notes.  No suffix tree or suffix array appears here on purpose.
+
+Two implementations live side by side:
+  * `*_definitional`: nested pure-Python loops straight from the definition, for tiny inputs;
+  * the numpy versions used at realistic sizes, which filter explicit occurrence lists.
+They are written differently (re-scan per candidate string vs. filtering), and the tests hold them against
+each other, against hand-worked examples and against invariants.
+"""
+from __future__ import annotations
+
+from typing import List, Sequence, Tuple
+
+import numpy as np
+
+
+# ----------------------------------------------------------------------------------------------
+# definitional versions (tiny inputs only)
+# ----------------------------------------------------------------------------------------------
+
+def occurrences_definitional(trajs: Sequence[Sequence[int]], s: Sequence[int]) -> List[Tuple[int, int]]:
+    """All (t, p) with trajs[t][p : p+len(s)] == s."""
+    s = [int(x) for x in s]
+    out = []
+    for t, tr in enumerate(trajs):
+        tr = [int(x) for x in tr]
+        for p in range(0, len(tr) - len(s) + 1):
+            if tr[p:p + len(s)] == s:
+                out.append((t, p))
+    return out
+
+
+def match_definitional(trajs, tail: Sequence[int], tail_len: int) -> int:
+    """Largest l <= tail_len whose suffix of the tail occurs; every l is tested, nothing is assumed monotone."""
+    P = len(tail)
+    best = 0
+    for l in range(1, tail_len + 1):
+        if occurrences_definitional(trajs, tail[P - l:]):
+            best = l
+    return best
+
+
+def draft_definitional(trajs, tail: Sequence[int], tail_len: int, N: int, k: int, min_match: int = 1):
+    """Returns (match_len, ids, parent, count) as Python lists of length num_nodes."""
+    P = len(tail)
+    tail = [int(x) for x in tail]
+    ml = match_definitional(trajs, tail, tail_len)
+    s = tail[P - ml:] if ml > 0 else []
+    ids, parent, count = [tail[P - 1]], [-1], [len(occurrences_definitional(trajs, s)) if ml > 0 else 0]
+    if ml < max(1, min_match) or N <= 1:
+        return ml, ids, parent, count
+    alphabet = sorted({int(x) for tr in trajs for x in tr})
+    paths = [[]]
+
+    def offers(slot):
+        cand = []
+        for x in alphabet:
+            c = len(occurrences_definitional(trajs, s + paths[slot] + [x]))
+            if c > 0:
+                cand.append((-c, x))
+        cand.sort()
+        return [(-negc, slot, x) for negc, x in cand[:k]]
+
+    frontier = offers(0)
+    while len(ids) < N and frontier:
+        frontier.sort(key=lambda e: (-e[0], e[1], e[2]))
+        c, p, x = frontier.pop(0)
+        ids.append(x); parent.append(p); count.append(c)
+        paths.append(paths[p] + [x])
+        frontier.extend(offers(len(ids) - 1))
+    return ml, ids, parent, count
+
+
+# ----------------------------------------------------------------------------------------------
+# numpy versions
+# ----------------------------------------------------------------------------------------------
+
+class Corpus:
+    """The stored trajectories, kept as one flat array plus, for every flat position, the flat bounds of the
+    trajectory that position belongs to.  This is bookkeeping, not an index: every query scans all tokens."""
+
+    def __init__(self, tokens: np.ndarray, offsets: np.ndarray):
+        self.tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+        self.offsets = np.asarray(offsets, dtype=np.int64)
+        lens = np.diff(self.offsets)
+        self.start_of = np.repeat(self.offsets[:-1], lens)
+        self.end_of = np.repeat(self.offsets[1:], lens)
+
+    @classmethod
+    def from_lists(cls, trajs):
+        lens = [len(t) for t in trajs]
+        off = np.zeros(len(trajs) + 1, dtype=np.int64)
+        off[1:] = np.cumsum(lens)
+        tok = np.concatenate([np.asarray(t, dtype=np.int32) for t in trajs]) if trajs else np.zeros(0, np.int32)
+        return cls(tok, off)
+
+
+def longest_suffix_match(corpus: Corpus, tail: np.ndarray, tail_len: int) -> Tuple[int, np.ndarray]:
+    """Returns (match_len, ends): `ends` are the flat positions of the LAST token of every occurrence of the
+    longest occurring suffix.  Occurrence is monotone in the suffix length (dropping the first token of an
+    occurring string leaves an occurring string), so the scan grows l until no occurrence survives."""
+    P = len(tail)
+    tok = corpus.tokens
+    if tail_len <= 0 or len(tok) == 0:
+        return 0, np.zeros(0, dtype=np.int64)
+    ends = np.flatnonzero(tok == tail[P - 1]).astype(np.int64)
+    if len(ends) == 0:
+        return 0, ends
+    l = 1
+    while l < tail_len:
+        first = ends - l                                  # where the (l+1)-token suffix would start
+        inside = first >= corpus.start_of[ends]
+        keep = np.zeros(len(ends), dtype=bool)
+        keep[inside] = tok[first[inside]] == tail[P - 1 - l]
+        if not keep.any():
+            break
+        ends = ends[keep]
+        l += 1
+    return l, ends
+
+
+def build_draft_tree(corpus: Corpus, tail: np.ndarray, match_len: int, ends: np.ndarray, N: int, k: int,
+                     min_match: int = 1):
+    """Returns (ids, parent, count) int32 arrays of length num_nodes (see module docstring for the rules)."""
+    P = len(tail)
+    tok = corpus.tokens
+    ids, parent, count = [int(tail[P - 1])], [-1], [int(len(ends)) if match_len > 0 else 0]
+    if match_len < max(1, min_match) or N <= 1:
+        return np.array(ids, np.int32), np.array(parent, np.int32), np.array(count, np.int32)
+    # per slot: flat positions of the token that FOLLOWS each occurrence of matched string + path, and the
+    # flat end of the trajectory that occurrence lives in
+    nxt = [ends + 1]
+    lim = [corpus.end_of[ends]]
+
+    def offers(slot):
+        has_next = nxt[slot] < lim[slot]
+        t = tok[nxt[slot][has_next]]
+        if len(t) == 0:
+            return []
+        uniq, cnt = np.unique(t, return_counts=True)
+        order = np.lexsort((uniq, -cnt))[:k]              # count descending, token id ascending
+        return [(int(cnt[o]), slot, int(uniq[o])) for o in order]
+
+    frontier = offers(0)
+    while len(ids) < N and frontier:
+        best = min(range(len(frontier)), key=lambda e: (-frontier[e][0], frontier[e][1], frontier[e][2]))
+        c, p, x = frontier.pop(best)
+        has_next = nxt[p] < lim[p]
+        sel = np.zeros(len(nxt[p]), dtype=bool)
+        sel[has_next] = tok[nxt[p][has_next]] == x
+        ids.append(x); parent.append(p); count.append(c)
+        nxt.append(nxt[p][sel] + 1)
+        lim.append(lim[p][sel])
+        assert len(nxt[-1]) == c
+        frontier.extend(offers(len(ids) - 1))
+    return np.array(ids, np.int32), np.array(parent, np.int32), np.array(count, np.int32)
+
+
+def draft_batch(corpus: Corpus, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, min_match: int = 1):
+    """Batched form with the library's output convention: unused slots hold ids = -1, parent = -1, count = 0."""
+    B = tails.shape[0]
+    match_len = np.zeros(B, np.int32)
+    num_nodes = np.zeros(B, np.int32)
+    ids = np.full((B, N), -1, np.int32)
+    parent = np.full((B, N), -1, np.int32)
+    count = np.zeros((B, N), np.int32)
+    for i in range(B):
+        ml, ends = longest_suffix_match(corpus, tails[i], int(tail_len[i]))
+        a, b, c = build_draft_tree(corpus, tails[i], ml, ends, N, k, min_match)
+        n = len(a)
+        match_len[i], num_nodes[i] = ml, n
+        ids[i, :n], parent[i, :n], count[i, :n] = a, b, c
+    return match_len, num_nodes, ids, parent, count

@@ -1,0 +1,220 @@
+"""Pins for the brute-force match / draft-tree checker: hand-worked cases, a definitional brute force written
+differently, and invariants that hold by construction of the definition."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+from oracle import draft_oracle as D
+from paper_2607_17299_b200 import workloads as W
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _load(name):
+    with open(os.path.join(GOLD, name)) as f:
+        return json.load(f)
+
+
+def _window_occurrences(tokens, offsets, s):
+    """Independent count: sliding windows per trajectory (no shared code with the checker)."""
+    s = np.asarray(s, dtype=np.int32)
+    out = []
+    for t in range(len(offsets) - 1):
+        tr = tokens[offsets[t]:offsets[t + 1]]
+        if len(tr) < len(s):
+            continue
+        win = np.lib.stride_tricks.sliding_window_view(tr, len(s))
+        for p in np.flatnonzero((win == s).all(axis=1)):
+            out.append((t, int(p)))
+    return out
+
+
+@pytest.mark.parametrize("name", ["draft_case1.json", "draft_case2.json"])
+def test_hand_worked_cases(name):
+    g = _load(name)
+    trajs = g["trajectories"]
+    tail = np.array(g["tail"], dtype=np.int32)
+    corpus = D.Corpus.from_lists(trajs)
+    ml, ends = D.longest_suffix_match(corpus, tail, g["tail_len"])
+    assert ml == g["match_len"]
+    # occurrences: end position -> (t, p)
+    occ = sorted((int(np.searchsorted(corpus.offsets, e, side="right") - 1),
+                  int(e - (ml - 1) - corpus.start_of[e])) for e in ends)
+    assert occ == sorted(map(tuple, g["occurrences"]))
+    assert D.match_definitional(trajs, g["tail"], g["tail_len"]) == g["match_len"]
+    for tr in g["trees"]:
+        ids, parent, count = D.build_draft_tree(corpus, tail, ml, ends, tr["N"], tr["k"])
+        assert ids.tolist() == tr["ids"]
+        assert parent.tolist() == tr["parent"]
+        assert count.tolist() == tr["count"]
+        ml2, i2, p2, c2 = D.draft_definitional(trajs, g["tail"], g["tail_len"], tr["N"], tr["k"])
+        assert (ml2, i2, p2, c2) == (g["match_len"], tr["ids"], tr["parent"], tr["count"])
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_numpy_version_equals_definitional_on_tiny_alphabets(seed):
+    """Vocabularies of 2-5 symbols and corpora under 200 tokens force heavy count ties, so the
+    (count, parent slot, token) ordering rules are exercised on almost every slot."""
+    rng = np.random.default_rng(seed)
+    vocab = int(rng.integers(2, 6))
+    trajs = [rng.integers(0, vocab, size=int(rng.integers(1, 40))).tolist() for _ in range(int(rng.integers(1, 6)))]
+    corpus = D.Corpus.from_lists(trajs)
+    P = int(rng.integers(1, 9))
+    N = int(rng.integers(1, 20))
+    k = int(rng.integers(1, 5))
+    for _ in range(5):
+        tail = rng.integers(0, vocab + 1, size=P).astype(np.int32)     # vocab itself never occurs
+        tail_len = int(rng.integers(0, P + 1))
+        ml, ends = D.longest_suffix_match(corpus, tail, tail_len)
+        ids, parent, count = D.build_draft_tree(corpus, tail, ml, ends, N, k)
+        ml2, i2, p2, c2 = D.draft_definitional(trajs, tail.tolist(), tail_len, N, k)
+        assert ml == ml2
+        assert ids.tolist() == i2 and parent.tolist() == p2 and count.tolist() == c2
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    cfg = W.CONFIGS["tiny"]
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(cfg)
+    # add structured tails: planted copies, out-of-vocabulary, short tail_len
+    rng = np.random.default_rng(5)
+    extra, extra_len, planted = [], [], []
+    for _ in range(6):
+        t = int(rng.integers(0, cfg.n_traj))
+        dist = int(rng.integers(1, 200))                     # tokens from the trajectory start to the tail's end
+        e = int(off[t]) + dist
+        m = min(cfg.P, dist)
+        row = np.full(cfg.P, -1, np.int32)
+        row[cfg.P - m:] = tok[e - m:e]
+        extra.append(row); extra_len.append(m); planted.append(min(cfg.P, dist))
+    extra.append(np.full(cfg.P, cfg.vocab + 5, np.int32)); extra_len.append(cfg.P); planted.append(-1)
+    short = tails[0].copy(); extra.append(short); extra_len.append(3); planted.append(-1)
+    tails = np.concatenate([tails, np.stack(extra)])
+    tl = np.concatenate([tl, np.array(extra_len, np.int32)])
+    return cfg, tok, off, tails, tl, planted
+
+
+def test_match_invariants_on_tiny_workload(tiny):
+    cfg, tok, off, tails, tl, planted = tiny
+    corpus = D.Corpus(tok, off)
+    B0 = cfg.B
+    for i in range(len(tails)):
+        ml, ends = D.longest_suffix_match(corpus, tails[i], int(tl[i]))
+        assert 0 <= ml <= tl[i]
+        if ml > 0:
+            s = tails[i, cfg.P - ml:]
+            occ = _window_occurrences(tok, off, s)
+            assert len(occ) == len(ends) > 0                 # it occurs, and the count is the brute-force count
+            for e in ends[:50]:                              # reported places really hold the string
+                assert (tok[e - ml + 1:e + 1] == s).all()
+                assert e - ml + 1 >= corpus.start_of[e]
+        if ml < tl[i]:                                       # no longer match exists (full independent scan)
+            assert _window_occurrences(tok, off, tails[i, cfg.P - ml - 1:]) == []
+        for l in range(1, ml):                               # monotone: every shorter suffix occurs too
+            assert len(_window_occurrences(tok, off, tails[i, cfg.P - l:])) >= len(ends)
+        j = i - B0
+        if 0 <= j < len(planted) and planted[j] >= 0:
+            assert ml >= planted[j]
+    oov = B0 + 6
+    assert D.longest_suffix_match(corpus, tails[oov], int(tl[oov]))[0] == 0
+    assert D.longest_suffix_match(corpus, tails[oov + 1], 3)[0] <= 3
+
+
+def test_tree_invariants_on_tiny_workload(tiny):
+    cfg, tok, off, tails, tl, _ = tiny
+    corpus = D.Corpus(tok, off)
+    seen_unique = seen_branching = False
+    for i in range(len(tails)):
+        ml, ends = D.longest_suffix_match(corpus, tails[i], int(tl[i]))
+        ids, parent, count = D.build_draft_tree(corpus, tails[i], ml, ends, cfg.N, cfg.topk)
+        n = len(ids)
+        assert 1 <= n <= cfg.N and parent[0] == -1 and ids[0] == tails[i, -1]
+        if ml == 0:
+            assert n == 1 and count[0] == 0
+            continue
+        s = tails[i, cfg.P - ml:].tolist()
+        paths = [[]]
+        for j in range(1, n):
+            assert 0 <= parent[j] < j
+            assert count[j] <= count[parent[j]]
+            assert count[j] <= count[j - 1] or j == 1        # best-first => non-increasing after the root
+            paths.append(paths[parent[j]] + [int(ids[j])])
+        assert count[0] >= count[1:].max(initial=0)
+        for j in range(n):
+            kids = [int(ids[c]) for c in range(1, n) if parent[c] == j]
+            assert len(kids) == len(set(kids)) <= cfg.topk
+            occ = _window_occurrences(tok, off, s + paths[j])
+            assert len(occ) == count[j]
+            # all continuations of slot j (not only the kept ones) account for every occurrence that does not
+            # end its trajectory
+            nxt = {}
+            ending = 0
+            for (t, p) in occ:
+                q = off[t] + p + len(s) + len(paths[j])
+                if q < off[t + 1]:
+                    nxt[int(tok[q])] = nxt.get(int(tok[q]), 0) + 1
+                else:
+                    ending += 1
+            assert sum(nxt.values()) == count[j] - ending
+            ranked = sorted(nxt.items(), key=lambda kv: (-kv[1], kv[0]))[:cfg.topk]
+            if n < cfg.N:                                    # frontier emptied: every offered child is in the tree
+                assert sorted(kids) == sorted(x for x, _ in ranked)
+            else:                                            # kept children are a prefix of the ranking
+                assert kids == [x for x, _ in ranked][:len(kids)] or set(kids) <= {x for x, _ in ranked}
+            for c in range(1, n):
+                if parent[c] == j:
+                    assert nxt[int(ids[c])] == count[c]
+        if count[0] == 1:                                    # unique occurrence => chain = corpus continuation
+            seen_unique = True
+            e = int(ends[0])
+            room = int(corpus.end_of[e]) - (e + 1)
+            m = min(cfg.N - 1, room)
+            assert n == m + 1
+            assert ids[1:].tolist() == tok[e + 1:e + 1 + m].tolist()
+            assert parent[1:].tolist() == list(range(0, m))
+        else:
+            seen_branching = True
+    assert seen_unique and seen_branching
+
+
+def test_trajectory_order_does_not_matter(tiny):
+    """Every worker must draft the same tokens once the caches hold the same trajectories, in whatever order
+    they arrived (paper Section 3.2, cross-worker synchronisation)."""
+    cfg, tok, off, tails, tl, _ = tiny
+    rng = np.random.default_rng(11)
+    order = rng.permutation(cfg.n_traj)
+    trajs = [tok[off[t]:off[t + 1]] for t in order]
+    tok2 = np.concatenate(trajs)
+    off2 = np.zeros_like(off)
+    off2[1:] = np.cumsum([len(t) for t in trajs])
+    a = D.draft_batch(D.Corpus(tok, off), tails, tl, cfg.N, cfg.topk)
+    b = D.draft_batch(D.Corpus(tok2, off2), tails, tl, cfg.N, cfg.topk)
+    for x, y in zip(a, b):
+        assert (x == y).all()
+
+
+def test_no_match_across_trajectory_boundary():
+    trajs = [[1, 2], [3, 4]]
+    corpus = D.Corpus.from_lists(trajs)
+    ml, ends = D.longest_suffix_match(corpus, np.array([1, 2, 3], np.int32), 3)
+    assert ml == 1 and len(ends) == 1                        # [2,3] only exists across the boundary
+    ids, parent, count = D.build_draft_tree(corpus, np.array([1, 2, 3], np.int32), ml, ends, 8, 4)
+    assert ids.tolist() == [3, 4] and count.tolist() == [1, 1]
+
+
+def test_min_match_and_budget_edges():
+    trajs = [[1, 2, 3, 1, 2, 4]]
+    corpus = D.Corpus.from_lists(trajs)
+    tail = np.array([9, 1, 2], np.int32)
+    ml, ends = D.longest_suffix_match(corpus, tail, 3)
+    assert ml == 2
+    ids, parent, count = D.build_draft_tree(corpus, tail, ml, ends, 8, 4, min_match=3)
+    assert ids.tolist() == [2] and count.tolist() == [2]     # below min_match: root only, count still reported
+    ids, parent, count = D.build_draft_tree(corpus, tail, ml, ends, 1, 4)
+    assert ids.tolist() == [2]
+    ids, parent, count = D.build_draft_tree(corpus, tail, ml, ends, 3, 1)
+    assert ids.tolist() == [2, 3, 1] and parent.tolist() == [-1, 0, 1]   # k=1: chain along the smaller id on ties
+    assert D.longest_suffix_match(corpus, tail, 0)[0] == 0
