@@ -1,0 +1,171 @@
+/*
+ * war.h -- C ABI of the batched SuffixDecoding speculate-and-verify step for one B200 (sm_100a).
+ *
+ * The paper (WAR: Workload-Aware Rollouts, Section 3 overview and Section 3.2 "SuffixDecoding") speeds up
+ * low-load agentic RL rollouts with model-free speculative decoding: a cache of previously generated
+ * trajectories is matched against each live request's current token pattern to produce draft tokens, the
+ * target model verifies all drafts in one forward pass, and the request advances by every accepted token.
+ * Sections 2.3 and 5.3 name the costs of that step: suffix lookup, draft construction, verification and
+ * tree-mask handling.  This library is that step, entirely on the device:
+ *
+ *   war_index_build / war_index_append   the trajectory cache: suffix array + capped LCP over the corpus
+ *   war_draft                            longest-suffix match + frequency-ranked draft token tree
+ *   war_verify_attn                      tree-masked GQA decode attention over a paged bf16 KV cache
+ *   war_accept                           longest root path of the tree that equals the target's tokens
+ *
+ * Conventions shared by every call
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller owns every buffer it
+ *     passes; the library neither frees nor keeps them beyond the stream order of the call.  The library
+ *     owns only war_index_t objects (and build scratch it allocates and frees itself).
+ *   - Every call enqueues its work on `stream` and returns without synchronising the host, except
+ *     war_index_build / war_index_append (they size and free scratch) and war_device_status.
+ *   - Errors are return codes.  Nothing throws, aborts or traps.  Problems visible on the host (null
+ *     pointer, unsupported shape, capacity) are reported before anything is launched.  Problems only the
+ *     device can see (a malformed parent array, a page index outside the pool, a bounded wait that ran
+ *     out) set a sticky device status word, give the offending request an empty result (num_nodes = 0 /
+ *     accept_len = 0 / untouched attention rows) and let the kernel finish normally; read the word with
+ *     war_device_status.
+ *   - Slot convention: a request's draft tree has at most N slots.  Slot 0 is the root = the request's
+ *     last context token (parent -1).  Slots 1 .. num_nodes-1 are draft tokens with parent[j] < j.
+ *     N therefore counts the root.  Limits: N <= 64, P <= 32, topk <= 8, D == 128.
+ */
+#ifndef WAR_H_
+#define WAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    WAR_OK = 0,
+    WAR_ERR_INVALID_ARG = 1,   /* null pointer, negative size, shape outside the stated limits      */
+    WAR_ERR_OOM = 2,           /* a device allocation made by the library failed                      */
+    WAR_ERR_CAPACITY = 3,      /* the index cannot hold the requested number of tokens                */
+    WAR_ERR_CUDA = 4,          /* a CUDA runtime call or launch failed                                */
+    WAR_ERR_TIMEOUT = 5,       /* device status only: a bounded in-kernel wait expired                */
+    WAR_ERR_UNSUPPORTED = 6,   /* valid request this build has no kernel for (e.g. a strided pool)    */
+    WAR_ERR_BAD_TREE = 7,      /* device status only: parent[j] outside [0, j) or num_nodes > N       */
+    WAR_ERR_BAD_PAGE = 8       /* device status only: page table entry outside [0, num_pages)         */
+} war_status_t;
+
+typedef struct CUstream_st* war_stream_t;      /* same type as cudaStream_t */
+typedef struct war_index war_index_t;          /* opaque; lives on the device that was current at build */
+
+/* ------------------------------------------------------------------------------------------------
+ * Trajectory cache (paper Section 3.2: SuffixDecoding "caches token-sequence patterns from previously
+ * generated trajectories"; the "external update interface" adds newly generated trajectories after each
+ * RL step).  Trajectory t is d_tokens[h_offsets[t] .. h_offsets[t+1]); token ids lie in [0, vocab).
+ * Inside the index the trajectories are joined with one unique negative separator each, so no match ever
+ * straddles two trajectories.  The suffix array is ordered to depth max_depth (>= P + N of every later
+ * war_draft call; <= 128) and LCP values are capped there.
+ *   capacity_tokens  upper bound on (sum of trajectory lengths + number of trajectories) over the whole
+ *                    life of the index, appends included.
+ * war_index_append leaves the index answering every query exactly as a fresh build over the old
+ * trajectories followed by the new ones would.  Exceeding the capacity returns WAR_ERR_CAPACITY and
+ * leaves the index unchanged.  Both calls synchronise `stream` before returning.
+ * ------------------------------------------------------------------------------------------------ */
+war_status_t war_index_build(const int32_t* d_tokens, const int64_t* h_offsets, int32_t T,
+                             int32_t vocab, int32_t max_depth, int64_t capacity_tokens,
+                             war_stream_t stream, war_index_t** out);
+war_status_t war_index_append(war_index_t* ix, const int32_t* d_tokens, const int64_t* h_offsets, int32_t T,
+                              war_stream_t stream);
+
+typedef struct {
+    int64_t M;                  /* corpus entries in use: tokens + one separator per trajectory */
+    int64_t capacity_tokens;
+    int32_t T;                  /* trajectories */
+    int32_t vocab;
+    int32_t max_depth;
+    int32_t reserved;
+    const int32_t* d_corpus;    /* [M]  separator of trajectory t is -(t+1) */
+    const int32_t* d_sa;        /* [M]  suffix array */
+    const uint8_t* d_lcp;       /* [M]  min(lcp(sa[i-1], sa[i]), max_depth); lcp[0] = 0 */
+    const int32_t* d_bucket;    /* [vocab+1] sa interval of every one-token string */
+} war_index_info_t;
+war_status_t war_index_info(const war_index_t* ix, war_index_info_t* out);
+war_status_t war_index_destroy(war_index_t* ix);
+
+/* ------------------------------------------------------------------------------------------------
+ * Draft (paper Section 3: SuffixDecoding "matches the current token pattern against [the historical
+ * trajectories] to generate draft tokens").  For each of B requests:
+ *   match   the largest l <= min(P, tail_len) such that the last l tokens of the tail occur contiguously
+ *           inside one stored trajectory (0 if none);
+ *   tree    slot 0 = the last tail token, count[0] = occurrences of the matched string.  Every further slot
+ *           is one continuation token; count = occurrences of matched string + root path (every occurrence
+ *           counts, overlapping ones too).  Each slot offers its topk most frequent continuations (count
+ *           descending, token id ascending); slots are created best-first from all offers (count
+ *           descending, parent slot ascending, token id ascending) until N slots exist or no offer is left.
+ *           If match_len < max(1, min_match) the tree is the root alone.
+ * d_tail is int32 [B, P], right-aligned: the most recent token is d_tail[b, P-1]; only the last tail_len[b]
+ * entries are read.  Tail tokens outside [0, vocab) never match.
+ * Outputs: d_match_len [B], d_num_nodes [B], d_ids / d_parent / d_count [B, N] (d_count may be NULL).
+ * Unused slots are written as ids = -1, parent = -1, count = 0.
+ * ------------------------------------------------------------------------------------------------ */
+typedef struct {
+    int32_t B, P, N, topk, min_match;
+} war_draft_params_t;
+war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, const int32_t* d_tail_len,
+                       const war_draft_params_t* params,
+                       int32_t* d_match_len, int32_t* d_num_nodes,
+                       int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Verification attention (paper Section 3.2: the predicted tokens "are then verified by the target model"
+ * in "a single forward pass"; Sections 2.3 / 5.3: this needs auxiliary attention-mask / tree-mask handling).
+ * For request b, slot j < num_nodes[b], query head h (kv head h / (Hq/Hkv)):
+ *     visible = { 0 .. prefix_len[b]-1 }  U  { prefix_len[b] + a : a == j or a is an ancestor of j }
+ *     out[b,j,h,:] = sum_c softmax_c(scale * <q[b,j,h,:], K[c,:]>) * V[c,:]      (c over visible)
+ *     lse[b,j,h]   = natural-log sum of exp of the same logits
+ * bf16 inputs, fp32 accumulation, bf16 out, fp32 lse.  The tree mask is derived from d_parent on the device.
+ * KV layout: logical position p of request b is row p % page_size of physical page
+ * d_page_table[b, p / page_size]; slot a's K/V are at logical position prefix_len[b] + a (the caller writes
+ * them before the call).  Pools are bf16 [num_pages, Hkv, page_size, D]; k_strides / v_strides give the
+ * element strides of (page, head, token, d).  This build requires the contiguous head-major layout
+ * (strides = {Hkv*page_size*D, page_size*D, D, 1}), page_size 16 or 32, D == 128, Hq % Hkv == 0,
+ * (Hq/Hkv) * N <= 512; anything else returns WAR_ERR_UNSUPPORTED / WAR_ERR_INVALID_ARG.
+ * Rows j >= num_nodes[b] of d_out / d_lse are left untouched.
+ * d_workspace: war_verify_attn_workspace_bytes(params) bytes of device memory, 256-byte aligned, private to
+ * the call while it runs (split-KV partial results and the work list live there).
+ *   kernel: 0 = default (tensor-core path), 1 = plain CUDA-core path kept for A/B checks.
+ * ------------------------------------------------------------------------------------------------ */
+typedef struct {
+    int32_t B, N, Hq, Hkv, D, page_size, max_pages_per_req, kernel;
+    int64_t num_pages;
+    float scale;
+    int32_t reserved;
+    int64_t k_strides[4], v_strides[4];
+} war_attn_params_t;
+size_t war_verify_attn_workspace_bytes(const war_attn_params_t* params);
+war_status_t war_verify_attn(const void* d_q, const void* d_kpool, const void* d_vpool,
+                             const int32_t* d_page_table, const int32_t* d_prefix_len,
+                             const int32_t* d_num_nodes, const int32_t* d_parent,
+                             const war_attn_params_t* params, void* d_workspace,
+                             void* d_out, float* d_lse, war_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Accept (paper Section 2.3: drafts are verified "while preserving the target output distribution";
+ * Section 3.2: the rollout advances "by multiple tokens ... when the drafts are accepted").  The caller
+ * supplies the target model's own token choices; a draft slot is accepted iff every slot on its root path
+ * equals the target's choice there.
+ *   target_mode 0: d_target_ids[b, p] is the token the target emits AFTER slot p; slot j matches iff
+ *                  ids[j] == target[parent[j]].  bonus = target[result slot].
+ *   target_mode 1: slot j matches iff ids[j] == target[j].  bonus = -1.
+ * Result slot = deepest slot whose whole root path matches (ties: lowest slot).  d_accept_len [B] = its depth,
+ * d_accept_path [B, N] = the slots from the root's child down to it, padded with -1, d_bonus [B].
+ * ------------------------------------------------------------------------------------------------ */
+war_status_t war_accept(const int32_t* d_ids, const int32_t* d_parent, const int32_t* d_num_nodes,
+                        const int32_t* d_target_ids, int32_t B, int32_t N, int32_t target_mode,
+                        int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, war_stream_t stream);
+
+/* Reads and clears the sticky device status word (synchronises `stream`).  *h_status receives a
+ * war_status_t value: WAR_OK, or the first device-side problem seen since the last read. */
+war_status_t war_device_status(war_stream_t stream, int32_t* h_status);
+const char* war_status_string(war_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WAR_H_ */

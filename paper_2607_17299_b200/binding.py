@@ -1,0 +1,222 @@
+"""Thin Python binding of libwar.so: argument marshalling only.
+
+Every function here has the name and the meaning of the C entry point it wraps (see include/war.h); tensors are
+torch CUDA tensors used as device buffers, and the current torch stream is the stream of the call.  Nothing is
+computed on the Python side, and there is no fallback: if the library has not been built, importing this module
+raises."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libwar.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_17299_b200.build` "
+                      "(there is no CPU or PyTorch fallback for this library)")
+_lib = C.CDLL(LIB_PATH)
+
+WAR_OK = 0
+STATUS_NAMES = {0: "WAR_OK", 1: "WAR_ERR_INVALID_ARG", 2: "WAR_ERR_OOM", 3: "WAR_ERR_CAPACITY", 4: "WAR_ERR_CUDA",
+                5: "WAR_ERR_TIMEOUT", 6: "WAR_ERR_UNSUPPORTED", 7: "WAR_ERR_BAD_TREE", 8: "WAR_ERR_BAD_PAGE"}
+
+EXPORTS = ["war_index_build", "war_index_append", "war_index_info", "war_index_destroy", "war_draft",
+           "war_verify_attn_workspace_bytes", "war_verify_attn", "war_accept", "war_device_status",
+           "war_status_string"]
+
+
+class WarError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        self.code = code
+        super().__init__(f"{fn} returned {STATUS_NAMES.get(code, code)}: {status_string(code)}")
+
+
+class IndexInfo(C.Structure):
+    _fields_ = [("M", C.c_int64), ("capacity_tokens", C.c_int64), ("T", C.c_int32), ("vocab", C.c_int32),
+                ("max_depth", C.c_int32), ("reserved", C.c_int32), ("d_corpus", C.c_void_p), ("d_sa", C.c_void_p),
+                ("d_lcp", C.c_void_p), ("d_bucket", C.c_void_p)]
+
+
+class DraftParams(C.Structure):
+    _fields_ = [("B", C.c_int32), ("P", C.c_int32), ("N", C.c_int32), ("topk", C.c_int32), ("min_match", C.c_int32)]
+
+
+class AttnParams(C.Structure):
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("D", C.c_int32),
+                ("page_size", C.c_int32), ("max_pages_per_req", C.c_int32), ("kernel", C.c_int32),
+                ("num_pages", C.c_int64), ("scale", C.c_float), ("reserved", C.c_int32),
+                ("k_strides", C.c_int64 * 4), ("v_strides", C.c_int64 * 4)]
+
+
+_lib.war_status_string.restype = C.c_char_p
+_lib.war_status_string.argtypes = [C.c_int]
+_lib.war_index_build.restype = C.c_int
+_lib.war_index_build.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_void_p,
+                                 C.POINTER(C.c_void_p)]
+_lib.war_index_append.restype = C.c_int
+_lib.war_index_append.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+_lib.war_index_info.restype = C.c_int
+_lib.war_index_info.argtypes = [C.c_void_p, C.POINTER(IndexInfo)]
+_lib.war_index_destroy.restype = C.c_int
+_lib.war_index_destroy.argtypes = [C.c_void_p]
+_lib.war_draft.restype = C.c_int
+_lib.war_draft.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(DraftParams)] + [C.c_void_p] * 6
+_lib.war_verify_attn_workspace_bytes.restype = C.c_size_t
+_lib.war_verify_attn_workspace_bytes.argtypes = [C.POINTER(AttnParams)]
+_lib.war_verify_attn.restype = C.c_int
+_lib.war_verify_attn.argtypes = [C.c_void_p] * 7 + [C.POINTER(AttnParams)] + [C.c_void_p] * 4
+_lib.war_accept.restype = C.c_int
+_lib.war_accept.argtypes = [C.c_void_p] * 4 + [C.c_int32] * 3 + [C.c_void_p] * 4
+_lib.war_device_status.restype = C.c_int
+_lib.war_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
+
+
+def status_string(code: int) -> str:
+    return _lib.war_status_string(int(code)).decode()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("device buffers must be contiguous CUDA tensors")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _check(fn: str, code: int) -> None:
+    if code != WAR_OK:
+        raise WarError(fn, code)
+
+
+class Index:
+    """Owner of a war_index_t*."""
+
+    def __init__(self, handle: int):
+        self._h = C.c_void_p(handle)
+
+    @property
+    def handle(self) -> C.c_void_p:
+        if not self._h:
+            raise ValueError("index already destroyed")
+        return self._h
+
+    def destroy(self) -> None:
+        if self._h:
+            _lib.war_index_destroy(self._h)
+            self._h = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def _offsets(h_offsets) -> np.ndarray:
+    off = np.ascontiguousarray(np.asarray(h_offsets, dtype=np.int64))
+    if off.ndim != 1 or len(off) < 1:
+        raise ValueError("h_offsets must be int64 [T+1]")
+    return off
+
+
+def war_index_build(d_tokens: torch.Tensor, h_offsets, vocab: int, max_depth: int, capacity_tokens: int) -> Index:
+    off = _offsets(h_offsets)
+    out = C.c_void_p(None)
+    code = _lib.war_index_build(_ptr(d_tokens, torch.int32), off.ctypes.data, len(off) - 1, vocab, max_depth,
+                                capacity_tokens, _stream(), C.byref(out))
+    _check("war_index_build", code)
+    return Index(out.value)
+
+
+def war_index_append(ix: Index, d_tokens: torch.Tensor, h_offsets) -> None:
+    off = _offsets(h_offsets)
+    _check("war_index_append", _lib.war_index_append(ix.handle, _ptr(d_tokens, torch.int32), off.ctypes.data,
+                                                     len(off) - 1, _stream()))
+
+
+def war_index_info(ix: Index) -> IndexInfo:
+    info = IndexInfo()
+    _check("war_index_info", _lib.war_index_info(ix.handle, C.byref(info)))
+    return info
+
+
+def war_index_destroy(ix: Index) -> None:
+    ix.destroy()
+
+
+def war_draft(ix: Index, d_tail: torch.Tensor, d_tail_len: torch.Tensor, N: int, topk: int, min_match: int,
+              d_match_len: torch.Tensor, d_num_nodes: torch.Tensor, d_ids: torch.Tensor, d_parent: torch.Tensor,
+              d_count: Optional[torch.Tensor]) -> None:
+    B, P = d_tail.shape
+    p = DraftParams(B, P, N, topk, min_match)
+    code = _lib.war_draft(ix.handle, _ptr(d_tail, torch.int32), _ptr(d_tail_len, torch.int32), C.byref(p),
+                          _ptr(d_match_len, torch.int32), _ptr(d_num_nodes, torch.int32), _ptr(d_ids, torch.int32),
+                          _ptr(d_parent, torch.int32), _ptr(d_count, torch.int32), _stream())
+    _check("war_draft", code)
+
+
+def attn_params(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, page_table: torch.Tensor, scale: float,
+                kernel: int = 0) -> AttnParams:
+    B, N, Hq, D = q.shape
+    num_pages, Hkv, pg, _ = k_pool.shape
+    p = AttnParams()
+    p.B, p.N, p.Hq, p.Hkv, p.D, p.page_size = B, N, Hq, Hkv, D, pg
+    p.max_pages_per_req = page_table.shape[1]
+    p.kernel = kernel
+    p.num_pages = num_pages
+    p.scale = scale
+    for i in range(4):
+        p.k_strides[i] = k_pool.stride(i)
+        p.v_strides[i] = v_pool.stride(i)
+    return p
+
+
+def war_verify_attn_workspace_bytes(params: AttnParams) -> int:
+    return int(_lib.war_verify_attn_workspace_bytes(C.byref(params)))
+
+
+def war_verify_attn(d_q: torch.Tensor, d_kpool: torch.Tensor, d_vpool: torch.Tensor, d_page_table: torch.Tensor,
+                    d_prefix_len: torch.Tensor, d_num_nodes: torch.Tensor, d_parent: torch.Tensor, params: AttnParams,
+                    d_workspace: torch.Tensor, d_out: torch.Tensor, d_lse: Optional[torch.Tensor]) -> None:
+    for t in (d_kpool, d_vpool):
+        if not t.is_cuda or t.dtype != torch.bfloat16:
+            raise ValueError("pools must be bf16 CUDA tensors")
+    code = _lib.war_verify_attn(_ptr(d_q, torch.bfloat16), d_kpool.data_ptr(), d_vpool.data_ptr(),
+                                _ptr(d_page_table, torch.int32), _ptr(d_prefix_len, torch.int32),
+                                _ptr(d_num_nodes, torch.int32), _ptr(d_parent, torch.int32), C.byref(params),
+                                _ptr(d_workspace), _ptr(d_out, torch.bfloat16), _ptr(d_lse, torch.float32), _stream())
+    _check("war_verify_attn", code)
+
+
+def war_accept(d_ids: torch.Tensor, d_parent: torch.Tensor, d_num_nodes: torch.Tensor, d_target_ids: torch.Tensor,
+               target_mode: int, d_accept_len: torch.Tensor, d_accept_path: torch.Tensor, d_bonus: torch.Tensor) -> None:
+    B, N = d_ids.shape
+    code = _lib.war_accept(_ptr(d_ids, torch.int32), _ptr(d_parent, torch.int32), _ptr(d_num_nodes, torch.int32),
+                           _ptr(d_target_ids, torch.int32), B, N, target_mode, _ptr(d_accept_len, torch.int32),
+                           _ptr(d_accept_path, torch.int32), _ptr(d_bonus, torch.int32), _stream())
+    _check("war_accept", code)
+
+
+def war_device_status() -> int:
+    v = C.c_int32(0)
+    _check("war_device_status", _lib.war_device_status(_stream(), C.byref(v)))
+    return int(v.value)
+
+
+def new_workspace(params: AttnParams, device) -> torch.Tensor:
+    """A device buffer of the size war_verify_attn asks for (torch's allocator returns 512-byte aligned blocks)."""
+    n = war_verify_attn_workspace_bytes(params)
+    if n == 0:
+        raise WarError("war_verify_attn_workspace_bytes", 6)
+    return torch.empty(n, dtype=torch.uint8, device=device)

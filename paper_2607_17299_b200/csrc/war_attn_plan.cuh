@@ -1,0 +1,63 @@
+// Work decomposition of the verify-attention call (library-internal).
+//
+// A unit = (request, kv head, row block, KV chunk).  The rows of a unit are the (slot, query head of the group)
+// pairs r = slot * G + g of one kv head, cut into row blocks of at most kRowBlock rows; its chunk is a range of
+// 128-key tiles.  A tiny planning kernel cuts every request into chunks so that about kTargetUnits units exist,
+// orders requests longest-first and writes the unit table; the attention kernel's CTAs pull units from an atomic
+// counter; units of a split request leave (max, sum, unnormalised output) partials that a combine kernel merges
+// in chunk order.  Everything lives in the caller's workspace, so no call allocates.
+#pragma once
+#include <stdint.h>
+#include "war.h"
+
+constexpr int kTileKeys = 128;          // planning granularity in keys
+constexpr int kRowBlock = 128;          // query rows per unit
+constexpr int kTargetUnits = 148 * 8;   // aim: several units per SM
+constexpr int kMinChunkTiles = 8;       // never cut finer than 1024 keys
+constexpr int kMaxPlanB = 4096;
+
+struct AttnUnit {
+    int req, kvh, rb, tile_begin, tile_end, n_chunks, chunk, pad;
+};
+struct AttnReq {
+    int base_unit, n_chunks, n_tiles, n_nodes;
+};
+
+struct AttnWorkspace {
+    int* counters;       // [0] next unit to hand out, [1] number of units, [2] chunk size in tiles
+    AttnReq* req;        // [B]
+    uint64_t* anc;       // [B, N] bit a of anc[b, j]: slot a is j or an ancestor of j
+    AttnUnit* units;     // [max_units]
+    float* part_ml;      // [max_units, rows, 2]  running max (log2 domain) and sum
+    float* part_o;       // [max_units, rows, D]  unnormalised output
+    int max_units, rows, row_blocks;
+    size_t bytes;
+};
+
+inline AttnWorkspace war_attn_workspace_layout(const war_attn_params_t* p, void* base) {
+    AttnWorkspace w;
+    const int G = p->Hq / p->Hkv;
+    const int R = G * p->N;
+    w.rows = R < kRowBlock ? R : kRowBlock;
+    w.row_blocks = (R + kRowBlock - 1) / kRowBlock;
+    w.max_units = kTargetUnits + p->B * p->Hkv * w.row_blocks;
+    auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    size_t at = 0;
+    char* b = (char*)base;
+    w.counters = (int*)(b + at); at += align(64 * sizeof(int));
+    w.req = (AttnReq*)(b + at); at += align(sizeof(AttnReq) * (size_t)p->B);
+    w.anc = (uint64_t*)(b + at); at += align(sizeof(uint64_t) * (size_t)p->B * p->N);
+    w.units = (AttnUnit*)(b + at); at += align(sizeof(AttnUnit) * (size_t)w.max_units);
+    w.part_ml = (float*)(b + at); at += align(sizeof(float) * 2 * (size_t)w.max_units * w.rows);
+    w.part_o = (float*)(b + at); at += align(sizeof(float) * (size_t)w.max_units * w.rows * p->D);
+    w.bytes = at;
+    return w;
+}
+
+// Launchers implemented per kernel family.  Both consume the same plan and leave the same partials.
+war_status_t war_attn_launch_simple(const void* q, const void* k, const void* v, const int32_t* page_table,
+                                    const int32_t* prefix_len, const war_attn_params_t* p, const AttnWorkspace& w,
+                                    void* out, float* lse, int* status_word, cudaStream_t s);
+war_status_t war_attn_launch_sm100(const void* q, const void* k, const void* v, const int32_t* page_table,
+                                   const int32_t* prefix_len, const war_attn_params_t* p, const AttnWorkspace& w,
+                                   void* out, float* lse, int* status_word, cudaStream_t s);

@@ -1,0 +1,299 @@
+// Trajectory cache: suffix array + capped LCP + first-token buckets over the separator-joined corpus.
+//
+// Only ordering to depth max_depth (<= 128) is ever needed by the draft kernel (it compares at most P pattern
+// tokens and descends at most N-1 further), so prefix doubling stops after ceil(log2(max_depth)) rounds.
+// Round r sorts 64-bit keys (rank of the first 2^r tokens, rank of the next 2^r tokens) with a device radix
+// sort and re-ranks by adjacent difference + scan.  Suffixes that still tie after the last round keep the
+// order the stable sort left them in; no output of the library depends on that order.
+#include <cub/cub.cuh>
+#include <new>
+#include "war_common.cuh"
+#include "war_index.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+struct MaxOp {
+    __device__ __forceinline__ uint32_t operator()(uint32_t a, uint32_t b) const { return a > b ? a : b; }
+};
+
+// corpus[dst_base + off[t] + t + i] = tokens[off[t] + i]; separator -(t0 + t + 1) after each trajectory.
+__global__ void scatter_corpus_kernel(const int32_t* __restrict__ tokens, const int64_t* __restrict__ off, int T,
+                                      int t0, int64_t dst_base, int32_t* __restrict__ corpus, int64_t n_out) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_out) return;
+    // trajectory t covers output positions [off[t] + t, off[t+1] + t]; the last one is its separator
+    int lo = 0, hi = T - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (off[mid] + mid <= i) lo = mid; else hi = mid - 1;
+    }
+    const int t = lo;
+    const int64_t local = i - (off[t] + t);
+    const int64_t len = off[t + 1] - off[t];
+    corpus[dst_base + i] = local < len ? tokens[off[t] + local] : -(t0 + t + 1);
+}
+
+// first-round key: separators (negative, unique) below every token
+__global__ void init_keys_kernel(const int32_t* __restrict__ corpus, int64_t M, int T, uint32_t* __restrict__ key,
+                                 int32_t* __restrict__ sa) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M) return;
+    key[i] = (uint32_t)(corpus[i] + T);
+    sa[i] = (int32_t)i;
+}
+
+__global__ void flag32_kernel(const uint32_t* __restrict__ key, int64_t M, uint32_t* __restrict__ flag) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M) return;
+    flag[i] = (i > 0 && key[i] != key[i - 1]) ? (uint32_t)i : 0u;
+}
+
+__global__ void flag64_kernel(const uint64_t* __restrict__ key, int64_t M, uint32_t* __restrict__ flag) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M) return;
+    flag[i] = (i > 0 && key[i] != key[i - 1]) ? (uint32_t)i : 0u;
+}
+
+// rank[sa[i]] = index of the first suffix of i's group
+__global__ void scatter_rank_kernel(const int32_t* __restrict__ sa, const uint32_t* __restrict__ group_start, int64_t M,
+                                    uint32_t* __restrict__ rank) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M) return;
+    rank[sa[i]] = group_start[i];
+}
+
+__global__ void make_pair_keys_kernel(const int32_t* __restrict__ sa, const uint32_t* __restrict__ rank, int64_t M, int64_t h,
+                                      uint64_t* __restrict__ key) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M) return;
+    const int64_t s = sa[i];
+    const uint64_t hi = rank[s];
+    const uint64_t lo = (s + h < M) ? (uint64_t)rank[s + h] + 1u : 0u;
+    key[i] = (hi << 32) | lo;
+}
+
+__global__ void lcp_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, int64_t M, int max_depth,
+                           uint8_t* __restrict__ lcp) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M) return;
+    int l = 0;
+    if (i > 0) {
+        const int64_t a = sa[i - 1], b = sa[i];
+        // separators are unique, so the comparison stops at the first one; the last corpus entry is a separator
+        while (l < max_depth && a + l < M && b + l < M && corpus[a + l] == corpus[b + l]) ++l;
+    }
+    lcp[i] = (uint8_t)l;
+}
+
+__global__ void histogram_kernel(const int32_t* __restrict__ corpus, int64_t M, int vocab, uint32_t* __restrict__ hist) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M) return;
+    const int32_t c = corpus[i];
+    if (c >= 0 && c < vocab) atomicAdd(&hist[c], 1u);
+}
+
+// bucket[v] = T + sum_{u<v} hist[u]  (the T separators sort first); single block
+__global__ void bucket_scan_kernel(const uint32_t* __restrict__ hist, int vocab, int T, int32_t* __restrict__ bucket) {
+    typedef cub::BlockScan<uint32_t, 1024> Scan;
+    __shared__ typename Scan::TempStorage tmp;
+    __shared__ uint32_t carry;
+    if (threadIdx.x == 0) carry = (uint32_t)T;
+    __syncthreads();
+    for (int base = 0; base < vocab + 1; base += 1024) {
+        const int v = base + threadIdx.x;
+        const uint32_t x = v < vocab ? hist[v] : 0u;
+        uint32_t excl, total;
+        Scan(tmp).ExclusiveSum(x, excl, total);
+        if (v <= vocab) bucket[v] = (int32_t)(carry + excl);
+        __syncthreads();
+        if (threadIdx.x == 0) carry += total;
+        __syncthreads();
+    }
+}
+
+struct Scratch {
+    void* p = nullptr;
+    ~Scratch() { if (p) cudaFree(p); }
+};
+
+inline dim3 grid_for(int64_t n) { return dim3((unsigned)((n + kThreads - 1) / kThreads)); }
+
+// (Re)builds sa / lcp / bucket from ix->corpus[0 .. M).
+war_status_t rebuild(war_index* ix, cudaStream_t s) {
+    const int64_t M = ix->M;
+    if (M == 0) {
+        WAR_CUDA_TRY(cudaMemsetAsync(ix->bucket, 0, sizeof(int32_t) * (ix->vocab + 1), s));
+        return WAR_OK;
+    }
+    const int n = (int)M;
+    // scratch: key64 x2, val x2, rank, flag, hist, cub temp
+    size_t temp_sort64 = 0, temp_sort32 = 0, temp_scan = 0;
+    {
+        cub::DoubleBuffer<uint64_t> k64(nullptr, nullptr);
+        cub::DoubleBuffer<uint32_t> k32(nullptr, nullptr);
+        cub::DoubleBuffer<int32_t> v(nullptr, nullptr);
+        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(nullptr, temp_sort64, k64, v, n, 0, 64, s));
+        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(nullptr, temp_sort32, k32, v, n, 0, 32, s));
+        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(nullptr, temp_scan, (uint32_t*)nullptr, (uint32_t*)nullptr, MaxOp(), n, s));
+    }
+    size_t temp_bytes = temp_sort64 > temp_sort32 ? temp_sort64 : temp_sort32;
+    if (temp_scan > temp_bytes) temp_bytes = temp_scan;
+    auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t b_key = align(sizeof(uint64_t) * M), b_val = align(sizeof(int32_t) * M), b_u32 = align(sizeof(uint32_t) * M);
+    const size_t b_hist = align(sizeof(uint32_t) * (ix->vocab + 1));
+    const size_t total = 2 * b_key + 2 * b_val + 2 * b_u32 + b_hist + align(temp_bytes);
+    Scratch scratch;
+    WAR_CUDA_TRY(cudaMalloc(&scratch.p, total));
+    char* at = (char*)scratch.p;
+    uint64_t* key_a = (uint64_t*)at; at += b_key;
+    uint64_t* key_b = (uint64_t*)at; at += b_key;
+    int32_t* val_a = (int32_t*)at; at += b_val;
+    int32_t* val_b = (int32_t*)at; at += b_val;
+    uint32_t* rank = (uint32_t*)at; at += b_u32;
+    uint32_t* flag = (uint32_t*)at; at += b_u32;
+    uint32_t* hist = (uint32_t*)at; at += b_hist;
+    void* temp = at;
+
+    int sym_bits = 1;
+    while (((int64_t)1 << sym_bits) < (int64_t)ix->vocab + ix->T) ++sym_bits;
+    int pos_bits = 1;
+    while (((int64_t)1 << pos_bits) < M + 1) ++pos_bits;
+
+    // round 0: order by the first token
+    cub::DoubleBuffer<int32_t> val(val_a, val_b);
+    {
+        cub::DoubleBuffer<uint32_t> k32((uint32_t*)key_a, (uint32_t*)key_b);
+        init_keys_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, M, ix->T, k32.Current(), val.Current());
+        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(temp, temp_bytes, k32, val, n, 0, sym_bits, s));
+        flag32_kernel<<<grid_for(M), kThreads, 0, s>>>(k32.Current(), M, flag);
+        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, flag, flag, MaxOp(), n, s));
+        scatter_rank_kernel<<<grid_for(M), kThreads, 0, s>>>(val.Current(), flag, M, rank);
+    }
+    for (int64_t h = 1; h < ix->max_depth; h <<= 1) {
+        cub::DoubleBuffer<uint64_t> k64(key_a, key_b);
+        make_pair_keys_kernel<<<grid_for(M), kThreads, 0, s>>>(val.Current(), rank, M, h, k64.Current());
+        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(temp, temp_bytes, k64, val, n, 0, 32 + pos_bits, s));
+        flag64_kernel<<<grid_for(M), kThreads, 0, s>>>(k64.Current(), M, flag);
+        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, flag, flag, MaxOp(), n, s));
+        scatter_rank_kernel<<<grid_for(M), kThreads, 0, s>>>(val.Current(), flag, M, rank);
+    }
+    WAR_CUDA_TRY(cudaMemcpyAsync(ix->sa, val.Current(), sizeof(int32_t) * M, cudaMemcpyDeviceToDevice, s));
+    lcp_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, ix->sa, M, ix->max_depth, ix->lcp);
+    WAR_CUDA_TRY(cudaMemsetAsync(hist, 0, b_hist, s));
+    histogram_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, M, ix->vocab, hist);
+    bucket_scan_kernel<<<1, 1024, 0, s>>>(hist, ix->vocab, ix->T, ix->bucket);
+    WAR_LAUNCH_CHECK();
+    WAR_CUDA_TRY(cudaStreamSynchronize(s));
+    return WAR_OK;
+}
+
+war_status_t check_offsets(const int64_t* h_offsets, int32_t T) {
+    if (T < 0) return WAR_ERR_INVALID_ARG;
+    if (T > 0 && !h_offsets) return WAR_ERR_INVALID_ARG;
+    for (int t = 0; t < T; ++t)
+        if (h_offsets[t + 1] < h_offsets[t]) return WAR_ERR_INVALID_ARG;
+    if (T > 0 && h_offsets[0] < 0) return WAR_ERR_INVALID_ARG;
+    return WAR_OK;
+}
+
+// Adds T trajectories (device tokens, host offsets) behind the current corpus content.
+war_status_t add_trajectories(war_index* ix, const int32_t* d_tokens, const int64_t* h_offsets, int32_t T, cudaStream_t s) {
+    if (T == 0) return WAR_OK;
+    const int64_t n_tok = h_offsets[T] - h_offsets[0];
+    const int64_t n_out = n_tok + T;
+    if (ix->M + n_out > ix->capacity || ix->M + n_out >= ((int64_t)1 << 31) - 256 || (int64_t)ix->T + T >= ((int64_t)1 << 30))
+        return WAR_ERR_CAPACITY;
+    if (n_tok > 0 && !d_tokens) return WAR_ERR_INVALID_ARG;
+    // offsets relative to the first trajectory of this batch
+    int64_t* rel = new (std::nothrow) int64_t[T + 1];
+    if (!rel) return WAR_ERR_OOM;
+    for (int t = 0; t <= T; ++t) rel[t] = h_offsets[t] - h_offsets[0];
+    Scratch off;
+    cudaError_t e = cudaMalloc(&off.p, sizeof(int64_t) * (T + 1));
+    if (e == cudaSuccess) e = cudaMemcpyAsync(off.p, rel, sizeof(int64_t) * (T + 1), cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) {
+        scatter_corpus_kernel<<<grid_for(n_out), kThreads, 0, s>>>(d_tokens + h_offsets[0], (const int64_t*)off.p, T, ix->T,
+                                                                  ix->M, ix->corpus, n_out);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    delete[] rel;
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return e == cudaErrorMemoryAllocation ? WAR_ERR_OOM : WAR_ERR_CUDA; }
+    ix->M += n_out;
+    ix->T += T;
+    return WAR_OK;
+}
+
+}  // namespace
+
+extern "C" war_status_t war_index_build(const int32_t* d_tokens, const int64_t* h_offsets, int32_t T, int32_t vocab,
+                                        int32_t max_depth, int64_t capacity_tokens, war_stream_t stream,
+                                        war_index_t** out) {
+    if (!out) return WAR_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (vocab < 1 || max_depth < 1 || max_depth > 128 || capacity_tokens < 0) return WAR_ERR_INVALID_ARG;
+    war_status_t st = check_offsets(h_offsets, T);
+    if (st != WAR_OK) return st;
+    if (capacity_tokens >= ((int64_t)1 << 31) - 256) return WAR_ERR_CAPACITY;
+    war_index* ix = new (std::nothrow) war_index();
+    if (!ix) return WAR_ERR_OOM;
+    ix->vocab = vocab;
+    ix->max_depth = max_depth;
+    ix->capacity = capacity_tokens;
+    cudaGetDevice(&ix->device);
+    const int64_t cap = capacity_tokens > 0 ? capacity_tokens : 1;
+    cudaError_t e = cudaMalloc((void**)&ix->corpus, sizeof(int32_t) * (cap + 128));   // +128: readable slack behind the last separator
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ix->sa, sizeof(int32_t) * cap);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ix->lcp, cap + 64);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ix->bucket, sizeof(int32_t) * (vocab + 1));
+    if (e == cudaSuccess) e = cudaMemsetAsync(ix->corpus, 0xff, sizeof(int32_t) * (cap + 128), stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ix->lcp, 0, cap + 64, stream);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        war_index_destroy(ix);
+        return e == cudaErrorMemoryAllocation ? WAR_ERR_OOM : WAR_ERR_CUDA;
+    }
+    st = add_trajectories(ix, d_tokens, h_offsets, T, stream);
+    if (st == WAR_OK) st = rebuild(ix, stream);
+    if (st != WAR_OK) { war_index_destroy(ix); return st; }
+    *out = ix;
+    return WAR_OK;
+}
+
+extern "C" war_status_t war_index_append(war_index_t* ix, const int32_t* d_tokens, const int64_t* h_offsets, int32_t T,
+                                         war_stream_t stream) {
+    if (!ix) return WAR_ERR_INVALID_ARG;
+    war_status_t st = check_offsets(h_offsets, T);
+    if (st != WAR_OK) return st;
+    if (T == 0) return WAR_OK;
+    st = add_trajectories(ix, d_tokens, h_offsets, T, stream);
+    if (st != WAR_OK) return st;
+    return rebuild(ix, stream);
+}
+
+extern "C" war_status_t war_index_info(const war_index_t* ix, war_index_info_t* out) {
+    if (!ix || !out) return WAR_ERR_INVALID_ARG;
+    out->M = ix->M;
+    out->capacity_tokens = ix->capacity;
+    out->T = ix->T;
+    out->vocab = ix->vocab;
+    out->max_depth = ix->max_depth;
+    out->reserved = 0;
+    out->d_corpus = ix->corpus;
+    out->d_sa = ix->sa;
+    out->d_lcp = ix->lcp;
+    out->d_bucket = ix->bucket;
+    return WAR_OK;
+}
+
+extern "C" war_status_t war_index_destroy(war_index_t* ix) {
+    if (!ix) return WAR_OK;
+    if (ix->corpus) cudaFree(ix->corpus);
+    if (ix->sa) cudaFree(ix->sa);
+    if (ix->lcp) cudaFree(ix->lcp);
+    if (ix->bucket) cudaFree(ix->bucket);
+    delete ix;
+    return WAR_OK;
+}

@@ -1,0 +1,68 @@
+"""Helpers shared by the GPU parity tests: run the library through its C-ABI binding and hand back numpy."""
+import numpy as np
+import torch
+
+
+def dev():
+    return torch.device("cuda:0")
+
+
+def build_index(war, tokens: np.ndarray, offsets: np.ndarray, vocab: int, max_depth: int = 96, capacity=None):
+    d_tok = torch.from_numpy(np.ascontiguousarray(tokens, dtype=np.int32)).to(dev())
+    cap = int(len(tokens) + len(offsets) - 1) if capacity is None else capacity
+    return war.war_index_build(d_tok, offsets, vocab, max_depth, cap)
+
+
+def run_draft(war, ix, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, min_match: int = 1, with_count=True):
+    B = tails.shape[0]
+    d = dev()
+    t = torch.from_numpy(np.ascontiguousarray(tails, dtype=np.int32)).to(d)
+    tl = torch.from_numpy(np.ascontiguousarray(tail_len, dtype=np.int32)).to(d)
+    ml = torch.full((B,), -7, dtype=torch.int32, device=d)
+    nn = torch.full((B,), -7, dtype=torch.int32, device=d)
+    ids = torch.full((B, N), -7, dtype=torch.int32, device=d)
+    par = torch.full((B, N), -7, dtype=torch.int32, device=d)
+    cnt = torch.full((B, N), -7, dtype=torch.int32, device=d) if with_count else None
+    war.war_draft(ix, t, tl, N, k, min_match, ml, nn, ids, par, cnt)
+    torch.cuda.synchronize()
+    out = [ml.cpu().numpy(), nn.cpu().numpy(), ids.cpu().numpy(), par.cpu().numpy()]
+    out.append(cnt.cpu().numpy() if with_count else None)
+    return out
+
+
+def run_attn(war, a, num_nodes: np.ndarray, parent: np.ndarray, scale: float, kernel: int = 0, fill: float = 7.0):
+    """`a` is workloads.AttnInputs already on the device.  Returns (out fp32 numpy [B,N,Hq,D], lse numpy [B,N,Hq])."""
+    d = dev()
+    params = war.attn_params(a.q, a.k_pool, a.v_pool, a.page_table, scale, kernel)
+    ws = war.new_workspace(params, d)
+    out = torch.full(a.q.shape, fill, dtype=torch.bfloat16, device=d)
+    lse = torch.full(a.q.shape[:3], fill, dtype=torch.float32, device=d)
+    nn = torch.from_numpy(np.ascontiguousarray(num_nodes, dtype=np.int32)).to(d)
+    par = torch.from_numpy(np.ascontiguousarray(parent, dtype=np.int32)).to(d)
+    war.war_verify_attn(a.q, a.k_pool, a.v_pool, a.page_table, a.prefix_len, nn, par, params, ws, out, lse)
+    torch.cuda.synchronize()
+    return out.float().cpu().numpy(), lse.cpu().numpy(), out
+
+
+def run_accept(war, ids, parent, num_nodes, target, mode):
+    d = dev()
+    B, N = ids.shape
+    t = lambda x: torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).to(d)
+    alen = torch.full((B,), -7, dtype=torch.int32, device=d)
+    path = torch.full((B, N), -7, dtype=torch.int32, device=d)
+    bonus = torch.full((B,), -7, dtype=torch.int32, device=d)
+    war.war_accept(t(ids), t(parent), t(num_nodes), t(target), mode, alen, path, bonus)
+    torch.cuda.synchronize()
+    return alen.cpu().numpy(), path.cpu().numpy(), bonus.cpu().numpy()
+
+
+def assert_attention_close(got, got_lse, want, want_lse, n):
+    """The stated bar (atol 1e-2 / rtol 1e-2 after casting both sides to fp32) plus the sharper per-row checks:
+    with N(0,1) inputs at long context the outputs are ~1e-2 in size, so the absolute bar alone proves little."""
+    want32 = want.astype(np.float32)
+    g = got[:n]
+    np.testing.assert_allclose(g, want32, atol=1e-2, rtol=1e-2)
+    num = np.sqrt(((g.astype(np.float64) - want) ** 2).sum(axis=-1))
+    den = np.sqrt((want ** 2).sum(axis=-1)) + 1e-30
+    assert (num / den).max() < 1e-2, f"relative L2 error {float((num / den).max()):.3e}"
+    np.testing.assert_allclose(got_lse[:n], want_lse.astype(np.float32), atol=1e-3, rtol=1e-4)

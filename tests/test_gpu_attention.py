@@ -1,0 +1,172 @@
+"""GPU parity: tree-masked verify attention against the fp64 checker, through the C-ABI.
+
+Bar: atol 1e-2 / rtol 1e-2 on the fp32 cast of both sides (the stated tolerance), plus a per-row relative L2
+bound of 1e-2 and lse within 1e-3, because the stated absolute bar is loose at long context."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention_oracle as A
+from oracle import draft_oracle as D
+from paper_2607_17299_b200 import workloads as W
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+KERNELS = [0, 1]
+
+
+@pytest.fixture(scope="module")
+def war():
+    from paper_2607_17299_b200 import binding
+    return binding
+
+
+def _random_trees(rng, B, N, n_fixed=None):
+    parent = np.full((B, N), -1, np.int32); nn = np.zeros(B, np.int32)
+    for i in range(B):
+        n = int(rng.integers(1, N + 1)) if n_fixed is None else n_fixed[i]
+        nn[i] = n
+        for j in range(1, n):
+            parent[i, j] = int(rng.integers(0, j))
+    return nn, parent
+
+
+def _check(war, cfg, ctx, nn, parent, kernel, scale=None, a=None):
+    scale = 1.0 / np.sqrt(cfg.D) if scale is None else scale
+    if a is None:
+        a = W.make_attention_inputs(cfg, ctx, device="cuda:0")
+    got, got_lse, raw = U.run_attn(war, a, nn, parent, scale, kernel)
+    want = A.verify_attention(a.q, a.k_pool, a.v_pool, a.page_table.cpu().numpy(), a.prefix_len.cpu().numpy(),
+                              nn, parent, scale)
+    for i in range(cfg.B):
+        n = int(nn[i])
+        if n:
+            U.assert_attention_close(got[i], got_lse[i], want[i][0], want[i][1], n)
+        assert (got[i, n:] == 7.0).all() and (got_lse[i, n:] == 7.0).all()       # rows beyond num_nodes untouched
+    assert war.war_device_status() == 0
+    return a, raw
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_tiny_config(war, kernel):
+    """8 requests x 4096 context, trees from the brute-force drafter; the plan splits every request into several
+    KV chunks here, so the combine pass is exercised as well."""
+    cfg = W.CONFIGS["tiny"]
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(cfg)
+    _, nn, _, parent, _ = D.draft_batch(D.Corpus(tok, off), tails, tl, cfg.N, cfg.topk)
+    ctx = W.context_lengths(cfg)
+    a, raw1 = _check(war, cfg, ctx, nn, parent, kernel)
+    _, _, raw2 = U.run_attn(war, a, nn, parent, 1.0 / np.sqrt(cfg.D), kernel)
+    assert torch.equal(raw1, raw2)                                           # deterministic
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("case", ["ragged16", "ragged32", "wide", "single", "deep"])
+def test_shapes_and_ragged_lengths(war, kernel, case):
+    rng = np.random.default_rng(hash(case) % 1000)
+    base = W.CONFIGS["tiny"]
+    if case == "ragged16":       # lengths around page and tile edges, empty prefix, an unused request
+        ctx = np.array([1, 2, 15, 16, 17, 113, 127, 128, 129, 1000, 1024, 1025, 2049, 3000])
+        cfg = W.scaled(base, B=len(ctx), N=16)
+        nn, parent = _random_trees(rng, cfg.B, cfg.N)
+        nn[3] = 0
+    elif case == "ragged32":     # page size 32, 24 slots (96 rows)
+        ctx = np.array([1, 31, 33, 500, 2047, 5000])
+        cfg = W.scaled(base, B=len(ctx), N=24, page_size=32)
+        nn, parent = _random_trees(rng, cfg.B, cfg.N)
+    elif case == "wide":         # 64 query heads on 8 kv heads, 64 slots: 512 rows per kv head, four row blocks
+        ctx = np.array([700, 2500, 40])
+        cfg = W.scaled(base, B=len(ctx), N=64, Hq=64)
+        nn, parent = _random_trees(rng, cfg.B, cfg.N, n_fixed=[64, 37, 5])
+    elif case == "single":       # one slot per request: ordinary decode attention
+        ctx = np.array([300, 4000, 9])
+        cfg = W.scaled(base, B=len(ctx), N=8)
+        nn, parent = _random_trees(rng, cfg.B, cfg.N, n_fixed=[1, 1, 1])
+    else:                        # chains as deep as the budget allows (every ancestor bit set)
+        ctx = np.array([257, 1500])
+        cfg = W.scaled(base, B=len(ctx), N=32)
+        nn = np.array([32, 32], np.int32)
+        parent = np.tile(np.arange(-1, 31, dtype=np.int32), (2, 1))
+    _check(war, cfg, ctx, nn, parent, kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_structured_values_with_order_one_outputs(war, kernel):
+    """Zero queries give a uniform softmax, so outputs are plain means of V rows (order one, exactly known), and a
+    sibling's V must not leak: the hand-worked case scaled to head size 128."""
+    with open(os.path.join(GOLD, "attention_case3.json")) as f:
+        g = json.load(f)
+    cfg = W.scaled(W.CONFIGS["tiny"], B=1, N=8)
+    ctx = np.array([g["prefix_len"] + 1])
+    a = W.make_attention_inputs(cfg, ctx, device="cuda:0")
+    a.q.zero_(); a.v_pool.zero_()
+    rows = g["prefix_v"] + g["slot_v"]
+    page = int(a.page_table[0, 0])
+    for pos, v in enumerate(rows):
+        a.v_pool[page, :, pos, 0] = v[0]
+        a.v_pool[page, :, pos, 1] = v[1]
+    nn = np.array([3], np.int32)
+    parent = np.array([g["parent"] + [-1] * 5], np.int32)
+    got, lse, _ = U.run_attn(war, a, nn, parent, g["scale"], kernel)
+    for j in range(3):
+        np.testing.assert_allclose(got[0, j, :, :2], np.tile(np.array(g["out"][j]), (cfg.Hq, 1)), atol=4e-3)
+        np.testing.assert_allclose(np.exp(lse[0, j]), g["lse_exp"][j], rtol=1e-4)
+    assert np.abs(got[0, :3, :, 2:]).max() == 0.0
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_needle_key_and_large_logits(war, kernel):
+    """One key with a huge logit deep inside a long context: the output is that key's V row (order-one values,
+    also a test of the running-max rescale: the needle sits after many ordinary tiles)."""
+    cfg = W.scaled(W.CONFIGS["tiny"], B=2, N=4)
+    ctx = np.array([3000, 2000])
+    a = W.make_attention_inputs(cfg, ctx, device="cuda:0")
+    nn = np.array([2, 1], np.int32)
+    parent = np.array([[-1, 0, -1, -1], [-1, -1, -1, -1]], np.int32)
+    pos = 2500
+    page = int(a.page_table[0, pos // cfg.page_size])
+    qv = a.q[0, 1, :, :].float()
+    a.k_pool[page, :, pos % cfg.page_size, :] = (qv.view(cfg.Hkv, -1, cfg.D)[:, 0, :] * 3).to(torch.bfloat16)
+    _check(war, cfg, ctx, nn, parent, kernel, a=a)
+    got, _, _ = U.run_attn(war, a, nn, parent, 1.0 / np.sqrt(cfg.D), kernel)
+    G = cfg.Hq // cfg.Hkv
+    want = a.v_pool[page, :, pos % cfg.page_size, :].float().cpu().numpy()
+    np.testing.assert_allclose(got[0, 1, ::G, :], want, atol=2e-2, rtol=2e-2)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_page_permutation_leaves_bits_unchanged(war, kernel):
+    cfg = W.scaled(W.CONFIGS["tiny"], B=3, N=16)
+    ctx = np.array([1500, 700, 3100])
+    rng = np.random.default_rng(2)
+    nn, parent = _random_trees(rng, cfg.B, cfg.N)
+    a = W.make_attention_inputs(cfg, ctx, device="cuda:0")
+    _, _, raw1 = U.run_attn(war, a, nn, parent, 0.1, kernel)
+    perm = torch.randperm(a.num_pages, generator=torch.Generator().manual_seed(1)).to("cuda:0")
+    inv = torch.empty_like(perm); inv[perm] = torch.arange(a.num_pages, device="cuda:0")
+    a.k_pool = a.k_pool[perm].contiguous(); a.v_pool = a.v_pool[perm].contiguous()
+    pt = a.page_table.long()
+    a.page_table = torch.where(pt >= 0, inv[pt.clamp(min=0)], pt).to(torch.int32)
+    _, _, raw2 = U.run_attn(war, a, nn, parent, 0.1, kernel)
+    assert torch.equal(raw1, raw2)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_malformed_inputs_are_reported_not_faulted(war, kernel):
+    cfg = W.scaled(W.CONFIGS["tiny"], B=2, N=8)
+    ctx = np.array([200, 300])
+    a = W.make_attention_inputs(cfg, ctx, device="cuda:0")
+    nn = np.array([3, 3], np.int32)
+    parent = np.array([[-1, 0, 5, -1, -1, -1, -1, -1], [-1, 0, 1, -1, -1, -1, -1, -1]], np.int32)
+    got, lse, _ = U.run_attn(war, a, nn, parent, 0.1, kernel)
+    assert (got[0] == 7.0).all()                                             # the bad request is skipped
+    assert (got[1, :3] != 7.0).any()
+    assert war.war_device_status() == 7
+    a.page_table[1, 2] = a.num_pages + 5                                     # a page index outside the pool
+    U.run_attn(war, a, np.array([0, 3], np.int32), parent, 0.1, kernel)
+    assert war.war_device_status() == 8

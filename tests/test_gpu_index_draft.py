@@ -1,0 +1,195 @@
+"""GPU parity: suffix index and draft trees, bit-exact against the brute-force checker, through the C-ABI."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import draft_oracle as D
+from paper_2607_17299_b200 import workloads as W
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+@pytest.fixture(scope="module")
+def war():
+    from paper_2607_17299_b200 import binding
+    return binding
+
+
+def _flat(trajs):
+    off = np.zeros(len(trajs) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(t) for t in trajs])
+    tok = np.concatenate([np.asarray(t, dtype=np.int32) for t in trajs]) if len(trajs) else np.zeros(0, np.int32)
+    return tok, off
+
+
+def _read_device(ptr, nbytes):
+    """Copies raw device memory to the host (test-only peek at the index internals)."""
+    import ctypes
+    cudart = ctypes.CDLL("libcudart.so.12")
+    host = np.empty(nbytes, dtype=np.uint8)
+    rc = cudart.cudaMemcpy(ctypes.c_void_p(host.ctypes.data), ctypes.c_void_p(ptr), ctypes.c_size_t(nbytes), 2)
+    assert rc == 0
+    return host
+
+
+def _compare_with_oracle(war, tok, off, vocab, tails, tl, N, k, min_match=1, ix=None):
+    own = ix is None
+    if own:
+        ix = U.build_index(war, tok, off, vocab)
+    got = U.run_draft(war, ix, tails, tl, N, k, min_match)
+    want = D.draft_batch(D.Corpus(tok, off), tails, tl, N, k, min_match)
+    names = ["match_len", "num_nodes", "ids", "parent", "count"]
+    for name, g, w in zip(names, got, want):
+        assert (g == w).all(), f"{name} differs at request(s) {np.flatnonzero((g != w).reshape(len(g), -1).any(axis=1))[:8]}"
+    assert war.war_device_status() == 0
+    if own:
+        ix.destroy()
+    return got
+
+
+def test_textbook_suffix_array_and_lcp(war):
+    """'banana$' with a=1, b=2, n=3: the suffix array and LCP array every textbook prints."""
+    tok, off = _flat([[2, 1, 3, 1, 3, 1]])
+    ix = U.build_index(war, tok, off, vocab=4)
+    info = war.war_index_info(ix)
+    assert info.M == 7 and info.T == 1
+    sa = _read_device(info.d_sa, 7 * 4).view(np.int32)
+    lcp = _read_device(info.d_lcp, 7)
+    corpus = _read_device(info.d_corpus, 7 * 4).view(np.int32)
+    bucket = _read_device(info.d_bucket, 5 * 4).view(np.int32)
+    assert corpus.tolist() == [2, 1, 3, 1, 3, 1, -1]
+    assert sa.tolist() == [6, 5, 3, 1, 0, 4, 2]
+    assert lcp.tolist() == [0, 0, 1, 3, 0, 0, 2]
+    assert bucket.tolist() == [1, 1, 4, 5, 7]
+    ix.destroy()
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_suffix_array_equals_naive_sort(war, seed):
+    rng = np.random.default_rng(seed)
+    trajs = [rng.integers(0, 4, size=int(rng.integers(0, 300))).tolist() for _ in range(7)]
+    tok, off = _flat(trajs)
+    depth = 96
+    ix = U.build_index(war, tok, off, vocab=4, max_depth=depth)
+    info = war.war_index_info(ix)
+    M = int(info.M)
+    assert M == len(tok) + len(trajs)
+    sa = _read_device(info.d_sa, M * 4).view(np.int32)
+    lcp = _read_device(info.d_lcp, M)
+    corpus = _read_device(info.d_corpus, M * 4).view(np.int32).tolist()
+    assert sorted(sa.tolist()) == list(range(M))                       # a permutation
+    naive = sorted(range(M), key=lambda i: corpus[i:])                 # separators are negative and unique
+    # order is only promised to depth 128 (the doubling's reach); beyond that ties may remain in any order
+    key = lambda i: corpus[i:i + 128]
+    assert [key(i) for i in sa] == [key(i) for i in naive]
+    for i in range(1, M):
+        a, b = corpus[sa[i - 1]:], corpus[sa[i]:]
+        l = 0
+        while l < min(len(a), len(b), depth) and a[l] == b[l]:
+            l += 1
+        assert lcp[i] == l
+    ix.destroy()
+
+
+@pytest.mark.parametrize("name", ["draft_case1.json", "draft_case2.json"])
+def test_hand_worked_cases(war, name):
+    with open(os.path.join(GOLD, name)) as f:
+        g = json.load(f)
+    tok, off = _flat(g["trajectories"])
+    ix = U.build_index(war, tok, off, vocab=16)
+    tail = np.array([g["tail"]], dtype=np.int32)
+    for tr in g["trees"]:
+        ml, nn, ids, par, cnt = U.run_draft(war, ix, tail, np.array([g["tail_len"]]), tr["N"], tr["k"])
+        n = len(tr["ids"])
+        assert ml[0] == g["match_len"] and nn[0] == n
+        assert ids[0, :n].tolist() == tr["ids"] and par[0, :n].tolist() == tr["parent"] and cnt[0, :n].tolist() == tr["count"]
+        assert (ids[0, n:] == -1).all() and (par[0, n:] == -1).all() and (cnt[0, n:] == 0).all()
+    ix.destroy()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_tiny_alphabets_force_ties(war, seed):
+    rng = np.random.default_rng(100 + seed)
+    vocab = int(rng.integers(2, 6))
+    trajs = [rng.integers(0, vocab, size=int(rng.integers(0, 120))).tolist() for _ in range(int(rng.integers(1, 9)))]
+    tok, off = _flat(trajs)
+    P = int(rng.integers(1, 33))
+    N = int(rng.integers(1, 65))
+    k = int(rng.integers(1, 9))
+    B = 24
+    tails = rng.integers(0, vocab + 1, size=(B, P)).astype(np.int32)
+    tails[0, :] = -1                                                   # negative ids must never match a separator
+    tl = rng.integers(0, P + 1, size=B).astype(np.int32)
+    _compare_with_oracle(war, tok, off, vocab + 1, tails, tl, N, k, min_match=int(rng.integers(0, 4)))
+
+
+def test_tiny_config_with_structured_tails(war):
+    cfg = W.CONFIGS["tiny"]
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(cfg)
+    rng = np.random.default_rng(5)
+    extra, extra_len = [], []
+    for _ in range(24):                                                # tails planted inside the corpus
+        t = int(rng.integers(0, cfg.n_traj)); dist = int(rng.integers(1, 300))
+        e = int(off[t]) + dist; m = min(cfg.P, dist)
+        row = np.full(cfg.P, -1, np.int32); row[cfg.P - m:] = tok[e - m:e]
+        extra.append(row); extra_len.append(m)
+    for v in (0, 1, 2, 5, 17):                                         # one-token matches on the most frequent ids:
+        row = np.full(cfg.P, cfg.vocab + 3, np.int32); row[-1] = v      # the largest intervals (block-wide scans)
+        extra.append(row); extra_len.append(cfg.P)
+    row = np.full(cfg.P, cfg.vocab + 9, np.int32); extra.append(row); extra_len.append(cfg.P)   # never seen
+    for t in range(3):                                                 # the very end of a trajectory: no continuation
+        row = tok[off[t + 1] - cfg.P:off[t + 1]].copy(); extra.append(row); extra_len.append(cfg.P)
+    tails = np.concatenate([tails, np.stack(extra)]); tl = np.concatenate([tl, np.array(extra_len, np.int32)])
+    got = _compare_with_oracle(war, tok, off, cfg.vocab, tails, tl, cfg.N, cfg.topk)
+    assert got[4][:, 0].max() >= 8192                                  # a block-wide scan really happened
+    for N, k in ((64, 8), (8, 4), (2, 1), (1, 4), (33, 3)):
+        _compare_with_oracle(war, tok, off, cfg.vocab, tails, tl, N, k)
+
+
+def test_append_equals_rebuild_and_order_independence(war):
+    cfg = W.CONFIGS["tiny"]
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(cfg)
+    T = cfg.n_traj
+    cut1, cut2 = 20, 45
+    cap = len(tok) + T
+    ix = U.build_index(war, tok[:off[cut1]], off[:cut1 + 1], cfg.vocab, capacity=cap)
+    d_tok = torch.from_numpy(tok).to("cuda:0")
+    war.war_index_append(ix, d_tok, off[cut1:cut2 + 1])                # offsets index into d_tok
+    war.war_index_append(ix, d_tok, off[cut2:])
+    assert war.war_index_info(ix).M == cap and war.war_index_info(ix).T == T
+    _compare_with_oracle(war, tok, off, cfg.vocab, tails, tl, cfg.N, cfg.topk, ix=ix)
+    with pytest.raises(war.WarError) as e:
+        war.war_index_append(ix, d_tok, off[:2])
+    assert e.value.code == 3                                           # capacity; the index is unchanged
+    assert war.war_index_info(ix).M == cap
+    _compare_with_oracle(war, tok, off, cfg.vocab, tails, tl, cfg.N, cfg.topk, ix=ix)
+    ix.destroy()
+    # same trajectories in another arrival order: same drafts
+    order = np.random.default_rng(3).permutation(T)
+    trajs = [tok[off[t]:off[t + 1]] for t in order]
+    tok2, off2 = _flat(trajs)
+    ix2 = U.build_index(war, tok2, off2, cfg.vocab)
+    a = U.run_draft(war, ix2, tails, tl, cfg.N, cfg.topk)
+    want = D.draft_batch(D.Corpus(tok, off), tails, tl, cfg.N, cfg.topk)
+    for g, w in zip(a, want):
+        assert (g == w).all()
+    ix2.destroy()
+
+
+def test_empty_and_degenerate_inputs(war):
+    ix = U.build_index(war, np.zeros(0, np.int32), np.zeros(1, np.int64), vocab=10, capacity=64)   # no trajectories
+    tails = np.array([[1, 2, 3, 4]], np.int32)
+    ml, nn, ids, par, cnt = U.run_draft(war, ix, tails, np.array([4]), 8, 4)
+    assert ml[0] == 0 and nn[0] == 1 and ids[0, 0] == 4 and cnt[0, 0] == 0
+    d_tok = torch.tensor([1, 2, 3, 4, 5], dtype=torch.int32, device="cuda:0")
+    war.war_index_append(ix, d_tok, np.array([0, 0, 5, 5]))            # empty trajectories around a real one
+    ml, nn, ids, par, cnt = U.run_draft(war, ix, tails, np.array([4]), 8, 4, with_count=False)
+    assert ml[0] == 4 and nn[0] == 2 and ids[0, :2].tolist() == [4, 5] and cnt is None
+    ix.destroy()
