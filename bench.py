@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the speculate-and-verify step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload high|low|longtail|wide|tiny] [--impl ours|reference]
+
+A step = one pass of the whole hot path over one batch of live requests: war_draft (suffix match + draft trees)
+-> war_verify_attn (tree-masked GQA attention over the paged bf16 KV cache) -> war_accept.  The index build is
+set-up and is reported separately.  The metric is verified tokens per second: sum over requests of
+(accepted draft tokens + the one token the target model always yields) divided by the step time.
+
+One JSON line is printed by rank 0.  `value` has every input resident in HBM; `e2e` repeats the step with the
+per-step inputs starting in pinned host memory and the results read back, copies inside the timed region;
+`roofline` puts the verify-attention call against the measured HBM copy bandwidth; `cpu_baseline` times the CPU
+checker (oracle/) on a bounded sample of the same requests on this machine's host cores.
+
+`--impl reference` times that CPU checker alone (there is no other reference implementation to run).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "verified tokens/s per speculate+verify step"
+UNIT = "tokens/s"
+LAUNCHES_PER_STEP = 5          # draft, attention plan, attention, split-KV combine, accept
+
+
+def kv_bytes(cfg, prefix_len: np.ndarray, num_nodes: np.ndarray) -> int:
+    """Bytes the verify attention must read once: K and V rows of every prefix position and every tree slot."""
+    tokens = int((prefix_len.astype(np.int64) + num_nodes.astype(np.int64))[num_nodes > 0].sum())
+    return tokens * cfg.Hkv * cfg.D * 2 * 2
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(cfg, corpus, tails, tail_len, attn, ctx, targets_fn, requests, budget_s=None):
+    """Runs the CPU checker on the given requests (in order, stopping once budget_s is spent, at least one).
+    Returns (tokens verified, seconds, requests done)."""
+    from oracle import accept_oracle, attention_oracle, draft_oracle
+    import torch
+    scale = 1.0 / float(np.sqrt(cfg.D))
+    t0 = time.perf_counter()
+    verified, done = 0, 0
+    pt = attn.page_table.cpu().numpy() if attn is not None else None
+    for i in requests:
+        ml, ends = draft_oracle.longest_suffix_match(corpus, tails[i], int(tail_len[i]))
+        ids, parent, count = draft_oracle.build_draft_tree(corpus, tails[i], ml, ends, cfg.N, cfg.topk)
+        n = len(ids)
+        full_ids = np.full((1, cfg.N), -1, np.int32); full_par = np.full((1, cfg.N), -1, np.int32)
+        full_ids[0, :n] = ids; full_par[0, :n] = parent
+        K, V = attention_oracle.gather_request_kv(attn.k_pool, attn.v_pool, pt[i], int(ctx[i]) - 1 + n)
+        q = attn.q[i].to("cpu").to(torch.float64).numpy()
+        attention_oracle.verify_attention_request(q, K, V, int(ctx[i]) - 1, full_par[0], n, scale)
+        target = targets_fn(i, full_ids, full_par, n)
+        alen, _, _ = accept_oracle.accept_request(full_ids[0], full_par[0], n, target, 0)
+        verified += alen + 1
+        done += 1
+        if budget_s is not None and time.perf_counter() - t0 > budget_s:
+            break
+    return verified, time.perf_counter() - t0, done
+
+
+def threads_in_use() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        n = 1
+    return int(min(n, len(os.sched_getaffinity(0))))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="high")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--kernel", type=int, default=0, help="0 = tensor-core verify attention, 1 = plain CUDA-core kernel")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    import torch
+    from paper_2607_17299_b200 import workloads as W
+    cfg = W.CONFIGS[args.workload]
+    base_config = {"workload": f"{cfg.name}: corpus {cfg.n_traj} trajectories, {cfg.B} requests, tree <= {cfg.N} slots, "
+                               f"{cfg.Hq}q/{cfg.Hkv}kv heads, d={cfg.D}, page {cfg.page_size}",
+                   "requests_per_gpu": cfg.B, "parallelism": f"replica x{world}" if world > 1 else "single gpu",
+                   "l2": "inputs (KV cache) far larger than L2, no flush needed" if cfg.name != "tiny" else
+                         "KV cache fits L2: value is an L2-resident number"}
+
+    # ------------------------------------------------------------------------------------------
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        from oracle import draft_oracle
+        tok, off = W.make_corpus(cfg)
+        tails, tl = W.make_request_tails(cfg)
+        ctx = W.context_lengths(cfg)
+        corpus = draft_oracle.Corpus(tok, off)
+        per_step = 4
+        # KV for a handful of distinct requests, generated once on the host (set-up, untimed); steps cycle through them
+        distinct = list(range(min(cfg.B, 16)))
+        sub = W.scaled(cfg, B=len(distinct))
+        attn = W.make_attention_inputs(sub, ctx[distinct], device="cpu")
+
+        def targets_fn(i, ids, par, n):
+            return W.make_targets(W.scaled(cfg, B=1), ids, par, np.array([n]), 0)[0]
+        times, verified = [], 0
+        for s in range(args.steps + args.warmup):
+            reqs = [(s * per_step + k) % len(distinct) for k in range(per_step)]
+            v, dt, _ = oracle_sample(cfg, corpus, tails, tl, attn, ctx, targets_fn, reqs)
+            if s >= args.warmup:
+                times.append(dt); verified += v
+        total = sum(times)
+        value = verified / total
+        cores = threads_in_use()
+        line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(1, args.steps),
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "config": dict(base_config, sample=f"{per_step} requests per step, cycling through the batch"),
+                "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                 "sample": f"{per_step} requests per step x {args.steps} steps"},
+                "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    # ------------------------------------------------------------------------------------------
+    from paper_2607_17299_b200 import binding as war
+    import torch.distributed as dist
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- set-up: corpus, index, requests, KV cache (all seeded, synthetic) ----
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(cfg)
+    ctx = W.context_lengths(cfg)
+    d_tok = torch.from_numpy(tok).to(dev)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    ix = war.war_index_build(d_tok, off, cfg.vocab, cfg.P + cfg.N, len(tok) + cfg.n_traj)
+    index_build_s = time.perf_counter() - t0
+    del d_tok
+    attn = W.make_attention_inputs(cfg, ctx, device=dev)
+    B, N = cfg.B, cfg.N
+    d_tails = torch.from_numpy(tails).to(dev)
+    d_tl = torch.from_numpy(tl).to(dev)
+    i32 = dict(dtype=torch.int32, device=dev)
+    d_ml, d_nn = torch.zeros(B, **i32), torch.zeros(B, **i32)
+    d_ids, d_par, d_cnt = torch.zeros((B, N), **i32), torch.zeros((B, N), **i32), torch.zeros((B, N), **i32)
+    d_alen, d_path, d_bonus = torch.zeros(B, **i32), torch.zeros((B, N), **i32), torch.zeros(B, **i32)
+    d_out = torch.zeros_like(attn.q)
+    d_lse = torch.zeros(attn.q.shape[:3], dtype=torch.float32, device=dev)
+    scale = 1.0 / float(np.sqrt(cfg.D))
+    params = war.attn_params(attn.q, attn.k_pool, attn.v_pool, attn.page_table, scale, args.kernel)
+    ws = war.new_workspace(params, dev)
+
+    # targets depend on the trees; the trees are a deterministic function of the inputs, so draft once to make them
+    war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt)
+    torch.cuda.synchronize()
+    h_ids, h_par, h_nn = d_ids.cpu().numpy(), d_par.cpu().numpy(), d_nn.cpu().numpy()
+    targets = W.make_targets(cfg, h_ids, h_par, h_nn, 0)
+    d_target = torch.from_numpy(targets).to(dev)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def step(attn_events=None):
+        war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt)
+        if attn_events is not None:
+            attn_events[0].record()
+        war.war_verify_attn(attn.q, attn.k_pool, attn.v_pool, attn.page_table, attn.prefix_len, d_nn, d_par, params, ws,
+                            d_out, d_lse)
+        if attn_events is not None:
+            attn_events[1].record()
+        war.war_accept(d_ids, d_par, d_nn, d_target, 0, d_alen, d_path, d_bonus)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    attn_ev = [(ev(), ev()) for _ in range(args.steps)]
+    draft_ev = [ev() for _ in range(args.steps + 1)]
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        start, stop = ev(), ev()
+        start.record()
+        for s in range(args.steps):
+            draft_ev[s].record()
+            step(attn_ev[s])
+        draft_ev[args.steps].record()
+        stop.record()
+        barrier()
+        total_ms = start.elapsed_time(stop)
+    attn_ms = float(np.mean([a.elapsed_time(b) for a, b in attn_ev]))
+    draft_ms = float(np.mean([draft_ev[s].elapsed_time(attn_ev[s][0]) for s in range(args.steps)]))
+    accept_ms = float(np.mean([attn_ev[s][1].elapsed_time(draft_ev[s + 1]) for s in range(args.steps)]))
+    status = war.war_device_status()
+    h_alen = d_alen.cpu().numpy()
+    verified = int((h_alen.astype(np.int64) + 1).sum())
+    slots = int(h_nn.sum())
+
+    # ---- end to end: per-step inputs start in pinned host memory, results are read back ----
+    pin = lambda t: t.cpu().pin_memory()
+    h_q, h_tails, h_tl, h_target = pin(attn.q), pin(d_tails), pin(d_tl), pin(d_target)
+    r_alen, r_path, r_bonus = pin(d_alen), pin(d_path), pin(d_bonus)
+    r_ids, r_par, r_nn, r_out = pin(d_ids), pin(d_par), pin(d_nn), pin(d_out)
+    h2d = sum(t.numel() * t.element_size() for t in (h_q, h_tails, h_tl, h_target))
+    d2h = sum(t.numel() * t.element_size() for t in (r_alen, r_path, r_bonus, r_ids, r_par, r_nn, r_out))
+
+    def e2e_step():
+        attn.q.copy_(h_q, non_blocking=True); d_tails.copy_(h_tails, non_blocking=True)
+        d_tl.copy_(h_tl, non_blocking=True); d_target.copy_(h_target, non_blocking=True)
+        step()
+        for dst, src in ((r_alen, d_alen), (r_path, d_path), (r_bonus, d_bonus), (r_ids, d_ids), (r_par, d_par),
+                         (r_nn, d_nn), (r_out, d_out)):
+            dst.copy_(src, non_blocking=True)
+        torch.cuda.synchronize()                        # the caller needs the accepted tokens before the next step
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()
+    barrier()
+    e2e_ms = 1e3 * (time.perf_counter() - t0)
+
+    # ---- max over ranks, totals over ranks ----
+    agg = torch.tensor([total_ms, e2e_ms, attn_ms], dtype=torch.float64, device=dev)
+    tot = torch.tensor([verified, slots], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(agg, op=dist.ReduceOp.MAX)
+        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+    total_ms, e2e_ms, attn_ms = [float(x) for x in agg.tolist()]
+    verified_all, slots_all = [float(x) for x in tot.tolist()]
+    ms_per_step = total_ms / args.steps
+
+    if rank == 0:
+        peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(peaks_path):
+            with open(peaks_path) as f:
+                peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy)"
+        else:
+            peak, peak_src = 6650.0, "fallback"
+        kvb = kv_bytes(cfg, ctx - 1, h_nn)
+        achieved = kvb / (attn_ms * 1e-3) / 1e9
+        traffic_path = os.path.join(ROOT, "profiles", f"traffic_{cfg.name}.json")
+        traffic = None
+        if os.path.exists(traffic_path):
+            with open(traffic_path) as f:
+                traffic = json.load(f).get("dram_bytes_per_launch")
+        line = {
+            "metric": METRIC, "value": verified_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": dict(base_config, kernel="tcgen05" if args.kernel == 0 else "cuda-core"),
+            "clocks": clocks.summary(),
+            "e2e": {"value": verified_all / (e2e_ms / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
+            "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "kernel": "war_verify_attn (plan + attention + combine launches)",
+                         "bytes_per_launch": kvb, "ms_per_launch": attn_ms, "peak_source": peak_src,
+                         "frac_of_8TBps_nominal": achieved / 8000.0},
+            "breakdown_ms": {"draft": draft_ms, "verify_attn": attn_ms, "accept": accept_ms},
+            "slots_verified_per_s": slots_all / (ms_per_step * 1e-3),
+            "accept_len_mean": float(h_alen.mean()), "index_build_s": index_build_s, "index_tokens": int(len(tok)),
+            "device_status": status,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            from oracle import draft_oracle
+            corpus = draft_oracle.Corpus(tok, off)
+            def targets_fn(i, ids, par, n):
+                return targets[i]
+            v, secs, done = oracle_sample(cfg, corpus, tails, tl, attn, ctx, targets_fn, list(range(cfg.B)), budget_s=15.0)
+            line["cpu_baseline"] = {"value": v / secs, "unit": UNIT, "cores": threads_in_use(), "kind": "oracle",
+                                    "sample": f"first {done} of {cfg.B} requests, {secs:.1f} s"}
+        print(json.dumps(line))
+    ix.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

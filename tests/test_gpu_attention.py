@@ -68,7 +68,7 @@ def test_tiny_config(war, kernel):
 @pytest.mark.parametrize("kernel", KERNELS)
 @pytest.mark.parametrize("case", ["ragged16", "ragged32", "wide", "single", "deep"])
 def test_shapes_and_ragged_lengths(war, kernel, case):
-    rng = np.random.default_rng(hash(case) % 1000)
+    rng = np.random.default_rng(["ragged16", "ragged32", "wide", "single", "deep"].index(case))
     base = W.CONFIGS["tiny"]
     if case == "ragged16":       # lengths around page and tile edges, empty prefix, an unused request
         ctx = np.array([1, 2, 15, 16, 17, 113, 127, 128, 129, 1000, 1024, 1025, 2049, 3000])
