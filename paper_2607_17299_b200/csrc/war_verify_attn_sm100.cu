@@ -1,9 +1,556 @@
-// Tensor-core verify attention (placeholder until the tcgen05 kernel lands): forwards to the plain kernel.
+// Tensor-core verify attention for sm_100a: TMA-staged KV pages -> tcgen05.mma with accumulators in TMEM ->
+// online softmax -> tcgen05.mma again, one persistent CTA per SM.
+//
+// Work unit (see war_attn_plan.cuh): up to 128 query rows (slot, head-of-group) of one kv head against a range of
+// 128-key tiles.  Per tile:   S = Q K^T   (M=128 rows, N=128 keys, K=128 dims; bf16 in, fp32 in TMEM)
+//                             P = exp2(S*scale*log2e - m), masked by the tree's ancestor bits on tree columns
+//                             O += P V    (M=128 rows, N=128 dims, K=128 keys; P staged in shared memory as bf16)
+// Warp roles:  warp 0  producer: reads the page table, issues one TMA tensor copy per (page, head) into a ring of
+//                      32 KB slots (K tile, V tile, K tile, ...); no multicast, this GPU's memory only
+//              warp 1  MMA issuer (one lane): S(t+1) is issued before PV(t) so the tensor pipe works while the
+//                      softmax warps are busy; owns the TMEM allocation
+//              warps 2-5  softmax: one thread per query row (TMEM lane), running max/sum in registers, rescale of
+//                      O in TMEM only when the max grows by more than 2^8, epilogue
+// Shared-memory operand layouts are the canonical 128-byte-swizzled ones: K-major for Q, K and P, MN-major for V.
+// A (page, head) block lands as [token/8][d/64][token%8][d%64], which serves both K (K-major, 8-row groups 2 KB
+// apart) and V (MN-major, 64-wide column blocks 1 KB apart, 8-key groups 2 KB apart) with one copy per block.
+// Every wait is bounded: on expiry the kernel records WAR_ERR_TIMEOUT, raises a CTA-wide abort flag and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <math_constants.h>
 #include "war_common.cuh"
 #include "war_attn_plan.cuh"
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kSlots = 5;
+constexpr int kSlotBytes = 32768;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr float kRescaleThreshold = 8.0f;           // log2 units
+constexpr unsigned long long kWaitBudgetNs = 2000000000ull;
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr int kOffQ = 0;
+constexpr int kOffP = 32768;
+constexpr int kOffRing = 65536;
+constexpr int kOffBar = kOffRing + kSlots * kSlotBytes;
+constexpr int kSmemBytes = kOffBar + 256 + 1024;
+
+struct Bars {
+    uint64_t full[kSlots], empty[kSlots];
+    uint64_t s_ready[2], s_free[2];
+    uint64_t p_ready, pv_done, q_ready;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false when the CTA is aborting (this wait ran out of time, or another one did).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Bars* bars, int* status_word) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    unsigned spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*(volatile int*)&bars->abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitBudgetNs) {
+                war_set_device_status(status_word, WAR_ERR_TIMEOUT);
+                atomicExch(&bars->abort_flag, 1);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_block(uint32_t dst, const CUtensorMap* map, int block, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %3, %3, %3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(block) : "memory");
+}
+
+// shared-memory matrix descriptor, 128-byte swizzle, sm_100 version field
+__device__ __forceinline__ uint64_t umma_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;          // descriptor version
+    d |= (uint64_t)2 << 61;          // SWIZZLE_128B
+    return d;
+}
+// instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major, M x N
+__device__ __forceinline__ constexpr uint32_t umma_idesc(int m, int n, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+          "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+          "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Unit k of this CTA under the snake deal of the longest-first list: even rounds left to right, odd rounds back.
+__device__ __forceinline__ int snake_unit(int k, int cta, int ctas) { return k * ctas + ((k & 1) ? ctas - 1 - cta : cta); }
+
+struct KernelArgs {
+    const __nv_bfloat16* q;
+    const int32_t* page_table;
+    const int32_t* prefix_len;
+    __nv_bfloat16* out;
+    float* lse;
+    int* status_word;
+    AttnWorkspace w;
+    long long num_pages;
+    float scale_log2;
+    int N, Hq, Hkv, G, page_size, max_pages;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const KernelArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    Bars* bars = (Bars*)(smem + kOffBar);
+    const uint32_t sQ = smem_u32(smem + kOffQ), sP = smem_u32(smem + kOffP), sRing = smem_u32(smem + kOffRing);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_units = a.w.counters[1];
+    const int pages_per_tile = kTileKeys / a.page_size;
+    const uint32_t page_bytes = (uint32_t)a.page_size * 256u;
+
+    if (tid == 0) {
+        for (int i = 0; i < kSlots; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&bars->s_ready[i], 1); mbar_init(&bars->s_free[i], 128); }
+        mbar_init(&bars->p_ready, 128);
+        mbar_init(&bars->pv_done, 1);
+        mbar_init(&bars->q_ready, 128);
+        bars->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+    const uint32_t tmem_S = tmem;                    // two buffers of 128 columns
+    const uint32_t tmem_O = tmem + 256;              // 128 columns
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        uint32_t ld = 0;                             // half-tile loads issued so far
+        bool ok = true;
+        for (int k = 0; ok; ++k) {
+            const int u = snake_unit(k, blockIdx.x, gridDim.x);
+            if (u >= n_units) break;
+            const AttnUnit un = a.w.units[u];
+            const int i = un.req;
+            const int L = a.prefix_len[i] + a.w.req[i].n_nodes;
+            const int total_pages = (L + a.page_size - 1) / a.page_size;
+            const int32_t* pt = a.page_table + (size_t)i * a.max_pages;
+            int page_next = -1;
+            if (lane < pages_per_tile) {
+                const int pi = un.tile_begin * pages_per_tile + lane;
+                page_next = pi < total_pages ? pt[pi] : -1;
+            }
+            for (int t = un.tile_begin; t < un.tile_end && ok; ++t) {
+                const int page = page_next;
+                if (t + 1 < un.tile_end && lane < pages_per_tile) {          // prefetch the next tile's page ids
+                    const int pi = (t + 1) * pages_per_tile + lane;
+                    page_next = pi < total_pages ? pt[pi] : -1;
+                }
+                const int n_valid = min(pages_per_tile, total_pages - t * pages_per_tile);
+                int block = -1;
+                if (lane < n_valid) {
+                    long long pg = page;
+                    if (pg < 0 || pg >= a.num_pages) { war_set_device_status(a.status_word, WAR_ERR_BAD_PAGE); pg = 0; }
+                    block = (int)(pg * a.Hkv + un.kvh);
+                }
+#pragma unroll
+                for (int which = 0; which < 2; ++which, ++ld) {
+                    const uint32_t slot = ld % kSlots, phase = (ld / kSlots) & 1u;
+                    ok = mbar_wait(&bars->empty[slot], phase ^ 1u, bars, a.status_word);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    if (lane == 0) mbar_arrive_expect_tx(&bars->full[slot], (uint32_t)n_valid * page_bytes);
+                    __syncwarp();
+                    if (block >= 0)
+                        tma_load_block(sRing + slot * kSlotBytes + lane * page_bytes, which ? &v_map : &k_map, block, &bars->full[slot]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        uint32_t ld = 0, it = 0, units_done = 0;
+        constexpr uint32_t idesc_s = umma_idesc(128, 128, 0);
+        constexpr uint32_t idesc_o = umma_idesc(128, 128, 1);
+        bool ok = true;
+        auto issue_s = [&](uint32_t it_s, uint32_t ld_k) -> bool {
+            const uint32_t slot = ld_k % kSlots, b = it_s & 1u;
+            if (!mbar_wait(&bars->full[slot], (ld_k / kSlots) & 1u, bars, a.status_word)) return false;
+            if (!mbar_wait(&bars->s_free[b], ((it_s >> 1) & 1u) ^ 1u, bars, a.status_word)) return false;
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t kb = sRing + slot * kSlotBytes;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32u;
+                    const uint32_t koff = (uint32_t)(ks >> 2) * 1024u + (uint32_t)(ks & 3) * 32u;
+                    umma_bf16(tmem_S + b * 128u, umma_desc(sQ + off, 16, 1024), umma_desc(kb + koff, 16, 2048), idesc_s, ks > 0);
+                }
+                umma_commit(&bars->s_ready[b]);
+                umma_commit(&bars->empty[slot]);
+            }
+            __syncwarp();
+            return true;
+        };
+        for (int k = 0; ok; ++k) {
+            const int u = snake_unit(k, blockIdx.x, gridDim.x);
+            if (u >= n_units) break;
+            const AttnUnit un = a.w.units[u];
+            const int n_tiles = un.tile_end - un.tile_begin;
+            ok = mbar_wait(&bars->q_ready, units_done & 1u, bars, a.status_word);
+            if (!ok) break;
+            ok = issue_s(it, ld);
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                if (t + 1 < n_tiles) ok = issue_s(it + t + 1, ld + 2 * (t + 1));
+                if (!ok) break;
+                const uint32_t ld_v = ld + 2 * t + 1, slot = ld_v % kSlots;
+                ok = mbar_wait(&bars->full[slot], (ld_v / kSlots) & 1u, bars, a.status_word) &&
+                     mbar_wait(&bars->p_ready, (it + t) & 1u, bars, a.status_word);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t vb = sRing + slot * kSlotBytes;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t off = (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32u;
+                        umma_bf16(tmem_O, umma_desc(sP + off, 16, 1024), umma_desc(vb + (uint32_t)ks * 4096u, 1024, 2048), idesc_o,
+                                  (t > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    umma_commit(&bars->pv_done);
+                    umma_commit(&bars->empty[slot]);
+                }
+                __syncwarp();
+            }
+            it += n_tiles;
+            ld += 2 * n_tiles;
+            ++units_done;
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax / epilogue, one thread per row
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int k = 0; ok; ++k) {
+            const int u = snake_unit(k, blockIdx.x, gridDim.x);
+            if (u >= n_units) break;
+            const AttnUnit un = a.w.units[u];
+            const int i = un.req;
+            const int n = a.w.req[i].n_nodes;
+            const int R = a.G * n;
+            const int pl = a.prefix_len[i];
+            const int L = pl + n;
+            const int gr = un.rb * kRowBlock + row;
+            const bool valid = gr < R;
+            const bool warp_valid = __any_sync(0xffffffffu, valid);
+            const int j = valid ? gr / a.G : 0, g = valid ? gr % a.G : 0;
+            const size_t qrow = ((size_t)i * a.N + j) * a.Hq + un.kvh * a.G + g;
+            const uint64_t anc = valid ? a.w.anc[(size_t)i * a.N + j] : 0ull;
+            // previous unit's MMAs are complete (its last pv_done was awaited in the epilogue), so Q may be replaced
+            {
+                const uint4* src = reinterpret_cast<const uint4*>(a.q + qrow * 128);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const uint4 x = valid ? src[c] : make_uint4(0, 0, 0, 0);
+                    const uint32_t dst = sQ + (uint32_t)(c >> 3) * 16384u + (uint32_t)row * 128u + (uint32_t)(((c & 7) ^ (row & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
+                }
+            }
+            fence_async_proxy();
+            mbar_arrive(&bars->q_ready);
+            float m_used = -CUDART_INF_F, l = 0.f;
+            const int n_tiles = un.tile_end - un.tile_begin;
+            for (int t = 0; t < n_tiles && ok; ++t, ++it) {
+                const uint32_t b = it & 1u;
+                const int key0 = (un.tile_begin + t) * kTileKeys;
+                const bool need_mask = key0 + kTileKeys > pl;
+                ok = mbar_wait(&bars->s_ready[b], (it >> 1) & 1u, bars, a.status_word);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t pk[64];                                   // P as packed bf16 pairs
+                float corr = 1.f;
+                bool rescale = false;
+                if (warp_valid) {
+                    const uint32_t s_addr = tmem_S + b * 128u + lane_addr;
+                    // pass 1: row maximum of the scaled, masked logits
+                    float mx = -CUDART_INF_F;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(s_addr + c * 32, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) {
+                            float s = __uint_as_float(r[e]) * a.scale_log2;
+                            if (need_mask) {
+                                const int kc = key0 + c * 32 + e;
+                                const bool vis = kc < pl || (kc < L && ((anc >> (kc - pl)) & 1ull));
+                                s = vis ? s : -CUDART_INF_F;
+                            }
+                            mx = fmaxf(mx, s);
+                        }
+                    }
+                    if (mx > m_used + kRescaleThreshold || (m_used == -CUDART_INF_F && mx > -CUDART_INF_F)) {
+                        corr = exp2f(m_used - mx);                 // 0 when nothing was accumulated yet
+                        l *= corr;
+                        m_used = mx;
+                        rescale = t > 0;
+                    }
+                    const float m_safe = m_used == -CUDART_INF_F ? 0.f : m_used;
+                    // pass 2: P = exp2(s - m), row sum, pack to bf16
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(s_addr + c * 32, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2) {
+                            float p0 = fast_exp2(fmaf(__uint_as_float(r[e]), a.scale_log2, -m_safe));
+                            float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, -m_safe));
+                            if (need_mask) {
+                                const int kc = key0 + c * 32 + e;
+                                const bool v0 = kc < pl || (kc < L && ((anc >> (kc - pl)) & 1ull));
+                                const bool v1 = kc + 1 < pl || (kc + 1 < L && ((anc >> (kc + 1 - pl)) & 1ull));
+                                p0 = v0 ? p0 : 0.f;
+                                p1 = v1 ? p1 : 0.f;
+                            }
+                            l += p0 + p1;
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                            pk[c * 16 + (e >> 1)] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(&bars->s_free[b]);
+                // P buffer and O accumulator are free once the previous tile's P V product has completed
+                if (it > 0) {
+                    ok = mbar_wait(&bars->pv_done, (it - 1) & 1u, bars, a.status_word);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                if (warp_valid) {
+                    if (__any_sync(0xffffffffu, rescale)) {
+                        const float f = rescale ? corr : 1.f;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t r[32];
+                            tmem_ld32(tmem_O + lane_addr + c * 32, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
+                            tmem_st32(tmem_O + lane_addr + c * 32, r);
+                        }
+                        tmem_wait_st();
+                    }
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const uint32_t dst = sP + (uint32_t)(c >> 3) * 16384u + (uint32_t)row * 128u + (uint32_t)(((c & 7) ^ (row & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * c]), "r"(pk[4 * c + 1]),
+                                     "r"(pk[4 * c + 2]), "r"(pk[4 * c + 3]) : "memory");
+                    }
+                }
+                // the last tile may hold rows past the request's last key: their V must not be NaN garbage (P is 0 there)
+                if (key0 + kTileKeys > L) {
+                    const uint32_t ld_v = 2u * it + 1u, slot = ld_v % kSlots;      // every tile is two ring loads: K, then V
+                    ok = mbar_wait(&bars->full[slot], (ld_v / kSlots) & 1u, bars, a.status_word);
+                    if (!ok) break;
+                    if (row >= L - key0) {
+                        const uint32_t base = sRing + slot * kSlotBytes + (uint32_t)(row >> 3) * 2048u + (uint32_t)(row & 7) * 128u;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int c = 0; c < 8; ++c)
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + h * 1024u + c * 16u), "r"(0) : "memory");
+                    }
+                }
+                fence_async_proxy();
+                tc_fence_before();
+                mbar_arrive(&bars->p_ready);
+            }
+            if (!ok) break;
+            // epilogue: wait for the unit's last P V product, read O, normalise, store
+            ok = mbar_wait(&bars->pv_done, (it - 1) & 1u, bars, a.status_word);
+            if (!ok) break;
+            tc_fence_after();
+            if (warp_valid) {
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_O + lane_addr + c * 32, r);
+                    tmem_wait_ld();
+                    if (valid) {
+                        if (un.n_chunks == 1) {
+                            uint4* dst = reinterpret_cast<uint4*>(a.out + qrow * 128 + c * 32);
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) {
+                                uint32_t w4[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2 * e]) * inv,
+                                                                                   __uint_as_float(r[v * 8 + 2 * e + 1]) * inv);
+                                    w4[e] = *reinterpret_cast<const uint32_t*>(&h);
+                                }
+                                dst[v] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                            }
+                        } else {
+                            uint4* dst = reinterpret_cast<uint4*>(a.w.part_o + ((size_t)u * a.w.rows + row) * 128 + c * 32);
+#pragma unroll
+                            for (int v = 0; v < 8; ++v) dst[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                        }
+                    }
+                }
+                if (valid) {
+                    if (un.n_chunks == 1) {
+                        if (a.lse) a.lse[qrow] = (m_used + log2f(l)) * kLn2;
+                    } else {
+                        a.w.part_ml[((size_t)u * a.w.rows + row) * 2] = m_used;
+                        a.w.part_ml[((size_t)u * a.w.rows + row) * 2 + 1] = l;
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+    }
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// A pool [num_pages, Hkv, page_size, 128] bf16 seen as blocks of (page, head): [blocks][token/8][d/64][token%8][d%64].
+bool make_pool_map(CUtensorMap* map, const void* pool, long long num_pages, int Hkv, int page_size) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[5] = {64, 8, 2, (cuuint64_t)(page_size / 8), (cuuint64_t)(num_pages * Hkv)};
+    const cuuint64_t strides[4] = {256, 128, 2048, (cuuint64_t)page_size * 256};
+    const cuuint32_t box[5] = {64, 8, 2, (cuuint32_t)(page_size / 8), 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(pool), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
 
 war_status_t war_attn_launch_sm100(const void* q, const void* k, const void* v, const int32_t* page_table,
                                    const int32_t* prefix_len, const war_attn_params_t* p, const AttnWorkspace& w,
                                    void* out, float* lse, int* status_word, cudaStream_t s) {
-    return war_attn_launch_simple(q, k, v, page_table, prefix_len, p, w, out, lse, status_word, s);
+    static int sm_count[64] = {0};
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    WAR_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return WAR_ERR_UNSUPPORTED;
+    if (!sm_count[dev]) WAR_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+    if (!attr_set[dev]) {
+        WAR_CUDA_TRY(cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        attr_set[dev] = true;
+    }
+    if (p->num_pages == 0) return WAR_ERR_INVALID_ARG;
+    CUtensorMap k_map, v_map;
+    if (!make_pool_map(&k_map, k, p->num_pages, p->Hkv, p->page_size) || !make_pool_map(&v_map, v, p->num_pages, p->Hkv, p->page_size))
+        return WAR_ERR_CUDA;
+    KernelArgs a;
+    a.q = (const __nv_bfloat16*)q; a.page_table = page_table; a.prefix_len = prefix_len;
+    a.out = (__nv_bfloat16*)out; a.lse = lse; a.status_word = status_word; a.w = w;
+    a.num_pages = p->num_pages; a.scale_log2 = p->scale * kLog2e;
+    a.N = p->N; a.Hq = p->Hq; a.Hkv = p->Hkv; a.G = p->Hq / p->Hkv; a.page_size = p->page_size; a.max_pages = p->max_pages_per_req;
+    attn_sm100_kernel<<<sm_count[dev], kThreads, kSmemBytes, s>>>(k_map, v_map, a);
+    WAR_LAUNCH_CHECK();
+    return WAR_OK;
 }
