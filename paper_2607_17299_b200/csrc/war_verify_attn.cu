@@ -293,7 +293,7 @@ bool contiguous_head_major(const int64_t* s, const war_attn_params_t* p) {
 war_status_t check_params(const war_attn_params_t* p) {
     if (!p) return WAR_ERR_INVALID_ARG;
     if (p->B < 0 || p->N < 1 || p->N > 64 || p->Hq < 1 || p->Hkv < 1 || p->Hq % p->Hkv != 0 || p->max_pages_per_req < 0 ||
-        p->num_pages < 0 || p->kernel < 0 || p->kernel > 1)
+        p->num_pages < 0 || p->kernel < 0 || p->kernel > 1 || !(p->scale > 0.f))
         return WAR_ERR_INVALID_ARG;
     if (p->D != 128 || (p->page_size != 16 && p->page_size != 32)) return WAR_ERR_UNSUPPORTED;
     if ((p->Hq / p->Hkv) * p->N > 512 || p->B > kMaxPlanB) return WAR_ERR_UNSUPPORTED;

@@ -2,16 +2,19 @@
 // online softmax -> tcgen05.mma again, one persistent CTA per SM.
 //
 // Work unit (see war_attn_plan.cuh): up to 128 query rows (slot, head-of-group) of one kv head against a range of
-// 128-key tiles.  Per tile:   S = Q K^T   (M=128 rows, N=128 keys, K=128 dims; bf16 in, fp32 in TMEM)
+// 128-key tiles.  Per tile:   S = Q K^T   (M=128 rows, N=128 keys, K=128 dims; bf16 operands in shared memory)
 //                             P = exp2(S*scale*log2e - m), masked by the tree's ancestor bits on tree columns
-//                             O += P V    (M=128 rows, N=128 dims, K=128 keys; P staged in shared memory as bf16)
-// Warp roles:  warp 0  producer: reads the page table, issues one TMA tensor copy per (page, head) into a ring of
-//                      32 KB slots (K tile, V tile, K tile, ...); no multicast, this GPU's memory only
-//              warp 1  MMA issuer (one lane): S(t+1) is issued before PV(t) so the tensor pipe works while the
-//                      softmax warps are busy; owns the TMEM allocation
-//              warps 2-5  softmax: one thread per query row (TMEM lane), running max/sum in registers, rescale of
-//                      O in TMEM only when the max grows by more than 2^8, epilogue
-// Shared-memory operand layouts are the canonical 128-byte-swizzled ones: K-major for Q, K and P, MN-major for V.
+//                             O += P V    (M=128 rows, N=128 dims, K=128 keys; P is read from TMEM)
+// Tiles alternate between two softmax groups, each with its own S/P region, running (max, sum) and O accumulator
+// in TMEM; the two partial results are merged once per unit.  Nothing synchronises the groups per tile.
+// Warp roles:  warp 0   producer: reads the page table, issues one TMA tensor copy per (page, head) into a ring of
+//                       32 KB slots in the order the tensor pipe consumes them (K0 K1 V0 K2 V1 ...); no multicast,
+//                       this GPU's memory only
+//              warp 1   MMA issuer (one lane): S(t+2) is queued right behind PV(t); owns the TMEM allocation
+//              warps 2-5 / 6-9  softmax group 0 / 1: one thread per query row (TMEM lane); the row of S is pulled
+//                       into registers, P goes back into the first 64 columns of the same TMEM region as packed
+//                       bf16; O is rescaled in TMEM only when the running max grows by more than 2^8
+// Shared-memory operand layouts are the canonical 128-byte-swizzled ones: K-major for Q and K, MN-major for V.
 // A (page, head) block lands as [token/8][d/64][token%8][d%64], which serves both K (K-major, 8-row groups 2 KB
 // apart) and V (MN-major, 64-wide column blocks 1 KB apart, 8-key groups 2 KB apart) with one copy per block.
 // Every wait is bounded: on expiry the kernel records WAR_ERR_TIMEOUT, raises a CTA-wide abort flag and returns.
@@ -25,27 +28,28 @@ namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr int kSlots = 5;
+constexpr int kSlots = 6;
 constexpr int kSlotBytes = 32768;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;           // log2 units
 constexpr unsigned long long kWaitBudgetNs = 2000000000ull;
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;
-constexpr int kOffP = 32768;
-constexpr int kOffRing = 65536;
+constexpr int kOffRing = 32768;
 constexpr int kOffBar = kOffRing + kSlots * kSlotBytes;
-constexpr int kSmemBytes = kOffBar + 256 + 1024;
+constexpr int kOffStats = kOffBar + 256;
+constexpr int kSmemBytes = kOffStats + 1024 + 1024;
 
 struct Bars {
     uint64_t full[kSlots], empty[kSlots];
-    uint64_t s_ready[2], s_free[2];
-    uint64_t p_ready, pv_done, q_ready;
+    uint64_t s_ready[2], p_ready[2], pv_done[2];
+    uint64_t q_ready, stats_ready, epi_done;
     uint32_t tmem_base;
     int abort_flag;
 };
+static_assert(sizeof(Bars) <= 256, "barrier block");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -140,6 +144,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
           "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
           "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -149,8 +160,20 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
 // Unit k of this CTA under the snake deal of the longest-first list: even rounds left to right, odd rounds back.
 __device__ __forceinline__ int snake_unit(int k, int cta, int ctas) { return k * ctas + ((k & 1) ? ctas - 1 - cta : cta); }
+
+// Ring sequence numbers inside a unit of T tiles whose first load has number ld0.  Loads are issued in the order
+// the tensor pipe consumes them: K0, K1, V0, K2, V1, ..., K(T-1), V(T-2), V(T-1).
+__device__ __forceinline__ uint32_t seq_k(uint32_t ld0, int t) { return t == 0 ? ld0 : ld0 + 2u * t - 1u; }
+__device__ __forceinline__ uint32_t seq_v(uint32_t ld0, int t, int T) { return t == T - 1 ? ld0 + 2u * T - 1u : ld0 + 2u * t + 2u; }
 
 struct KernelArgs {
     const __nv_bfloat16* q;
@@ -165,12 +188,17 @@ struct KernelArgs {
     int N, Hq, Hkv, G, page_size, max_pages;
 };
 
+__device__ __forceinline__ bool key_visible(int kc, int pl, int L, uint64_t anc) {
+    return kc < pl || (kc < L && ((anc >> (kc - pl)) & 1ull));
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const KernelArgs a) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     Bars* bars = (Bars*)(smem + kOffBar);
-    const uint32_t sQ = smem_u32(smem + kOffQ), sP = smem_u32(smem + kOffP), sRing = smem_u32(smem + kOffRing);
+    float2* stats = (float2*)(smem + kOffStats);     // group 1's (max, sum) per row, for the merge
+    const uint32_t sQ = smem_u32(smem + kOffQ), sRing = smem_u32(smem + kOffRing);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_units = a.w.counters[1];
     const int pages_per_tile = kTileKeys / a.page_size;
@@ -178,10 +206,10 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
 
     if (tid == 0) {
         for (int i = 0; i < kSlots; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&bars->s_ready[i], 1); mbar_init(&bars->s_free[i], 128); }
-        mbar_init(&bars->p_ready, 128);
-        mbar_init(&bars->pv_done, 1);
-        mbar_init(&bars->q_ready, 128);
+        for (int i = 0; i < 2; ++i) { mbar_init(&bars->s_ready[i], 1); mbar_init(&bars->p_ready[i], 128); mbar_init(&bars->pv_done[i], 1); }
+        mbar_init(&bars->q_ready, 256);
+        mbar_init(&bars->stats_ready, 128);
+        mbar_init(&bars->epi_done, 128);
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -193,12 +221,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
-    const uint32_t tmem_S = tmem;                    // two buffers of 128 columns
-    const uint32_t tmem_O = tmem + 256;              // 128 columns
+    // columns: [0,128) S/P of group 0, [128,256) S/P of group 1, [256,384) O of group 0, [384,512) O of group 1
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
-        uint32_t ld = 0;                             // half-tile loads issued so far
+        uint32_t ld = 0;
         bool ok = true;
         for (int k = 0; ok; ++k) {
             const int u = snake_unit(k, blockIdx.x, gridDim.x);
@@ -208,101 +235,103 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
             const int L = a.prefix_len[i] + a.w.req[i].n_nodes;
             const int total_pages = (L + a.page_size - 1) / a.page_size;
             const int32_t* pt = a.page_table + (size_t)i * a.max_pages;
-            int page_next = -1;
-            if (lane < pages_per_tile) {
-                const int pi = un.tile_begin * pages_per_tile + lane;
-                page_next = pi < total_pages ? pt[pi] : -1;
-            }
-            for (int t = un.tile_begin; t < un.tile_end && ok; ++t) {
-                const int page = page_next;
-                if (t + 1 < un.tile_end && lane < pages_per_tile) {          // prefetch the next tile's page ids
-                    const int pi = (t + 1) * pages_per_tile + lane;
-                    page_next = pi < total_pages ? pt[pi] : -1;
-                }
-                const int n_valid = min(pages_per_tile, total_pages - t * pages_per_tile);
-                int block = -1;
+            const int T = un.tile_end - un.tile_begin;
+            auto page_of = [&](int t) -> int {                   // this lane's page id in local tile t (-1: none)
+                if (t >= T || lane >= pages_per_tile) return -1;
+                const int pi = (un.tile_begin + t) * pages_per_tile + lane;
+                return pi < total_pages ? pt[pi] : -1;
+            };
+            auto load = [&](int t, int page, bool is_v) -> bool {
+                const uint32_t slot = ld % kSlots, phase = (ld / kSlots) & 1u;
+                ++ld;
+                bool w = mbar_wait(&bars->empty[slot], phase ^ 1u, bars, a.status_word);
+                w = __all_sync(0xffffffffu, w);
+                if (!w) return false;
+                const int n_valid = min(pages_per_tile, total_pages - (un.tile_begin + t) * pages_per_tile);
+                if (lane == 0) mbar_arrive_expect_tx(&bars->full[slot], (uint32_t)n_valid * page_bytes);
+                __syncwarp();
                 if (lane < n_valid) {
                     long long pg = page;
                     if (pg < 0 || pg >= a.num_pages) { war_set_device_status(a.status_word, WAR_ERR_BAD_PAGE); pg = 0; }
-                    block = (int)(pg * a.Hkv + un.kvh);
+                    tma_load_block(sRing + slot * kSlotBytes + lane * page_bytes, is_v ? &v_map : &k_map,
+                                   (int)(pg * a.Hkv + un.kvh), &bars->full[slot]);
                 }
-#pragma unroll
-                for (int which = 0; which < 2; ++which, ++ld) {
-                    const uint32_t slot = ld % kSlots, phase = (ld / kSlots) & 1u;
-                    ok = mbar_wait(&bars->empty[slot], phase ^ 1u, bars, a.status_word);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    if (lane == 0) mbar_arrive_expect_tx(&bars->full[slot], (uint32_t)n_valid * page_bytes);
-                    __syncwarp();
-                    if (block >= 0)
-                        tma_load_block(sRing + slot * kSlotBytes + lane * page_bytes, which ? &v_map : &k_map, block, &bars->full[slot]);
-                }
+                return true;
+            };
+            int pg_cur = page_of(0), pg_nxt = page_of(1);
+            ok = load(0, pg_cur, false);                                    // K0
+            for (int t = 0; t < T && ok; ++t) {
+                const int pg_nn = page_of(t + 2);                            // page ids two tiles ahead, off the critical path
+                if (t + 1 < T) ok = load(t + 1, pg_nxt, false);              // K(t+1)
+                if (ok) ok = load(t, pg_cur, true);                          // V(t)
+                pg_cur = pg_nxt; pg_nxt = pg_nn;
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        uint32_t ld = 0, it = 0, units_done = 0;
+        uint32_t ld0 = 0, cg[2] = {0, 0}, units_done = 0;
         constexpr uint32_t idesc_s = umma_idesc(128, 128, 0);
         constexpr uint32_t idesc_o = umma_idesc(128, 128, 1);
         bool ok = true;
-        auto issue_s = [&](uint32_t it_s, uint32_t ld_k) -> bool {
-            const uint32_t slot = ld_k % kSlots, b = it_s & 1u;
-            if (!mbar_wait(&bars->full[slot], (ld_k / kSlots) & 1u, bars, a.status_word)) return false;
-            if (!mbar_wait(&bars->s_free[b], ((it_s >> 1) & 1u) ^ 1u, bars, a.status_word)) return false;
-            tc_fence_after();
-            if (lane == 0) {
-                const uint32_t kb = sRing + slot * kSlotBytes;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32u;
-                    const uint32_t koff = (uint32_t)(ks >> 2) * 1024u + (uint32_t)(ks & 3) * 32u;
-                    umma_bf16(tmem_S + b * 128u, umma_desc(sQ + off, 16, 1024), umma_desc(kb + koff, 16, 2048), idesc_s, ks > 0);
-                }
-                umma_commit(&bars->s_ready[b]);
-                umma_commit(&bars->empty[slot]);
-            }
-            __syncwarp();
-            return true;
-        };
         for (int k = 0; ok; ++k) {
             const int u = snake_unit(k, blockIdx.x, gridDim.x);
             if (u >= n_units) break;
             const AttnUnit un = a.w.units[u];
-            const int n_tiles = un.tile_end - un.tile_begin;
+            const int T = un.tile_end - un.tile_begin;
+            auto issue_s = [&](int t) -> bool {
+                const uint32_t sq = seq_k(ld0, t), slot = sq % kSlots, g = t & 1;
+                if (!mbar_wait(&bars->full[slot], (sq / kSlots) & 1u, bars, a.status_word)) return false;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t kb = sRing + slot * kSlotBytes;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t qoff = (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32u;
+                        const uint32_t koff = (uint32_t)(ks >> 2) * 1024u + (uint32_t)(ks & 3) * 32u;
+                        umma_bf16(tmem + g * 128u, umma_desc(sQ + qoff, 16, 1024), umma_desc(kb + koff, 16, 2048), idesc_s, ks > 0);
+                    }
+                    umma_commit(&bars->s_ready[g]);
+                    umma_commit(&bars->empty[slot]);
+                }
+                __syncwarp();
+                return true;
+            };
             ok = mbar_wait(&bars->q_ready, units_done & 1u, bars, a.status_word);
-            if (!ok) break;
-            ok = issue_s(it, ld);
-            for (int t = 0; t < n_tiles && ok; ++t) {
-                if (t + 1 < n_tiles) ok = issue_s(it + t + 1, ld + 2 * (t + 1));
-                if (!ok) break;
-                const uint32_t ld_v = ld + 2 * t + 1, slot = ld_v % kSlots;
-                ok = mbar_wait(&bars->full[slot], (ld_v / kSlots) & 1u, bars, a.status_word) &&
-                     mbar_wait(&bars->p_ready, (it + t) & 1u, bars, a.status_word);
+            if (ok) ok = issue_s(0);
+            if (ok && T > 1) ok = issue_s(1);
+            for (int t = 0; t < T && ok; ++t) {
+                const uint32_t g = t & 1, tg = cg[g] + (uint32_t)(t >> 1);
+                const uint32_t sq = seq_v(ld0, t, T), slot = sq % kSlots;
+                ok = mbar_wait(&bars->p_ready[g], tg & 1u, bars, a.status_word) &&
+                     mbar_wait(&bars->full[slot], (sq / kSlots) & 1u, bars, a.status_word);
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
                     const uint32_t vb = sRing + slot * kSlotBytes;
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t off = (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32u;
-                        umma_bf16(tmem_O, umma_desc(sP + off, 16, 1024), umma_desc(vb + (uint32_t)ks * 4096u, 1024, 2048), idesc_o,
-                                  (t > 0 || ks > 0) ? 1u : 0u);
-                    }
-                    umma_commit(&bars->pv_done);
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_bf16_ts(tmem + 256u + g * 128u, tmem + g * 128u + (uint32_t)ks * 8u,
+                                     umma_desc(vb + (uint32_t)ks * 4096u, 1024, 2048), idesc_o, (t > 1 || ks > 0) ? 1u : 0u);
+                    umma_commit(&bars->pv_done[g]);
                     umma_commit(&bars->empty[slot]);
                 }
                 __syncwarp();
+                if (t + 2 < T) ok = issue_s(t + 2);
             }
-            it += n_tiles;
-            ld += 2 * n_tiles;
+            cg[0] += (uint32_t)(T + 1) >> 1;
+            cg[1] += (uint32_t)T >> 1;
+            ld0 += 2u * T;
             ++units_done;
         }
     } else {
-        // ------------------------------------------------------------------ softmax / epilogue, one thread per row
+        // ------------------------------------------------------------------ softmax groups, one thread per row
+        const int grp = (warp - 2) >> 2;
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-        uint32_t it = 0;
+        const uint32_t tS = tmem + grp * 128u + lane_addr;          // S, later P, of this group
+        const uint32_t tO = tmem + 256u + grp * 128u + lane_addr;
+        uint32_t ld0 = 0, cgm = 0, cg_other = 0, units_done = 0;    // cgm: tiles this group has processed so far
         bool ok = true;
         for (int k = 0; ok; ++k) {
             const int u = snake_unit(k, blockIdx.x, gridDim.x);
@@ -319,113 +348,115 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
             const int j = valid ? gr / a.G : 0, g = valid ? gr % a.G : 0;
             const size_t qrow = ((size_t)i * a.N + j) * a.Hq + un.kvh * a.G + g;
             const uint64_t anc = valid ? a.w.anc[(size_t)i * a.N + j] : 0ull;
-            // previous unit's MMAs are complete (its last pv_done was awaited in the epilogue), so Q may be replaced
-            {
-                const uint4* src = reinterpret_cast<const uint4*>(a.q + qrow * 128);
+            const int T = un.tile_end - un.tile_begin;
+            // group 1 may not touch Q, O or its statistics before group 0 has finished the previous unit's epilogue
+            if (grp == 1 && units_done > 0) {
+                ok = mbar_wait(&bars->epi_done, (units_done - 1) & 1u, bars, a.status_word);
+                if (!ok) break;
+            }
+            {   // each group writes one 64-wide half of every Q row (swizzled K-major)
+                const uint4* src = reinterpret_cast<const uint4*>(a.q + qrow * 128) + grp * 8;
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
+                for (int c = 0; c < 8; ++c) {
                     const uint4 x = valid ? src[c] : make_uint4(0, 0, 0, 0);
-                    const uint32_t dst = sQ + (uint32_t)(c >> 3) * 16384u + (uint32_t)row * 128u + (uint32_t)(((c & 7) ^ (row & 7)) << 4);
+                    const uint32_t dst = sQ + (uint32_t)grp * 16384u + (uint32_t)row * 128u + (uint32_t)((c ^ (row & 7)) << 4);
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(x.x), "r"(x.y), "r"(x.z), "r"(x.w) : "memory");
                 }
             }
             fence_async_proxy();
             mbar_arrive(&bars->q_ready);
             float m_used = -CUDART_INF_F, l = 0.f;
-            const int n_tiles = un.tile_end - un.tile_begin;
-            for (int t = 0; t < n_tiles && ok; ++t, ++it) {
-                const uint32_t b = it & 1u;
+            for (int t = grp; t < T && ok; t += 2, ++cgm) {
                 const int key0 = (un.tile_begin + t) * kTileKeys;
                 const bool need_mask = key0 + kTileKeys > pl;
-                ok = mbar_wait(&bars->s_ready[b], (it >> 1) & 1u, bars, a.status_word);
+                ok = mbar_wait(&bars->s_ready[grp], cgm & 1u, bars, a.status_word);
                 if (!ok) break;
                 tc_fence_after();
-                uint32_t pk[64];                                   // P as packed bf16 pairs
-                float corr = 1.f;
-                bool rescale = false;
                 if (warp_valid) {
-                    const uint32_t s_addr = tmem_S + b * 128u + lane_addr;
-                    // pass 1: row maximum of the scaled, masked logits
-                    float mx = -CUDART_INF_F;
+                    // pass 1: row maximum (four independent chains); the whole row is in flight at once
+                    float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+                    {
+                        uint32_t r[128];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t r[32];
-                        tmem_ld32(s_addr + c * 32, r);
+                        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, r + c * 32);
                         tmem_wait_ld();
+                        if (need_mask) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            float s = __uint_as_float(r[e]) * a.scale_log2;
-                            if (need_mask) {
-                                const int kc = key0 + c * 32 + e;
-                                const bool vis = kc < pl || (kc < L && ((anc >> (kc - pl)) & 1ull));
-                                s = vis ? s : -CUDART_INF_F;
-                            }
-                            mx = fmaxf(mx, s);
+                            for (int e = 0; e < 128; ++e)
+                                if (!key_visible(key0 + e, pl, L, anc)) r[e] = 0xff800000u;     // -inf
+                        }
+#pragma unroll
+                        for (int e = 0; e < 128; e += 4) {
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) mx4[v] = fmaxf(mx4[v], __uint_as_float(r[e + v]));
                         }
                     }
+                    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;    // scale > 0
+                    float corr = 1.f;
+                    bool rescale = false;
                     if (mx > m_used + kRescaleThreshold || (m_used == -CUDART_INF_F && mx > -CUDART_INF_F)) {
                         corr = exp2f(m_used - mx);                 // 0 when nothing was accumulated yet
                         l *= corr;
                         m_used = mx;
-                        rescale = t > 0;
+                        rescale = t > grp;                         // O of this group holds earlier tiles of the unit
                     }
-                    const float m_safe = m_used == -CUDART_INF_F ? 0.f : m_used;
-                    // pass 2: P = exp2(s - m), row sum, pack to bf16
+                    const float neg_m = m_used == -CUDART_INF_F ? 0.f : -m_used;
+                    // pass 2: P = exp2(s*scale - m) in 32-column pieces, the next piece loading while this one is processed
+                    float l4[4] = {0.f, 0.f, 0.f, 0.f};
+                    uint32_t pk[64];
+                    uint32_t buf[2][32];
+                    tmem_ld32(tS, buf[0]);
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        uint32_t r[32];
-                        tmem_ld32(s_addr + c * 32, r);
                         tmem_wait_ld();
+                        if (c < 3) tmem_ld32(tS + (c + 1) * 32, buf[(c + 1) & 1]);
+                        uint32_t* r = buf[c & 1];
+                        if (need_mask) {
 #pragma unroll
-                        for (int e = 0; e < 32; e += 2) {
-                            float p0 = fast_exp2(fmaf(__uint_as_float(r[e]), a.scale_log2, -m_safe));
-                            float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 1]), a.scale_log2, -m_safe));
-                            if (need_mask) {
-                                const int kc = key0 + c * 32 + e;
-                                const bool v0 = kc < pl || (kc < L && ((anc >> (kc - pl)) & 1ull));
-                                const bool v1 = kc + 1 < pl || (kc + 1 < L && ((anc >> (kc + 1 - pl)) & 1ull));
-                                p0 = v0 ? p0 : 0.f;
-                                p1 = v1 ? p1 : 0.f;
+                            for (int e = 0; e < 32; ++e)
+                                if (!key_visible(key0 + c * 32 + e, pl, L, anc)) r[e] = 0xff800000u;
+                        }
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8) {
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) {
+                                const float p0 = fast_exp2(fmaf(__uint_as_float(r[e + 2 * v]), a.scale_log2, neg_m));       // exp2(-inf) = 0
+                                const float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 2 * v + 1]), a.scale_log2, neg_m));
+                                l4[v] += p0 + p1;
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                                pk[c * 16 + (e >> 1) + v] = *reinterpret_cast<const uint32_t*>(&h);
                             }
-                            l += p0 + p1;
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                            pk[c * 16 + (e >> 1)] = *reinterpret_cast<const uint32_t*>(&h);
                         }
                     }
-                }
-                tc_fence_before();
-                mbar_arrive(&bars->s_free[b]);
-                // P buffer and O accumulator are free once the previous tile's P V product has completed
-                if (it > 0) {
-                    ok = mbar_wait(&bars->pv_done, (it - 1) & 1u, bars, a.status_word);
-                    if (!ok) break;
-                    tc_fence_after();
-                }
-                if (warp_valid) {
+                    l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
                     if (__any_sync(0xffffffffu, rescale)) {
-                        const float f = rescale ? corr : 1.f;
+                        // O of this group is stable once its previous P V product has completed
+                        ok = mbar_wait(&bars->pv_done[grp], (cgm - 1) & 1u, bars, a.status_word);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (ok) {
+                            tc_fence_after();
+                            const float f = rescale ? corr : 1.f;
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t r[32];
-                            tmem_ld32(tmem_O + lane_addr + c * 32, r);
-                            tmem_wait_ld();
+                            for (int c = 0; c < 4; ++c) {
+                                uint32_t o[32];
+                                tmem_ld32(tO + c * 32, o);
+                                tmem_wait_ld();
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
-                            tmem_st32(tmem_O + lane_addr + c * 32, r);
+                                for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
+                                tmem_st32(tO + c * 32, o);
+                            }
                         }
-                        tmem_wait_st();
                     }
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const uint32_t dst = sP + (uint32_t)(c >> 3) * 16384u + (uint32_t)row * 128u + (uint32_t)(((c & 7) ^ (row & 7)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * c]), "r"(pk[4 * c + 1]),
-                                     "r"(pk[4 * c + 2]), "r"(pk[4 * c + 3]) : "memory");
-                    }
+                    tmem_st32(tS, pk);
+                    tmem_st32(tS + 32, pk + 32);
+                    tmem_wait_st();
                 }
-                // the last tile may hold rows past the request's last key: their V must not be NaN garbage (P is 0 there)
+                if (!ok) break;
+                // the unit's last tile may hold rows past the request's last key: zero their V (P is exactly 0 there,
+                // but 0 x NaN garbage would still poison the product)
                 if (key0 + kTileKeys > L) {
-                    const uint32_t ld_v = 2u * it + 1u, slot = ld_v % kSlots;      // every tile is two ring loads: K, then V
-                    ok = mbar_wait(&bars->full[slot], (ld_v / kSlots) & 1u, bars, a.status_word);
+                    const uint32_t sq = seq_v(ld0, t, T), slot = sq % kSlots;
+                    ok = mbar_wait(&bars->full[slot], (sq / kSlots) & 1u, bars, a.status_word);
                     if (!ok) break;
                     if (row >= L - key0) {
                         const uint32_t base = sRing + slot * kSlotBytes + (uint32_t)(row >> 3) * 2048u + (uint32_t)(row & 7) * 128u;
@@ -435,54 +466,81 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                             for (int c = 0; c < 8; ++c)
                                 asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + h * 1024u + c * 16u), "r"(0) : "memory");
                     }
+                    fence_async_proxy();
                 }
-                fence_async_proxy();
                 tc_fence_before();
-                mbar_arrive(&bars->p_ready);
+                mbar_arrive(&bars->p_ready[grp]);
             }
             if (!ok) break;
-            // epilogue: wait for the unit's last P V product, read O, normalise, store
-            ok = mbar_wait(&bars->pv_done, (it - 1) & 1u, bars, a.status_word);
-            if (!ok) break;
-            tc_fence_after();
-            if (warp_valid) {
-                const float inv = l > 0.f ? 1.f / l : 0.f;
+            const uint32_t mine = (uint32_t)(T + 1 - grp) >> 1, theirs = (uint32_t)(T + grp) >> 1;   // tiles of this unit per group
+            if (grp == 1) {
+                stats[row] = make_float2(m_used, l);
+                mbar_arrive(&bars->stats_ready);
+            } else {
+                // epilogue: both groups' last products, then merge (max, sum, O) of the two groups and store
+                ok = mbar_wait(&bars->pv_done[0], (cgm - 1) & 1u, bars, a.status_word) &&
+                     mbar_wait(&bars->stats_ready, units_done & 1u, bars, a.status_word);
+                if (ok && theirs > 0) ok = mbar_wait(&bars->pv_done[1], (cg_other + theirs - 1) & 1u, bars, a.status_word);
+                if (!ok) break;
+                tc_fence_after();
+                if (warp_valid) {
+                    const float2 st = stats[row];
+                    const float m1 = theirs > 0 ? st.x : -CUDART_INF_F, l1 = theirs > 0 ? st.y : 0.f;
+                    const float M = fmaxf(m_used, m1);
+                    const float w0 = m_used == -CUDART_INF_F ? 0.f : exp2f(m_used - M);
+                    const float w1 = m1 == -CUDART_INF_F ? 0.f : exp2f(m1 - M);
+                    const float lsum = l * w0 + l1 * w1;
+                    const bool split = un.n_chunks != 1;
+                    const float f0 = split ? w0 : (lsum > 0.f ? w0 / lsum : 0.f), f1 = split ? w1 : (lsum > 0.f ? w1 / lsum : 0.f);
+                    const bool use1 = theirs > 0;                  // uniform: O of group 1 is stale when it had no tile
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem_O + lane_addr + c * 32, r);
-                    tmem_wait_ld();
-                    if (valid) {
-                        if (un.n_chunks == 1) {
-                            uint4* dst = reinterpret_cast<uint4*>(a.out + qrow * 128 + c * 32);
+                    for (int c = 0; c < 8; ++c) {
+                        uint32_t o0[16], o1[16];
+                        tmem_ld16(tO + c * 16, o0);
+                        if (use1) tmem_ld16(tO + 128u + c * 16, o1);
+                        tmem_wait_ld();
+                        float x[16];
 #pragma unroll
-                            for (int v = 0; v < 4; ++v) {
-                                uint32_t w4[4];
+                        for (int e = 0; e < 16; ++e) {
+                            x[e] = __uint_as_float(o0[e]) * f0;
+                            if (use1) x[e] = fmaf(__uint_as_float(o1[e]), f1, x[e]);
+                        }
+                        if (valid) {
+                            if (!split) {
+                                uint4* dst = reinterpret_cast<uint4*>(a.out + qrow * 128 + c * 16);
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2 * e]) * inv,
-                                                                                   __uint_as_float(r[v * 8 + 2 * e + 1]) * inv);
-                                    w4[e] = *reinterpret_cast<const uint32_t*>(&h);
+                                for (int v = 0; v < 2; ++v) {
+                                    uint32_t w4[4];
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) {
+                                        const __nv_bfloat162 h = __floats2bfloat162_rn(x[v * 8 + 2 * e], x[v * 8 + 2 * e + 1]);
+                                        w4[e] = *reinterpret_cast<const uint32_t*>(&h);
+                                    }
+                                    dst[v] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                                 }
-                                dst[v] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-                            }
-                        } else {
-                            uint4* dst = reinterpret_cast<uint4*>(a.w.part_o + ((size_t)u * a.w.rows + row) * 128 + c * 32);
+                            } else {
+                                float4* dst = reinterpret_cast<float4*>(a.w.part_o + ((size_t)u * a.w.rows + row) * 128 + c * 16);
 #pragma unroll
-                            for (int v = 0; v < 8; ++v) dst[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                                for (int v = 0; v < 4; ++v) dst[v] = make_float4(x[4 * v], x[4 * v + 1], x[4 * v + 2], x[4 * v + 3]);
+                            }
+                        }
+                    }
+                    if (valid) {
+                        if (!split) {
+                            if (a.lse) a.lse[qrow] = (M + log2f(lsum)) * kLn2;
+                        } else {
+                            a.w.part_ml[((size_t)u * a.w.rows + row) * 2] = M;
+                            a.w.part_ml[((size_t)u * a.w.rows + row) * 2 + 1] = lsum;
                         }
                     }
                 }
-                if (valid) {
-                    if (un.n_chunks == 1) {
-                        if (a.lse) a.lse[qrow] = (m_used + log2f(l)) * kLn2;
-                    } else {
-                        a.w.part_ml[((size_t)u * a.w.rows + row) * 2] = m_used;
-                        a.w.part_ml[((size_t)u * a.w.rows + row) * 2 + 1] = l;
-                    }
-                }
+                tc_fence_before();
+                mbar_arrive(&bars->epi_done);
             }
-            tc_fence_before();
+            (void)mine;
+            cg_other += theirs;
+            ld0 += 2u * T;
+            ++units_done;
         }
     }
     // ---------------------------------------------------------------------- teardown
