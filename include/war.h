@@ -146,6 +146,29 @@ war_status_t war_verify_attn(const void* d_q, const void* d_kpool, const void* d
                              void* d_out, float* d_lse, war_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * war_verify_attn for callers that cannot allocate device memory.  The paper has no counterpart: this is a
+ * packaging variant of the call above, for users such as an engine whose memory pool is already frozen when the
+ * decode loop runs, a plugin that only ever receives its input and output buffers, or a thread that must not
+ * enter the CUDA allocator.  Same arguments and results as war_verify_attn, without d_workspace: the scratch
+ * (work list, split-KV partials) lives in one fixed array inside the library image, WAR_VERIFY_ATTN_NOALLOC_MAX_BYTES
+ * long, which every GPU that loads the library holds until the process exits.
+ *   - The call allocates nothing and frees nothing (no cudaMalloc/cudaFree, no allocating library routine).
+ *   - If war_verify_attn_workspace_bytes(params) exceeds WAR_VERIFY_ATTN_NOALLOC_MAX_BYTES the call returns
+ *     WAR_ERR_CAPACITY and launches nothing.
+ *   - The first call on each device looks up the array's device address (with that device current); make that
+ *     first call before starting any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents (nothing in it needs
+ *     clearing: every call rewrites what it reads).  Two calls that overlap on the GPU, e.g. on two streams,
+ *     race on it; run them in stream order.
+ * ------------------------------------------------------------------------------------------------ */
+#define WAR_VERIFY_ATTN_NOALLOC_MAX_BYTES (64u * 1024u * 1024u)
+war_status_t war_verify_attn_noalloc(const void* d_q, const void* d_kpool, const void* d_vpool,
+                                     const int32_t* d_page_table, const int32_t* d_prefix_len,
+                                     const int32_t* d_num_nodes, const int32_t* d_parent,
+                                     const war_attn_params_t* params, void* d_out, float* d_lse,
+                                     war_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
  * Accept (paper Section 2.3: drafts are verified "while preserving the target output distribution";
  * Section 3.2: the rollout advances "by multiple tokens ... when the drafts are accepted").  The caller
  * supplies the target model's own token choices; a draft slot is accepted iff every slot on its root path

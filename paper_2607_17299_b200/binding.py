@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "WAR_OK", 1: "WAR_ERR_INVALID_ARG", 2: "WAR_ERR_OOM", 3: "WAR
                 5: "WAR_ERR_TIMEOUT", 6: "WAR_ERR_UNSUPPORTED", 7: "WAR_ERR_BAD_TREE", 8: "WAR_ERR_BAD_PAGE"}
 
 EXPORTS = ["war_index_build", "war_index_append", "war_index_info", "war_index_destroy", "war_draft",
-           "war_verify_attn_workspace_bytes", "war_verify_attn", "war_accept", "war_device_status",
+           "war_verify_attn_workspace_bytes", "war_verify_attn", "war_verify_attn_noalloc", "war_accept", "war_device_status",
            "war_status_string"]
 
 
@@ -70,6 +70,8 @@ _lib.war_verify_attn_workspace_bytes.restype = C.c_size_t
 _lib.war_verify_attn_workspace_bytes.argtypes = [C.POINTER(AttnParams)]
 _lib.war_verify_attn.restype = C.c_int
 _lib.war_verify_attn.argtypes = [C.c_void_p] * 7 + [C.POINTER(AttnParams)] + [C.c_void_p] * 4
+_lib.war_verify_attn_noalloc.restype = C.c_int
+_lib.war_verify_attn_noalloc.argtypes = [C.c_void_p] * 7 + [C.POINTER(AttnParams)] + [C.c_void_p] * 3
 _lib.war_accept.restype = C.c_int
 _lib.war_accept.argtypes = [C.c_void_p] * 4 + [C.c_int32] * 3 + [C.c_void_p] * 4
 _lib.war_device_status.restype = C.c_int
@@ -197,6 +199,25 @@ def war_verify_attn(d_q: torch.Tensor, d_kpool: torch.Tensor, d_vpool: torch.Ten
                                 _ptr(d_num_nodes, torch.int32), _ptr(d_parent, torch.int32), C.byref(params),
                                 _ptr(d_workspace), _ptr(d_out, torch.bfloat16), _ptr(d_lse, torch.float32), _stream())
     _check("war_verify_attn", code)
+
+
+NOALLOC_MAX_BYTES = 64 * 1024 * 1024
+
+
+def war_verify_attn_noalloc(d_q: torch.Tensor, d_kpool: torch.Tensor, d_vpool: torch.Tensor, d_page_table: torch.Tensor,
+                            d_prefix_len: torch.Tensor, d_num_nodes: torch.Tensor, d_parent: torch.Tensor,
+                            params: AttnParams, d_out: torch.Tensor, d_lse: Optional[torch.Tensor]) -> None:
+    """war_verify_attn without a workspace argument, for callers that cannot allocate device memory: the scratch
+    is a fixed array inside the library (NOALLOC_MAX_BYTES).  Calls on one device share it, so keep them in stream
+    order; make the first call on a device outside any stream capture."""
+    for t in (d_kpool, d_vpool):
+        if not t.is_cuda or t.dtype != torch.bfloat16:
+            raise ValueError("pools must be bf16 CUDA tensors")
+    code = _lib.war_verify_attn_noalloc(_ptr(d_q, torch.bfloat16), d_kpool.data_ptr(), d_vpool.data_ptr(),
+                                        _ptr(d_page_table, torch.int32), _ptr(d_prefix_len, torch.int32),
+                                        _ptr(d_num_nodes, torch.int32), _ptr(d_parent, torch.int32), C.byref(params),
+                                        _ptr(d_out, torch.bfloat16), _ptr(d_lse, torch.float32), _stream())
+    _check("war_verify_attn_noalloc", code)
 
 
 def war_accept(d_ids: torch.Tensor, d_parent: torch.Tensor, d_num_nodes: torch.Tensor, d_target_ids: torch.Tensor,
