@@ -25,15 +25,21 @@ constexpr int kMaxK = 8;
 constexpr int kMaxP = 32;
 constexpr int kPoolCap = kMaxN * kMaxK;
 constexpr int kBlockScanMin = 8192;          // intervals at least this long are scanned by every warp
+constexpr int kLongRunFirstMin = 1024;       // intervals at least this long first look for runs of 16 or more only
 
 struct TopK {                                 // warp-uniform, sorted by (cnt desc, start asc)
     int cnt[kMaxK];
     int start[kMaxK];
-    int tok[kMaxK];
     int n;
 };
 
-__device__ __forceinline__ void topk_insert(TopK& t, int k, int cnt, int start, int tok) {
+__device__ __forceinline__ void topk_clear(TopK& t) {
+    t.n = 0;
+#pragma unroll
+    for (int i = 0; i < kMaxK; ++i) { t.cnt[i] = 0; t.start[i] = 0; }
+}
+
+__device__ __forceinline__ void topk_insert(TopK& t, int k, int cnt, int start) {
     // position = first entry that ranks below the newcomer
     int pos = t.n;
 #pragma unroll
@@ -42,10 +48,10 @@ __device__ __forceinline__ void topk_insert(TopK& t, int k, int cnt, int start, 
     if (pos >= k) return;
 #pragma unroll
     for (int i = kMaxK - 1; i >= 1; --i)
-        if (i > pos && i < k) { t.cnt[i] = t.cnt[i - 1]; t.start[i] = t.start[i - 1]; t.tok[i] = t.tok[i - 1]; }
+        if (i > pos && i < k) { t.cnt[i] = t.cnt[i - 1]; t.start[i] = t.start[i - 1]; }
 #pragma unroll
     for (int i = 0; i < kMaxK; ++i)
-        if (i == pos) { t.cnt[i] = cnt; t.start[i] = start; t.tok[i] = tok; }
+        if (i == pos) { t.cnt[i] = cnt; t.start[i] = start; }
     if (t.n < k) ++t.n;
 }
 
@@ -61,67 +67,98 @@ __device__ __forceinline__ unsigned le_mask16(uint4 v, unsigned drep) {
     return out;
 }
 
-// One warp scans positions [sb, se) of the interval [lo, hi) at depth d.  Complete runs (both boundaries inside
-// the span) go to the warp's top-k; the first and last boundary are returned for stitching.
-__device__ void warp_scan_span(const uint8_t* __restrict__ lcp, const int32_t* __restrict__ sa,
-                               const int32_t* __restrict__ corpus, int d, int sb, int se, int k, int lane,
-                               TopK& tk, int& first_b, int& last_b) {
-    tk.n = 0;
-#pragma unroll
-    for (int i = 0; i < kMaxK; ++i) { tk.cnt[i] = 0; tk.start[i] = 0; tk.tok[i] = 0; }
-    int thr = 0;                                           // a run must beat this count to enter the top-k
+// One warp scans positions [sb, se) of a node's token range at depth d (suffixes that end at d are already cut
+// off, so every run is a real continuation token).  Complete runs (both boundaries inside the span) go to the
+// warp's top-k; the first and last boundary are returned for stitching.  No token is read here: a run is known by
+// (count, start) and its token is looked up once, for the winners only.
+//
+// thr_shared is the largest "k-th best count" any warp of the CTA has published for this node: k runs at least
+// that long exist somewhere in the node, so a run shorter than that cannot be among the node's k best (an equally
+// long one still can, by its earlier start).  Once the bar is at 16 or more, no run that lies inside one lane's 16
+// positions can pass it, and only the run ending at a lane's first boundary needs a look.
+__device__ void warp_scan_span(const uint8_t* __restrict__ lcp, int d, int sb, int se, int k, int lane,
+                               TopK& tk, int& first_b, int& last_b, int* thr_shared) {
+    topk_clear(tk);
+    int thr_local = 0;                                     // a run must beat this count to enter this warp's top-k
     int carry = -1, my_first = -1;
     const unsigned drep = 0x01010101u * (unsigned)d;
-    for (int base = sb & ~15; base < se; base += 512) {
-        const int pos0 = base + lane * 16;
-        unsigned bits = 0;
-        if (pos0 < se) {
-            const uint4 v = *reinterpret_cast<const uint4*>(lcp + pos0);
-            bits = le_mask16(v, drep);
-            if (pos0 < sb) bits &= ~((1u << (sb - pos0)) - 1u);
-            if (pos0 + 16 > se) bits &= (1u << (se - pos0)) - 1u;
-        }
-        int last_pos = bits ? pos0 + 31 - __clz(bits) : -1;
-        int incl = last_pos;
+    constexpr int kAhead = 4;                               // 16-byte loads in flight per lane (2 KB per warp step)
+    for (int base0 = sb & ~15; base0 < se; base0 += 512 * kAhead) {
+        uint4 v[kAhead];
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int y = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl = max(incl, y);
+        for (int q = 0; q < kAhead; ++q) {
+            const int p0 = base0 + q * 512 + lane * 16;
+            v[q] = p0 < se ? *reinterpret_cast<const uint4*>(lcp + p0) : make_uint4(0, 0, 0, 0);
         }
-        int prev = __shfl_up_sync(0xffffffffu, incl, 1);
-        if (lane == 0) prev = -1;
-        prev = max(prev, carry);
-        carry = max(carry, __shfl_sync(0xffffffffu, incl, 31));
-        // candidates in ascending position order: lowest lane first, ascending inside a lane
-        bool have = false;
-        int c_cnt = 0, c_start = 0;
-        while (true) {
-            if (!have) {
-                while (bits) {
-                    const int t = __ffs(bits) - 1;
-                    bits &= bits - 1;
-                    const int bpos = pos0 + t;
+#pragma unroll
+        for (int q = 0; q < kAhead; ++q) {
+            const int base = base0 + q * 512;
+            if (base >= se) break;                              // warp-uniform
+            const int pos0 = base + lane * 16;
+            unsigned bits = 0;
+            if (pos0 < se) {
+                bits = le_mask16(v[q], drep);
+                if (pos0 < sb) bits &= ~((1u << (sb - pos0)) - 1u);
+                if (pos0 + 16 > se) bits &= (1u << (se - pos0)) - 1u;
+            }
+            int last_pos = bits ? pos0 + 31 - __clz(bits) : -1;
+            int incl = last_pos;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl = max(incl, y);
+            }
+            int prev = __shfl_up_sync(0xffffffffu, incl, 1);
+            if (lane == 0) prev = -1;
+            prev = max(prev, carry);
+            carry = max(carry, __shfl_sync(0xffffffffu, incl, 31));
+            int thr = max(thr_local, *(volatile int*)thr_shared - 1);
+            thr = __shfl_sync(0xffffffffu, thr, 0);                // one value for the whole warp
+            // candidates in ascending position order: lowest lane first, ascending inside a lane
+            bool have = false;
+            int c_cnt = 0, c_start = 0;
+            if (thr >= 15) {
+                // only the run that ends at this lane's first boundary can be long enough
+                if (bits) {
+                    const int bpos = pos0 + __ffs(bits) - 1;
                     if (prev >= 0) {
                         const int c = bpos - prev;
-                        if (c > thr) { c_cnt = c; c_start = prev; prev = bpos; have = true; break; }
+                        if (c > thr) { c_cnt = c; c_start = prev; have = true; }
                     } else {
                         my_first = bpos;
                     }
-                    prev = bpos;
+                    bits = 0;
                 }
             }
-            const unsigned vote = __ballot_sync(0xffffffffu, have);
-            if (!vote) break;
-            const int src = __ffs(vote) - 1;
-            const int cc = __shfl_sync(0xffffffffu, c_cnt, src);
-            const int cs = __shfl_sync(0xffffffffu, c_start, src);
-            if (lane == src) have = false;
-            if (cc > thr) {
-                const int tok = corpus[(int64_t)sa[cs] + d];
-                if (tok >= 0) {
-                    topk_insert(tk, k, cc, cs, tok);
+            while (true) {
+                if (!have) {
+                    while (bits) {
+                        const int t = __ffs(bits) - 1;
+                        bits &= bits - 1;
+                        const int bpos = pos0 + t;
+                        if (prev >= 0) {
+                            const int c = bpos - prev;
+                            if (c > thr) { c_cnt = c; c_start = prev; prev = bpos; have = true; break; }
+                        } else {
+                            my_first = bpos;
+                        }
+                        prev = bpos;
+                    }
+                }
+                const unsigned vote = __ballot_sync(0xffffffffu, have);
+                if (!vote) break;
+                const int src = __ffs(vote) - 1;
+                const int cc = __shfl_sync(0xffffffffu, c_cnt, src);
+                const int cs = __shfl_sync(0xffffffffu, c_start, src);
+                if (lane == src) have = false;
+                if (cc > thr) {
+                    topk_insert(tk, k, cc, cs);
+                    if (tk.n == k) {
 #pragma unroll
-                    for (int i = 0; i < kMaxK; ++i) if (i == k - 1 && tk.n == k) thr = tk.cnt[i];
+                        for (int i = 0; i < kMaxK; ++i) if (i == k - 1) thr_local = tk.cnt[i];
+                        if (lane == 0) atomicMax(thr_shared, thr_local);
+                        thr = max(thr, thr_local);
+                    }
                 }
             }
         }
@@ -132,27 +169,76 @@ __device__ void warp_scan_span(const uint8_t* __restrict__ lcp, const int32_t* _
     last_b = carry;
 }
 
+// Number of suffixes of the interval [lo, hi) whose entry at depth d is a separator (the occurrence ends its
+// trajectory there).  They sort before every real token, so this is the first position holding a token >= 0,
+// found by a 32-way search of one warp; almost always the very first probe answers.
+__device__ int count_ending(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, int lo, int hi, int d, int lane) {
+    int first = corpus[(int64_t)sa[lo] + d];
+    if (first >= 0) return 0;
+    int a = lo + 1, z = hi;                                 // answer in [a, z]: positions < a hold separators
+    while (a < z) {
+        const int span = z - a;
+        const int step = (span + 31) / 32;
+        const int pos = min(a + lane * step, z - 1);
+        const bool sep = corpus[(int64_t)sa[pos] + d] < 0;
+        const unsigned m = __ballot_sync(0xffffffffu, !sep);
+        if (m == 0) { a = min(a + 31 * step, z - 1) + 1; continue; }
+        const int f = __ffs(m) - 1;                          // first probe holding a real token
+        z = min(a + f * step, z - 1);
+        a = f == 0 ? a : min(a + (f - 1) * step, z - 1) + 1;
+        if (f == 0) break;
+    }
+    return z - lo;
+}
+
 struct Shared {
     int pat[kMaxP];
     int pool_cnt[kPoolCap], pool_par[kPoolCap], pool_tok[kPoolCap], pool_lo[kPoolCap];
-    int slot_lo[kMaxN], slot_cnt[kMaxN], slot_depth[kMaxN];
+    int slot_depth[kMaxN];
     int w_first[kWarps], w_last[kWarps], w_n[kWarps];
-    int w_cnt[kWarps][kMaxK], w_start[kWarps][kMaxK], w_tok[kWarps][kMaxK];
+    int w_cnt[kWarps][kMaxK], w_start[kWarps][kMaxK];
+    int st_cnt[32], st_start[32];               // runs that cross span edges (one per span) and the closing run
     int fin_cnt[kMaxK], fin_start[kMaxK], fin_tok[kMaxK];
-    int mode, cur, lo, cnt, depth, n_nodes, pool_n;
+    int mode, cur, lo, cnt, depth, n_nodes, pool_n, thr_shared, long_runs_only;
 };
 
-__device__ __forceinline__ int compare_suffix(const int32_t* __restrict__ corpus, int64_t s, const int* pat, int len) {
-    // tokens 1 .. len-1 of the suffix at s against the pattern (token 0 is fixed by the bucket)
-    for (int t = 1; t < len; ++t) {
-        const int c = corpus[s + t];
-        const int p = pat[t];
-        if (c != p) return c < p ? -1 : 1;
+// Tokens from index `from` on of the suffix at s against the pattern; returns the sign and, in `matched`, how many
+// leading tokens agree.  Four corpus tokens are (then sixteen) corpus tokens are requested at a time so their latencies overlap (the corpus has
+// readable slack behind its last separator, and a separator always ends the walk).
+__device__ __forceinline__ int compare_suffix(const int32_t* __restrict__ corpus, int64_t s, const int* pat, int len, int from,
+                                              int& matched) {
+    int t = from;
+    {
+        int c[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c[i] = corpus[s + t + i];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (t + i < len) {
+                const int p = pat[t + i];
+                if (c[i] != p) { matched = t + i; return c[i] < p ? -1 : 1; }
+            }
+        }
+        t += 4;
     }
+    // most comparisons end above; the ones that go on share a long prefix, so fetch far ahead
+    for (; t < len; t += 16) {
+        int c[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) c[i] = (t + i < len) ? corpus[s + t + i] : 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            if (t + i < len) {
+                const int p = pat[t + i];
+                if (c[i] != p) { matched = t + i; return c[i] < p ? -1 : 1; }
+            }
+        }
+    }
+    matched = len;
     return 0;
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 2)
 war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, const uint8_t* __restrict__ lcp,
                  const int32_t* __restrict__ bucket, int vocab, const int32_t* __restrict__ tail,
                  const int32_t* __restrict__ tail_len, int P, int N, int K, int min_match,
@@ -168,54 +254,88 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
     if (tid < P) sh.pat[tid] = tail[(size_t)b * P + tid];
     __syncthreads();
 
+    // Publishes the next node to expand: its token range (the interval minus the suffixes that end at this depth).
+    auto publish = [&](int slot, int lo, int cnt, int depth) {          // warp 0, all lanes
+        if (cnt <= 32) {                                                // handled in registers, one suffix per lane
+            if (lane == 0) { sh.cur = slot; sh.lo = lo; sh.cnt = cnt; sh.depth = depth; sh.long_runs_only = 0; sh.mode = 3; }
+            return;
+        }
+        const int e = count_ending(corpus, sa, lo, lo + cnt, depth, lane);
+        if (lane == 0) {
+            sh.cur = slot; sh.lo = lo + e; sh.cnt = cnt - e; sh.depth = depth;
+            // Large nodes are first scanned for runs of 16 positions or more only (bar preset to 16): that pass never
+            // walks the boundaries inside a lane.  It is exact whenever it finds k such runs; otherwise the node is
+            // scanned again without the preset.
+            sh.long_runs_only = (cnt - e) >= kLongRunFirstMin;
+            sh.thr_shared = sh.long_runs_only ? 16 : 0;
+            sh.mode = (cnt - e) >= kBlockScanMin ? 2 : 1;
+        }
+    };
+
     if (warp == 0) {
         // ---- longest-suffix match ----
         const int tl = min(max(tail_len[b], 0), P);
         const int len = lane + 1;
-        int lo = 0, hi = 0;
+        int lo = 0, bucket_hi = 0;
+        bool occurs = false;
         if (len <= tl) {
             const int* pat = sh.pat + (P - len);
             bool valid = true;
             for (int t = 0; t < len; ++t) valid = valid && pat[t] >= 0 && pat[t] < vocab;
             if (valid) {
                 lo = bucket[pat[0]];
-                hi = bucket[pat[0] + 1];
-                if (len > 1 && hi > lo) {
-                    int a = lo, z = hi;                          // lower bound: first suffix >= pattern
-                    while (a < z) {
+                bucket_hi = bucket[pat[0] + 1];
+                occurs = bucket_hi > lo;
+                if (len > 1 && occurs) {
+                    // lower bound by binary search; it remembers how many tokens the pattern shares with the suffixes
+                    // at its current ends, so comparisons restart there (all bucket members share token 0)
+                    int a = lo, z = bucket_hi, ma = 1, mz = 1, m;
+                    while (a < z) {                              // first suffix >= pattern
                         const int mid = a + ((z - a) >> 1);
-                        if (compare_suffix(corpus, sa[mid], pat, len) < 0) a = mid + 1; else z = mid;
+                        if (compare_suffix(corpus, sa[mid], pat, len, min(ma, mz), m) < 0) { a = mid + 1; ma = m; } else { z = mid; mz = m; }
                     }
-                    const int first = a;
-                    z = hi;                                      // upper bound: first suffix > pattern
-                    while (a < z) {
-                        const int mid = a + ((z - a) >> 1);
-                        if (compare_suffix(corpus, sa[mid], pat, len) <= 0) a = mid + 1; else z = mid;
-                    }
-                    lo = first;
-                    hi = a;
+                    lo = a;
+                    // the pattern occurs iff the suffix there starts with it
+                    occurs = lo < bucket_hi && compare_suffix(corpus, sa[lo], pat, len, 1, m) == 0;
                 }
             }
         }
-        const unsigned found = __ballot_sync(0xffffffffu, hi > lo);
+        const unsigned found = __ballot_sync(0xffffffffu, occurs);
         const int ml = found ? 32 - __clz(found) : 0;
         const int src = ml > 0 ? ml - 1 : 0;
         lo = __shfl_sync(0xffffffffu, lo, src);
-        hi = __shfl_sync(0xffffffffu, hi, src);
+        bucket_hi = __shfl_sync(0xffffffffu, bucket_hi, src);
+        // Only the longest match needs its upper end: 32-way search by the whole warp over (lo, bucket end) for the
+        // first suffix that no longer starts with the pattern (one probe per lane and round).
+        int hi = bucket_hi;
+        if (ml > 1) {
+            const int* pat = sh.pat + (P - ml);
+            int a = lo + 1, z = bucket_hi, m;                    // positions < a match, positions >= z do not
+            while (a < z) {
+                const int step = (z - a + 31) / 32;
+                const int pos = min(a + lane * step, z - 1);
+                const bool hit = compare_suffix(corpus, sa[pos], pat, ml, 1, m) == 0;
+                const int nm = __popc(__ballot_sync(0xffffffffu, hit));          // hits are a prefix of the lanes
+                if (nm == 32) { a = min(a + 31 * step, z - 1) + 1; continue; }
+                const int z_old = z;
+                z = min(a + nm * step, z_old - 1);
+                if (nm > 0) a = min(a + (nm - 1) * step, z_old - 1) + 1;
+            }
+            hi = a;
+        }
+        const int c0 = ml > 0 ? hi - lo : 0;
+        const bool expand = ml >= max(1, min_match) && N > 1;
         if (lane == 0) {
-            const int c0 = ml > 0 ? hi - lo : 0;
             match_len[b] = ml;
             o_ids[0] = sh.pat[P - 1];
             o_par[0] = -1;
             if (o_cnt) o_cnt[0] = c0;
-            sh.slot_lo[0] = lo; sh.slot_cnt[0] = c0; sh.slot_depth[0] = ml;
+            sh.slot_depth[0] = ml;
             sh.n_nodes = 1;
             sh.pool_n = 0;
-            sh.cur = 0;
-            const bool expand = ml >= max(1, min_match) && N > 1;
-            sh.lo = lo; sh.cnt = c0; sh.depth = ml;
-            sh.mode = !expand ? 0 : (c0 >= kBlockScanMin ? 2 : 1);
+            sh.mode = 0;
         }
+        if (expand) publish(0, lo, c0, ml);
     }
 
     // ---- best-first expansion ----
@@ -231,63 +351,107 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             const int sb = max(lo, a0 + warp * span), se = min(hi, a0 + (warp + 1) * span);
             TopK tk;
             int fb = -1, lb = -1;
-            tk.n = 0;
-#pragma unroll
-            for (int i = 0; i < kMaxK; ++i) { tk.cnt[i] = 0; tk.start[i] = 0; tk.tok[i] = 0; }
-            if (sb < se) warp_scan_span(lcp, sa, corpus, d, sb, se, K, lane, tk, fb, lb);
+            topk_clear(tk);
+            if (sb < se) warp_scan_span(lcp, d, sb, se, K, lane, tk, fb, lb, &sh.thr_shared);
             if (lane == 0) {
                 sh.w_first[warp] = fb; sh.w_last[warp] = lb; sh.w_n[warp] = tk.n;
 #pragma unroll
-                for (int i = 0; i < kMaxK; ++i) { sh.w_cnt[warp][i] = tk.cnt[i]; sh.w_start[warp][i] = tk.start[i]; sh.w_tok[warp][i] = tk.tok[i]; }
+                for (int i = 0; i < kMaxK; ++i) { sh.w_cnt[warp][i] = tk.cnt[i]; sh.w_start[warp][i] = tk.start[i]; }
             }
             __syncthreads();
         }
         if (warp == 0) {
             const int cur = sh.cur;
             int n_fin = 0;
-            if (cnt == 1) {
-                // a unique occurrence continues with the next corpus token, if the trajectory goes on
-                if (lane == 0) {
-                    const int tok = corpus[(int64_t)sa[lo] + d];
-                    if (tok >= 0) { sh.fin_cnt[0] = 1; sh.fin_start[0] = lo; sh.fin_tok[0] = tok; n_fin = 1; }
+            if (mode == 3) {
+                // at most 32 suffixes: lane i reads the continuation token of suffix lo+i; suffixes that end here hold a
+                // separator (negative) and sort first; equal tokens are adjacent, so a run is a head lane plus followers
+                const int tok = lane < cnt ? corpus[(int64_t)sa[lo + lane] + d] : -1;
+                const int prev_tok = __shfl_up_sync(0xffffffffu, tok, 1);
+                const bool real = lane < cnt && tok >= 0;
+                const bool head = real && (lane == 0 || tok != prev_tok);
+                const unsigned hm = __ballot_sync(0xffffffffu, head);
+                const unsigned vm = __ballot_sync(0xffffffffu, real);
+                const int end = vm ? 32 - __clz(vm) : 0;
+                const unsigned after = (hm >> 1) >> lane;                  // heads strictly after this lane
+                int c = head ? (after ? lane + __ffs(after) : end) - lane : 0;
+                for (int r = 0; r < K; ++r) {
+                    const int key = __reduce_max_sync(0xffffffffu, c * 64 + (63 - lane));
+                    if (key < 64) break;                                  // no run left
+                    const int wl = 63 - (key & 63);
+                    const int wt = __shfl_sync(0xffffffffu, tok, wl);
+                    if (lane == 0) { sh.fin_cnt[n_fin] = key >> 6; sh.fin_start[n_fin] = lo + wl; sh.fin_tok[n_fin] = wt; }
+                    if (lane == wl) c = 0;
+                    ++n_fin;
                 }
-            } else {
+            } else if (cnt > 0) {
                 int nw = kWarps;
                 if (mode == 1) {
                     TopK tk;
                     int fb, lb;
-                    warp_scan_span(lcp, sa, corpus, d, lo, hi, K, lane, tk, fb, lb);
+                    warp_scan_span(lcp, d, lo, hi, K, lane, tk, fb, lb, &sh.thr_shared);
                     if (lane == 0) {
                         sh.w_first[0] = fb; sh.w_last[0] = lb; sh.w_n[0] = tk.n;
 #pragma unroll
-                        for (int i = 0; i < kMaxK; ++i) { sh.w_cnt[0][i] = tk.cnt[i]; sh.w_start[0][i] = tk.start[i]; sh.w_tok[0][i] = tk.tok[i]; }
+                        for (int i = 0; i < kMaxK; ++i) { sh.w_cnt[0][i] = tk.cnt[i]; sh.w_start[0][i] = tk.start[i]; }
                     }
                     nw = 1;
                 }
                 __syncwarp();
-                if (lane == 0) {
-                    // stitch the runs that cross span edges, then merge everything under (cnt desc, start asc)
-                    auto offer = [&](int c, int s, int tok) {
-                        int pos = n_fin;
-                        for (int i = n_fin - 1; i >= 0; --i)
-                            if (c > sh.fin_cnt[i] || (c == sh.fin_cnt[i] && s < sh.fin_start[i])) pos = i;
-                        if (pos >= K) return;
-                        if (tok == INT_MIN) { tok = corpus[(int64_t)sa[s] + d]; if (tok < 0) return; }
-                        const int last = min(n_fin, K - 1);
-                        for (int i = last; i > pos; --i) { sh.fin_cnt[i] = sh.fin_cnt[i - 1]; sh.fin_start[i] = sh.fin_start[i - 1]; sh.fin_tok[i] = sh.fin_tok[i - 1]; }
-                        sh.fin_cnt[pos] = c; sh.fin_start[pos] = s; sh.fin_tok[pos] = tok;
-                        if (n_fin < K) ++n_fin;
-                    };
-                    int carry = -1;
-                    for (int w = 0; w < nw; ++w) {
-                        if (sh.w_first[w] < 0) continue;
-                        if (carry >= 0) offer(sh.w_first[w] - carry, carry, INT_MIN);
-                        for (int e = 0; e < sh.w_n[w]; ++e) offer(sh.w_cnt[w][e], sh.w_start[w][e], sh.w_tok[w][e]);
-                        carry = sh.w_last[w];
+                // runs that cross span edges: span w's first boundary closes the run opened by the last boundary before it
+                const int wf = lane < nw ? sh.w_first[lane] : -1;
+                const int wl = lane < nw ? sh.w_last[lane] : -1;
+                int incl = wl;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl = max(incl, y);
+                }
+                int carry = __shfl_up_sync(0xffffffffu, incl, 1);
+                if (lane == 0) carry = -1;
+                const int last_all = __shfl_sync(0xffffffffu, incl, 31);
+                int st_c = 0, st_s = 0;
+                if (wf >= 0 && carry >= 0) { st_c = wf - carry; st_s = carry; }
+                if (lane == 31 && last_all >= 0) { st_c = hi - last_all; st_s = last_all; }      // the closing run
+                sh.st_cnt[lane] = st_c; sh.st_start[lane] = st_s;
+                __syncwarp();
+                // the K best of all candidates under (count desc, start asc), one warp arg-max per winner
+                int* wc = &sh.w_cnt[0][0];
+                int* ws = &sh.w_start[0][0];
+                for (int r = 0; r < K; ++r) {
+                    int bc = 0, bs = 0, bsrc = -1;
+                    for (int i = lane; i < nw * kMaxK; i += 32) {
+                        const int c = wc[i], st = ws[i];
+                        if (c > bc || (c == bc && c > 0 && st < bs)) { bc = c; bs = st; bsrc = i; }
                     }
-                    if (carry >= 0) offer(hi - carry, carry, INT_MIN);
+                    {
+                        const int c = sh.st_cnt[lane], st = sh.st_start[lane];
+                        if (c > bc || (c == bc && c > 0 && st < bs)) { bc = c; bs = st; bsrc = 0x1000 + lane; }
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const int oc = __shfl_xor_sync(0xffffffffu, bc, o), os = __shfl_xor_sync(0xffffffffu, bs, o);
+                        const int osrc = __shfl_xor_sync(0xffffffffu, bsrc, o);
+                        if (oc > bc || (oc == bc && oc > 0 && os < bs)) { bc = oc; bs = os; bsrc = osrc; }
+                    }
+                    if (bc <= 0) break;                                  // uniform: no candidate left
+                    if (lane == 0) {
+                        sh.fin_cnt[n_fin] = bc; sh.fin_start[n_fin] = bs;
+                        if (bsrc >= 0x1000) sh.st_cnt[bsrc - 0x1000] = 0; else wc[bsrc] = 0;
+                    }
+                    ++n_fin;
+                    __syncwarp();
                 }
             }
+            __syncwarp();
+            if (sh.long_runs_only && n_fin < K) {                        // uniform: fewer than k long runs, look at all runs
+                __syncwarp();
+                if (lane == 0) { sh.long_runs_only = 0; sh.thr_shared = 0; }
+                continue;
+            }
+            // tokens of the winners, one lane each (the register path above already has them)
+            if (mode != 3 && lane < n_fin) sh.fin_tok[lane] = corpus[(int64_t)sa[sh.fin_start[lane]] + d];
+            __syncwarp();
             if (lane == 0) {
                 int pn = sh.pool_n;
                 for (int e = 0; e < n_fin && pn < kPoolCap; ++e, ++pn) {
@@ -309,27 +473,26 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 const int op = __shfl_xor_sync(0xffffffffu, bp, o), ot = __shfl_xor_sync(0xffffffffu, bt, o);
                 if (oi >= 0 && (bi < 0 || oc > bc || (oc == bc && (op < bp || (op == bp && ot < bt))))) { bi = oi; bc = oc; bp = op; bt = ot; }
             }
-            if (lane == 0) {
-                if (bi < 0) {
-                    sh.mode = 0;
-                } else {
-                    const int j = sh.n_nodes;
-                    const int slo = sh.pool_lo[bi];
+            // every lane now holds the same winner
+            if (bi < 0) {
+                if (lane == 0) sh.mode = 0;
+            } else {
+                const int j = sh.n_nodes;
+                const int slo = sh.pool_lo[bi];
+                const int depth = sh.slot_depth[bp] + 1;
+                __syncwarp();
+                if (lane == 0) {
                     const int last = pn - 1;
                     sh.pool_cnt[bi] = sh.pool_cnt[last]; sh.pool_par[bi] = sh.pool_par[last];
                     sh.pool_tok[bi] = sh.pool_tok[last]; sh.pool_lo[bi] = sh.pool_lo[last];
                     sh.pool_n = last;
                     o_ids[j] = bt; o_par[j] = bp;
                     if (o_cnt) o_cnt[j] = bc;
-                    sh.slot_lo[j] = slo; sh.slot_cnt[j] = bc; sh.slot_depth[j] = sh.slot_depth[bp] + 1;
+                    sh.slot_depth[j] = depth;
                     sh.n_nodes = j + 1;
-                    if (j + 1 >= N) {
-                        sh.mode = 0;
-                    } else {
-                        sh.cur = j; sh.lo = slo; sh.cnt = bc; sh.depth = sh.slot_depth[j];
-                        sh.mode = bc >= kBlockScanMin ? 2 : 1;
-                    }
+                    sh.mode = 0;
                 }
+                if (j + 1 < N) publish(j, slo, bc, depth);
             }
         }
     }

@@ -29,13 +29,15 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         const int pl = prefix_len[i];
         bool bad = n < 0 || n > N || pl < 0;
         if (!bad && n > 0) {
-            uint64_t* anc = w.anc + (size_t)i * N;
-            for (int j = 0; j < n; ++j) {
+            uint64_t local[64];
+            local[0] = 1ull;
+            for (int j = 1; j < n; ++j) {
                 const int p = parent[(size_t)i * N + j];
-                if (j == 0) { anc[0] = 1ull; continue; }
                 if (p < 0 || p >= j) { bad = true; break; }
-                anc[j] = anc[p] | (1ull << j);
+                local[j] = local[p] | (1ull << j);
             }
+            if (!bad)
+                for (int j = 0; j < n; ++j) w.anc[(size_t)i * N + j] = local[j];
         }
         if (bad) { war_set_device_status(status_word, WAR_ERR_BAD_TREE); n = 0; }
         int tiles = 0;
@@ -126,35 +128,46 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
 // ------------------------------------------------------------------------------------------------
 // combine: merges the partials of split requests in chunk order (deterministic)
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128)
+constexpr int kCombineWarps = 4;
+
+// One warp per output row: lanes first reduce the chunk maxima, then stream the chunks' partial rows (float4 per
+// lane, all loads independent) and accumulate in chunk order.
+__global__ void __launch_bounds__(kCombineWarps * 32)
 attn_combine_kernel(AttnWorkspace w, int N, int Hq, int Hkv, int G, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     const int i = blockIdx.x / Hkv, kvh = blockIdx.x % Hkv;
     const AttnReq rq = w.req[i];
     if (rq.n_chunks <= 1 || rq.n_nodes <= 0) return;
     const int R = G * rq.n_nodes;
     const int rbs = (R + kRowBlock - 1) / kRowBlock;
-    const int d = threadIdx.x;                      // D == 128
-    for (int r = 0; r < R; ++r) {
-        const int rb = r / kRowBlock, rr = r % kRowBlock;
-        float M = -CUDART_INF_F;
-        for (int c = 0; c < rq.n_chunks; ++c) {
-            const int u = rq.base_unit + (c * Hkv + kvh) * rbs + rb;
-            M = fmaxf(M, w.part_ml[((size_t)u * w.rows + rr) * 2]);
-        }
-        float l = 0.f, o = 0.f;
-        for (int c = 0; c < rq.n_chunks; ++c) {
-            const int u = rq.base_unit + (c * Hkv + kvh) * rbs + rb;
-            const float m = w.part_ml[((size_t)u * w.rows + rr) * 2];
-            if (m == -CUDART_INF_F) continue;
-            const float sc = exp2f(m - M);
-            l += w.part_ml[((size_t)u * w.rows + rr) * 2 + 1] * sc;
-            o += w.part_o[((size_t)u * w.rows + rr) * 128 + d] * sc;
-        }
-        const int j = r / G, g = r % G;
-        const size_t row = ((size_t)i * N + j) * Hq + kvh * G + g;
-        out[row * 128 + d] = __float2bfloat16(o / l);
-        if (lse && d == 0) lse[row] = (M + log2f(l)) * kLn2;
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.y * kCombineWarps + (threadIdx.x >> 5);
+    if (r >= R) return;
+    const int rb = r / kRowBlock, rr = r % kRowBlock;
+    const int u0 = rq.base_unit + kvh * rbs + rb, ustep = Hkv * rbs;       // unit of chunk c = u0 + c * ustep
+    float M = -CUDART_INF_F;
+    for (int c = lane; c < rq.n_chunks; c += 32)
+        M = fmaxf(M, w.part_ml[((size_t)(u0 + c * ustep) * w.rows + rr) * 2]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = 0; c < rq.n_chunks; ++c) {
+        const size_t base = (size_t)(u0 + c * ustep) * w.rows + rr;
+        const float2 ml = *reinterpret_cast<const float2*>(w.part_ml + base * 2);
+        const float4 o = *reinterpret_cast<const float4*>(w.part_o + base * 128 + lane * 4);
+        const float sc = ml.x == -CUDART_INF_F ? 0.f : exp2f(ml.x - M);
+        l = fmaf(ml.y, sc, l);
+        acc.x = fmaf(o.x, sc, acc.x); acc.y = fmaf(o.y, sc, acc.y); acc.z = fmaf(o.z, sc, acc.z); acc.w = fmaf(o.w, sc, acc.w);
     }
+    const float inv = 1.f / l;
+    const int j = r / G, g = r % G;
+    const size_t row = ((size_t)i * N + j) * Hq + kvh * G + g;
+    const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), h1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    uint2 packed;
+    packed.x = *reinterpret_cast<const uint32_t*>(&h0);
+    packed.y = *reinterpret_cast<const uint32_t*>(&h1);
+    *reinterpret_cast<uint2*>(out + row * 128 + lane * 4) = packed;
+    if (lse && lane == 0) lse[row] = (M + log2f(l)) * kLn2;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -344,7 +357,8 @@ extern "C" war_status_t war_verify_attn(const void* d_q, const void* d_kpool, co
     else
         st = war_attn_launch_sm100(d_q, d_kpool, d_vpool, d_page_table, d_prefix_len, p, w, d_out, d_lse, status_word, stream);
     if (st != WAR_OK) return st;
-    attn_combine_kernel<<<p->B * p->Hkv, 128, 0, stream>>>(w, p->N, p->Hq, p->Hkv, G, (__nv_bfloat16*)d_out, d_lse);
+    attn_combine_kernel<<<dim3(p->B * p->Hkv, (G * p->N + kCombineWarps - 1) / kCombineWarps), kCombineWarps * 32, 0, stream>>>(
+        w, p->N, p->Hq, p->Hkv, G, (__nv_bfloat16*)d_out, d_lse);
     WAR_LAUNCH_CHECK();
     return WAR_OK;
 }
