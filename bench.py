@@ -132,6 +132,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kernel", type=int, default=0, help="0 = tensor-core verify attention, 1 = plain CUDA-core kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--requests", type=int, default=0,
+                    help="run the workload's recipe with this many requests instead of its own count (profiling-size cases)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -142,6 +144,8 @@ def main():
     import torch
     from paper_2607_17299_b200 import workloads as W
     cfg = W.CONFIGS[args.workload]
+    if args.requests > 0:
+        cfg = W.scaled(cfg, B=args.requests)
     base_config = {"workload": f"{cfg.name}: corpus {cfg.n_traj} trajectories, {cfg.B} requests, tree <= {cfg.N} slots, "
                                f"{cfg.Hq}q/{cfg.Hkv}kv heads, d={cfg.D}, page {cfg.page_size}",
                    "requests_per_gpu": cfg.B, "parallelism": f"replica x{world}" if world > 1 else "single gpu",
@@ -309,11 +313,14 @@ def main():
             peak, peak_src = 6650.0, "fallback"
         kvb = kv_bytes(cfg, ctx - 1, h_nn)
         achieved = kvb / (attn_ms * 1e-3) / 1e9
-        traffic_path = os.path.join(ROOT, "profiles", f"traffic_{cfg.name}.json")
+        # DRAM bytes per launch of the attention kernel from the committed ncu summary of this workload, if there is one
         traffic = None
-        if os.path.exists(traffic_path):
+        traffic_path = os.path.join(ROOT, "profiles", f"attn_sm100_kernel_{cfg.name}_traffic.md")
+        if os.path.exists(traffic_path) and args.requests == 0:
+            import re
             with open(traffic_path) as f:
-                traffic = json.load(f).get("dram_bytes_per_launch")
+                m = re.search(r"^dram_bytes_per_launch\s*=\s*(\d+)", f.read(), flags=re.M)
+            traffic = int(m.group(1)) if m else None
         line = {
             "metric": METRIC, "value": verified_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
