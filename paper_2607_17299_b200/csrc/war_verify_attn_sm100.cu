@@ -7,13 +7,14 @@
 //                             O += P V    (M=128 rows, N=128 dims, K=128 keys; P is read from TMEM)
 // Tiles alternate between two softmax groups, each with its own S/P region, running (max, sum) and O accumulator
 // in TMEM; the two partial results are merged once per unit.  Nothing synchronises the groups per tile.
-// Warp roles:  warp 0   producer: reads the page table, issues one TMA tensor copy per (page, head) into a ring of
+// Warp roles:  warp 8   producer: reads the page table, issues one TMA tensor copy per (page, head) into a ring of
 //                       32 KB slots in the order the tensor pipe consumes them (K0 K1 V0 K2 V1 ...); no multicast,
 //                       this GPU's memory only
-//              warp 1   MMA issuer (one lane): S(t+2) is queued right behind PV(t); owns the TMEM allocation
-//              warps 2-5 / 6-9  softmax group 0 / 1: one thread per query row (TMEM lane); the row of S is pulled
-//                       into registers, P goes back into the first 64 columns of the same TMEM region as packed
-//                       bf16; O is rescaled in TMEM only when the running max grows by more than 2^8
+//              warp 9   MMA issuer (one lane): S(t+2) is queued right behind PV(t); owns the TMEM allocation
+//              warps 0-3 / 4-7  softmax group 0 / 1: one thread per query row (TMEM lane); the whole row of S is
+//                       pulled into registers once, P goes back into the first 64 columns of the same TMEM region
+//                       as packed bf16; O is rescaled in TMEM only when the running max grows by more than 2^8
+//              The softmax warpgroups take registers from the third one (setmaxnreg) so a row of S fits.
 // Shared-memory operand layouts are the canonical 128-byte-swizzled ones: K-major for Q and K, MN-major for V.
 // A (page, head) block lands as [token/8][d/64][token%8][d%64], which serves both K (K-major, 8-row groups 2 KB
 // apart) and V (MN-major, 64-wide column blocks 1 KB apart, 8-key groups 2 KB apart) with one copy per block.
@@ -30,7 +31,9 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kSlots = 6;
 constexpr int kSlotBytes = 32768;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;                      // three warpgroups: softmax 0, softmax 1, {producer, MMA, 2 spare warps}
+constexpr int kRegsSoftmax = 224;                   // register budget after the hand-over below
+constexpr int kRegsOther = 48;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;           // log2 units
 constexpr unsigned long long kWaitBudgetNs = 2000000000ull;
@@ -213,7 +216,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == 9) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -223,7 +226,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     const uint32_t tmem = bars->tmem_base;
     // columns: [0,128) S/P of group 0, [128,256) S/P of group 1, [256,384) O of group 0, [384,512) O of group 1
 
-    if (warp == 0) {
+    // register hand-over between warpgroups: the third warpgroup gives registers up, the softmax warpgroups take them
+    // (each instruction is executed by all four warps of its warpgroup, and the role code stays inside that branch)
+    if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+    if (warp == 8) {
         // ------------------------------------------------------------------ producer
         uint32_t ld = 0;
         bool ok = true;
@@ -267,7 +274,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                 pg_cur = pg_nxt; pg_nxt = pg_nn;
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 9) {
         // ------------------------------------------------------------------ MMA issuer
         uint32_t ld0 = 0, cg[2] = {0, 0}, units_done = 0;
         constexpr uint32_t idesc_s = umma_idesc(128, 128, 0);
@@ -323,9 +330,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
             ld0 += 2u * T;
             ++units_done;
         }
+    }
     } else {
         // ------------------------------------------------------------------ softmax groups, one thread per row
-        const int grp = (warp - 2) >> 2;
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+        const int grp = warp >> 2;
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
@@ -373,23 +382,21 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                 if (!ok) break;
                 tc_fence_after();
                 if (warp_valid) {
-                    // pass 1: row maximum (four independent chains); the whole row is in flight at once
+                    // the whole row of S comes into registers once
+                    uint32_t r[128];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, r + c * 32);
+                    tmem_wait_ld();
+                    if (need_mask) {
+#pragma unroll
+                        for (int e = 0; e < 128; ++e)
+                            if (!key_visible(key0 + e, pl, L, anc)) r[e] = 0xff800000u;     // -inf
+                    }
                     float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-                    {
-                        uint32_t r[128];
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, r + c * 32);
-                        tmem_wait_ld();
-                        if (need_mask) {
+                    for (int e = 0; e < 128; e += 4) {
 #pragma unroll
-                            for (int e = 0; e < 128; ++e)
-                                if (!key_visible(key0 + e, pl, L, anc)) r[e] = 0xff800000u;     // -inf
-                        }
-#pragma unroll
-                        for (int e = 0; e < 128; e += 4) {
-#pragma unroll
-                            for (int v = 0; v < 4; ++v) mx4[v] = fmaxf(mx4[v], __uint_as_float(r[e + v]));
-                        }
+                        for (int v = 0; v < 4; ++v) mx4[v] = fmaxf(mx4[v], __uint_as_float(r[e + v]));
                     }
                     const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;    // scale > 0
                     float corr = 1.f;
@@ -401,31 +408,18 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                         rescale = t > grp;                         // O of this group holds earlier tiles of the unit
                     }
                     const float neg_m = m_used == -CUDART_INF_F ? 0.f : -m_used;
-                    // pass 2: P = exp2(s*scale - m) in 32-column pieces, the next piece loading while this one is processed
+                    // P = exp2(s*scale - m), packed to bf16 pairs in place (pair i lands in r[i], already consumed)
                     float l4[4] = {0.f, 0.f, 0.f, 0.f};
-                    uint32_t pk[64];
-                    uint32_t buf[2][32];
-                    tmem_ld32(tS, buf[0]);
+                    uint32_t* pk = r;
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        tmem_wait_ld();
-                        if (c < 3) tmem_ld32(tS + (c + 1) * 32, buf[(c + 1) & 1]);
-                        uint32_t* r = buf[c & 1];
-                        if (need_mask) {
+                    for (int e = 0; e < 128; e += 8) {
 #pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                if (!key_visible(key0 + c * 32 + e, pl, L, anc)) r[e] = 0xff800000u;
-                        }
-#pragma unroll
-                        for (int e = 0; e < 32; e += 8) {
-#pragma unroll
-                            for (int v = 0; v < 4; ++v) {
-                                const float p0 = fast_exp2(fmaf(__uint_as_float(r[e + 2 * v]), a.scale_log2, neg_m));       // exp2(-inf) = 0
-                                const float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 2 * v + 1]), a.scale_log2, neg_m));
-                                l4[v] += p0 + p1;
-                                const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                                pk[c * 16 + (e >> 1) + v] = *reinterpret_cast<const uint32_t*>(&h);
-                            }
+                        for (int v = 0; v < 4; ++v) {
+                            const float p0 = fast_exp2(fmaf(__uint_as_float(r[e + 2 * v]), a.scale_log2, neg_m));       // exp2(-inf) = 0
+                            const float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 2 * v + 1]), a.scale_log2, neg_m));
+                            l4[v] += p0 + p1;
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                            pk[(e >> 1) + v] = *reinterpret_cast<const uint32_t*>(&h);
                         }
                     }
                     l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
@@ -546,7 +540,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     // ---------------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == 9) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
