@@ -157,6 +157,11 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -394,9 +399,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                     }
                     float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-                    for (int e = 0; e < 128; e += 4) {
+                    for (int e = 0; e < 128; e += 8) {                      // three-input max: two columns per instruction
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) mx4[v] = fmaxf(mx4[v], __uint_as_float(r[e + v]));
+                        for (int v = 0; v < 4; ++v) mx4[v] = max3(mx4[v], __uint_as_float(r[e + 2 * v]), __uint_as_float(r[e + 2 * v + 1]));
                     }
                     const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;    // scale > 0
                     float corr = 1.f;
@@ -409,20 +414,22 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                     }
                     const float neg_m = m_used == -CUDART_INF_F ? 0.f : -m_used;
                     // P = exp2(s*scale - m), packed to bf16 pairs in place (pair i lands in r[i], already consumed)
-                    float l4[4] = {0.f, 0.f, 0.f, 0.f};
+                    float2 l4[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+                    const float2 sc2 = make_float2(a.scale_log2, a.scale_log2), nm2 = make_float2(neg_m, neg_m);
                     uint32_t* pk = r;
 #pragma unroll
                     for (int e = 0; e < 128; e += 8) {
 #pragma unroll
                         for (int v = 0; v < 4; ++v) {
-                            const float p0 = fast_exp2(fmaf(__uint_as_float(r[e + 2 * v]), a.scale_log2, neg_m));       // exp2(-inf) = 0
-                            const float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 2 * v + 1]), a.scale_log2, neg_m));
-                            l4[v] += p0 + p1;
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                            // two columns per FMA / add instruction (packed fp32 pairs)
+                            const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[e + 2 * v]), __uint_as_float(r[e + 2 * v + 1])), sc2, nm2);
+                            const float2 pp = make_float2(fast_exp2(x.x), fast_exp2(x.y));          // exp2(-inf) = 0
+                            l4[v] = __fadd2_rn(l4[v], pp);
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(pp.x, pp.y);
                             pk[(e >> 1) + v] = *reinterpret_cast<const uint32_t*>(&h);
                         }
                     }
-                    l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
+                    l += ((l4[0].x + l4[0].y) + (l4[1].x + l4[1].y)) + ((l4[2].x + l4[2].y) + (l4[3].x + l4[3].y));
                     if (__any_sync(0xffffffffu, rescale)) {
                         // O of this group is stable once its previous P V product has completed
                         ok = mbar_wait(&bars->pv_done[grp], (cgm - 1) & 1u, bars, a.status_word);

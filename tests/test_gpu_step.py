@@ -63,7 +63,7 @@ def test_tiny_step_every_request(war):
     _step(war, cfg, sample=list(range(cfg.B)))
 
 
-@pytest.mark.parametrize("name,sample", [("high", [0, 17, 101, 255]), ("low", [3, 30])])
+@pytest.mark.parametrize("name,sample", [("high", [0, 17, 101, 255]), ("low", [3, 30]), ("longtail", [5, 41]), ("wide", [7])])
 def test_full_size_sampled(war, name, sample):
     cfg = W.CONFIGS[name]
     ctx = W.context_lengths(cfg)
