@@ -102,14 +102,15 @@ __device__ __forceinline__ void tma_load_block(uint32_t dst, const CUtensorMap* 
         ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(block) : "memory");
 }
 
-// shared-memory matrix descriptor, 128-byte swizzle, sm_100 version field
-__device__ __forceinline__ uint64_t umma_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-    d |= (uint64_t)1 << 46;          // descriptor version
-    d |= (uint64_t)2 << 61;          // SWIZZLE_128B
+// shared-memory matrix descriptors: 128-byte swizzle, sm_100 version field.
+// The upper word of a descriptor (stride between 8-row groups, version, swizzle) is fixed per operand kind and the
+// lower word is an address plus a constant, so the issuing thread only adds small constants between MMAs: it is a
+// single thread, and every extra instruction between two tcgen05.mma stretches the issue interval.
+__device__ __forceinline__ constexpr uint32_t umma_desc_hi(uint32_t sbo_bytes) { return (sbo_bytes >> 4) | (1u << 14) | (2u << 29); }
+__device__ __forceinline__ constexpr uint32_t umma_desc_lo(uint32_t addr, uint32_t lbo_bytes) { return ((addr >> 4) & 0x3FFFu) | ((lbo_bytes >> 4) << 16); }
+__device__ __forceinline__ uint64_t pack64(uint32_t lo, uint32_t hi) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
     return d;
 }
 // instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major, M x N
@@ -284,6 +285,10 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         uint32_t ld0 = 0, cg[2] = {0, 0}, units_done = 0;
         constexpr uint32_t idesc_s = umma_idesc(128, 128, 0);
         constexpr uint32_t idesc_o = umma_idesc(128, 128, 1);
+        constexpr uint32_t hi_q = umma_desc_hi(1024), hi_kv = umma_desc_hi(2048);
+        const uint32_t q_lo = umma_desc_lo(sQ, 16);                  // Q: K-major, 8-row groups 1 KB apart
+        const uint32_t ring_lo = umma_desc_lo(sRing, 16);             // K: K-major, 8-row groups 2 KB apart
+        const uint32_t ring_lo_v = umma_desc_lo(sRing, 1024);         // V: MN-major, 64-wide column blocks 1 KB apart
         bool ok = true;
         for (int k = 0; ok; ++k) {
             const int u = snake_unit(k, blockIdx.x, gridDim.x);
@@ -295,12 +300,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                 if (!mbar_wait(&bars->full[slot], (sq / kSlots) & 1u, bars, a.status_word)) return false;
                 tc_fence_after();
                 if (lane == 0) {
-                    const uint32_t kb = sRing + slot * kSlotBytes;
+                    const uint32_t k_lo = ring_lo + slot * (kSlotBytes >> 4), d_s = tmem + g * 128u;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t qoff = (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32u;
-                        const uint32_t koff = (uint32_t)(ks >> 2) * 1024u + (uint32_t)(ks & 3) * 32u;
-                        umma_bf16(tmem + g * 128u, umma_desc(sQ + qoff, 16, 1024), umma_desc(kb + koff, 16, 2048), idesc_s, ks > 0);
+                        constexpr uint32_t kHalfQ = 16384u >> 4, kHalfK = 1024u >> 4;
+                        const uint32_t qo = (uint32_t)(ks >> 2) * kHalfQ + (uint32_t)(ks & 3) * 2u;
+                        const uint32_t ko = (uint32_t)(ks >> 2) * kHalfK + (uint32_t)(ks & 3) * 2u;
+                        umma_bf16(d_s, pack64(q_lo + qo, hi_q), pack64(k_lo + ko, hi_kv), idesc_s, ks > 0);
                     }
                     umma_commit(&bars->s_ready[g]);
                     umma_commit(&bars->empty[slot]);
@@ -319,11 +325,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
-                    const uint32_t vb = sRing + slot * kSlotBytes;
+                    const uint32_t v_lo = ring_lo_v + slot * (kSlotBytes >> 4), d_o = tmem + 256u + g * 128u, a_p = tmem + g * 128u;
+                    const uint32_t acc0 = t > 1 ? 1u : 0u;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
-                        umma_bf16_ts(tmem + 256u + g * 128u, tmem + g * 128u + (uint32_t)ks * 8u,
-                                     umma_desc(vb + (uint32_t)ks * 4096u, 1024, 2048), idesc_o, (t > 1 || ks > 0) ? 1u : 0u);
+                        umma_bf16_ts(d_o, a_p + (uint32_t)ks * 8u, pack64(v_lo + (uint32_t)ks * (4096u >> 4), hi_kv), idesc_o, ks > 0 ? 1u : acc0);
                     umma_commit(&bars->pv_done[g]);
                     umma_commit(&bars->empty[slot]);
                 }
