@@ -313,6 +313,18 @@ def main():
             peak, peak_src = 6650.0, "fallback"
         kvb = kv_bytes(cfg, ctx - 1, h_nn)
         achieved = kvb / (attn_ms * 1e-3) / 1e9
+        # the same launch seen from the tensor pipe: 4 * rows * D flops per KV token and kv head (QK^T and PV), rows = the
+        # (slot, head-of-group) pairs that exist (not the padded MMA tile)
+        G = cfg.Hq // cfg.Hkv
+        live = h_nn > 0
+        flops = float(((ctx - 1 + h_nn)[live].astype(np.float64) * (4.0 * G * h_nn[live] * cfg.D)).sum() * cfg.Hkv)
+        peak_tf = None
+        if os.path.exists(peaks_path):
+            with open(peaks_path) as f:
+                peak_tf = float(json.load(f).get("bf16_tflops_sustained", 0.0)) or None
+        peak_tf = peak_tf or 1400.0
+        t_hbm, t_tensor = kvb / (peak * 1e9), flops / (peak_tf * 1e12)
+        tensor_bound = t_tensor > t_hbm
         # DRAM bytes per launch of the attention kernel from the committed ncu summary of this workload, if there is one
         traffic = None
         traffic_path = os.path.join(ROOT, "profiles", f"attn_sm100_kernel_{cfg.name}_traffic.md")
@@ -330,10 +342,15 @@ def main():
             "e2e": {"value": verified_all / (e2e_ms / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
             "gpu_launches": LAUNCHES_PER_STEP * args.steps,
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": traffic, "kernel": "war_verify_attn (plan + attention + combine launches)",
-                         "bytes_per_launch": kvb, "ms_per_launch": attn_ms, "peak_source": peak_src,
-                         "frac_of_8TBps_nominal": achieved / 8000.0},
+            "roofline": ({"bound": "tensor", "achieved": flops / (attn_ms * 1e-3) / 1e12, "peak": peak_tf, "unit": "TFLOP/s",
+                          "frac": t_tensor / (attn_ms * 1e-3), "traffic": traffic, "flops_per_launch": flops,
+                          "peak_source": "measured (MEASURED_PEAKS.json bf16_tflops_sustained)" if os.path.exists(peaks_path) else "fallback",
+                          "hbm_gbs": achieved} if tensor_bound else
+                         {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                          "traffic": traffic, "frac_of_8TBps_nominal": achieved / 8000.0, "peak_source": peak_src,
+                          "tensor_tflops": flops / (attn_ms * 1e-3) / 1e12}),
+            "roofline_kernel": {"name": "war_verify_attn (plan + attention + combine launches)", "bytes_per_launch": kvb,
+                                "ms_per_launch": attn_ms},
             "breakdown_ms": {"draft": draft_ms, "verify_attn": attn_ms, "accept": accept_ms},
             "slots_verified_per_s": slots_all / (ms_per_step * 1e-3),
             "accept_len_mean": float(h_alen.mean()), "index_build_s": index_build_s, "index_tokens": int(len(tok)),

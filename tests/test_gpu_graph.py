@@ -1,0 +1,74 @@
+"""The three calls of a step enqueue work and return without touching the host, so a whole step can be captured
+in a CUDA graph and replayed (the paper's engine keeps separate CUDA graphs for speculative and plain decoding,
+Section 3.2).  Replays must reproduce the eager results bit for bit, also after the inputs change in place."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_17299_b200 import workloads as W
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def war():
+    from paper_2607_17299_b200 import binding
+    return binding
+
+
+def test_step_replays_from_a_cuda_graph(war):
+    dev = torch.device("cuda:0")
+    cfg = W.scaled(W.CONFIGS["tiny"], B=6, N=16)
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(cfg)
+    ctx = np.array([4096, 777, 1300, 2049, 40, 3000])
+    ix = U.build_index(war, tok, off, cfg.vocab, max_depth=cfg.P + cfg.N)
+    a = W.make_attention_inputs(cfg, ctx, device=dev)
+    B, N = cfg.B, cfg.N
+    i32 = dict(dtype=torch.int32, device=dev)
+    d_tails, d_tl = torch.from_numpy(tails).to(dev), torch.from_numpy(tl).to(dev)
+    ml, nn = torch.zeros(B, **i32), torch.zeros(B, **i32)
+    ids, par, cnt = torch.zeros((B, N), **i32), torch.zeros((B, N), **i32), torch.zeros((B, N), **i32)
+    alen, path, bonus = torch.zeros(B, **i32), torch.zeros((B, N), **i32), torch.zeros(B, **i32)
+    target = torch.randint(0, cfg.vocab, (B, N), dtype=torch.int32, device=dev)
+    out = torch.zeros_like(a.q)
+    lse = torch.zeros(a.q.shape[:3], dtype=torch.float32, device=dev)
+    params = war.attn_params(a.q, a.k_pool, a.v_pool, a.page_table, 1.0 / np.sqrt(cfg.D), 0)
+    ws = war.new_workspace(params, dev)
+
+    def step():
+        war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, ml, nn, ids, par, cnt)
+        war.war_verify_attn(a.q, a.k_pool, a.v_pool, a.page_table, a.prefix_len, nn, par, params, ws, out, lse)
+        war.war_accept(ids, par, nn, target, 0, alen, path, bonus)
+
+    def snapshot():
+        torch.cuda.synchronize()
+        return [t.clone() for t in (ml, nn, ids, par, cnt, out, lse, alen, path, bonus)]
+
+    step()                                                    # eager: also does the one-time per-device set-up
+    eager = snapshot()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    for t in (ml, nn, ids, par, cnt, out, lse, alen, path, bonus):
+        t.zero_()
+    g.replay()
+    for x, y in zip(snapshot(), eager):
+        assert torch.equal(x, y)
+    # new inputs in the same buffers: the replay recomputes everything on the device
+    d_tails.copy_(torch.roll(d_tails, 1, dims=0)); d_tl.copy_(torch.roll(d_tl, 1, dims=0))
+    a.q.copy_(torch.roll(a.q, 1, dims=0))
+    g.replay()
+    replayed = snapshot()
+    step()
+    for x, y in zip(replayed, snapshot()):
+        assert torch.equal(x, y)
+    assert not torch.equal(replayed[2], eager[2])
+    assert war.war_device_status() == 0
+    ix.destroy()
