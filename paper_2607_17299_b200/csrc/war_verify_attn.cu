@@ -29,10 +29,21 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         const int pl = prefix_len[i];
         bool bad = n < 0 || n > N || pl < 0;
         if (!bad && n > 0) {
+            // all parent ids of the request are requested before any is used, so their latencies overlap
+            int pbuf[64];
+            const int4* prow = reinterpret_cast<const int4*>(parent + (size_t)i * N);
+            if ((N & 3) == 0 && (reinterpret_cast<uintptr_t>(parent) & 15) == 0) {
+                for (int j = 0; j < n; j += 4) {
+                    const int4 v = prow[j >> 2];
+                    pbuf[j] = v.x; pbuf[j + 1] = v.y; pbuf[j + 2] = v.z; pbuf[j + 3] = v.w;
+                }
+            } else {
+                for (int j = 0; j < n; ++j) pbuf[j] = parent[(size_t)i * N + j];
+            }
             uint64_t local[64];
             local[0] = 1ull;
             for (int j = 1; j < n; ++j) {
-                const int p = parent[(size_t)i * N + j];
+                const int p = pbuf[j];
                 if (p < 0 || p >= j) { bad = true; break; }
                 local[j] = local[p] | (1ull << j);
             }
