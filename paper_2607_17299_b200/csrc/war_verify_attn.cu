@@ -17,14 +17,21 @@ __global__ void __launch_bounds__(1024)
 attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ num_nodes,
                  const int32_t* __restrict__ parent, int B, int N, int Hkv, int G, int page_size, int max_pages,
                  AttnWorkspace w, int* status_word) {
+    constexpr int kPer = kMaxPlanB / 1024;    // requests per thread, kept in registers through all phases
     __shared__ int s_tiles[kMaxPlanB];
-    __shared__ int s_units[kMaxPlanB];      // units per request, indexed by sorted position; then exclusive scan
+    __shared__ int s_units[kMaxPlanB];        // units per request, indexed by sorted position; then exclusive scan
     __shared__ int s_red[32];
+    __shared__ long long s_sum[32];
     __shared__ int s_chunk_tiles;
     const int tid = threadIdx.x;
+    int r_n[kPer], r_tiles[kPer], r_rbs[kPer], r_pos[kPer], r_nc[kPer];
     // per request: validate, ancestor masks, tile count
     long long my_tiles = 0;
-    for (int i = tid; i < B; i += blockDim.x) {
+#pragma unroll
+    for (int k = 0; k < kPer; ++k) {
+        const int i = tid + k * 1024;
+        r_n[k] = 0; r_tiles[k] = 0; r_rbs[k] = 0; r_pos[k] = 0; r_nc[k] = 0;
+        if (i >= B) continue;
         int n = num_nodes[i];
         const int pl = prefix_len[i];
         bool bad = n < 0 || n > N || pl < 0;
@@ -58,14 +65,12 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
             else tiles = (int)((L + kTileKeys - 1) / kTileKeys);
         }
         s_tiles[i] = tiles;
-        w.req[i].n_nodes = n;
-        w.req[i].n_tiles = tiles;
-        const int rbs = n > 0 ? (G * n + kRowBlock - 1) / kRowBlock : 0;
-        my_tiles += (long long)tiles * rbs;
+        r_n[k] = n; r_tiles[k] = tiles;
+        r_rbs[k] = n > 0 ? (G * n + kRowBlock - 1) / kRowBlock : 0;
+        my_tiles += (long long)tiles * r_rbs[k];
     }
     // block sum of tiles (weighted by row blocks and kv heads)
     for (int o = 16; o > 0; o >>= 1) my_tiles += __shfl_xor_sync(0xffffffffu, my_tiles, o);
-    __shared__ long long s_sum[32];
     if ((tid & 31) == 0) s_sum[tid >> 5] = my_tiles;
     __syncthreads();
     if (tid == 0) {
@@ -81,27 +86,27 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     __syncthreads();
     const int chunk_tiles = s_chunk_tiles;
     // longest-first order: position = number of requests that rank before this one
-    for (int i = tid; i < B; i += blockDim.x) {
-        const int t = s_tiles[i];
+#pragma unroll
+    for (int k = 0; k < kPer; ++k) {
+        const int i = tid + k * 1024;
+        if (i >= B) continue;
+        const int t = r_tiles[k];
         int pos = 0;
-        for (int k = 0; k < B; ++k) {
-            const int tk = s_tiles[k];
-            pos += (tk > t) || (tk == t && k < i);
+        for (int q = 0; q < B; ++q) {
+            const int tq = s_tiles[q];
+            pos += (tq > t) || (tq == t && q < i);
         }
-        const int n = w.req[i].n_nodes;
-        const int nc = t > 0 ? (t + chunk_tiles - 1) / chunk_tiles : 0;
-        const int rbs = n > 0 ? (G * n + kRowBlock - 1) / kRowBlock : 0;
-        w.req[i].n_chunks = nc;
-        w.req[i].base_unit = pos;                 // temporarily the sorted position
-        s_units[pos] = nc * Hkv * rbs;
+        r_pos[k] = pos;
+        r_nc[k] = t > 0 ? (t + chunk_tiles - 1) / chunk_tiles : 0;
+        s_units[pos] = r_nc[k] * Hkv * r_rbs[k];
     }
     __syncthreads();
-    // exclusive scan of s_units (B <= 4096): per-thread serial segments + warp scans
+    // exclusive scan of s_units: per-thread serial segments + warp scans
     {
         const int per = (B + blockDim.x - 1) / blockDim.x;
         const int b0 = tid * per, b1 = min(B, b0 + per);
         int sum = 0;
-        for (int k = b0; k < b1; ++k) sum += s_units[k];
+        for (int q = b0; q < b1; ++q) sum += s_units[q];
         int incl = sum;
         for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if ((tid & 31) >= o) incl += y; }
         if ((tid & 31) == 31) s_red[tid >> 5] = incl;
@@ -114,15 +119,19 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         }
         __syncthreads();
         int run = s_red[tid >> 5] + incl - sum;
-        for (int k = b0; k < b1; ++k) { const int u = s_units[k]; s_units[k] = run; run += u; }
+        for (int q = b0; q < b1; ++q) { const int u = s_units[q]; s_units[q] = run; run += u; }
     }
     __syncthreads();
     // unit table: per request, chunks balanced to within one tile, order (chunk, kv head, row block)
-    for (int i = tid; i < B; i += blockDim.x) {
-        const int base = s_units[w.req[i].base_unit];
-        w.req[i].base_unit = base;
-        const int nc = w.req[i].n_chunks, t = s_tiles[i], n = w.req[i].n_nodes;
-        const int rbs = n > 0 ? (G * n + kRowBlock - 1) / kRowBlock : 0;
+#pragma unroll
+    for (int k = 0; k < kPer; ++k) {
+        const int i = tid + k * 1024;
+        if (i >= B) continue;
+        const int base = s_units[r_pos[k]];
+        const int nc = r_nc[k], t = r_tiles[k], rbs = r_rbs[k];
+        AttnReq rq;
+        rq.base_unit = base; rq.n_chunks = nc; rq.n_tiles = t; rq.n_nodes = r_n[k];
+        w.req[i] = rq;
         int u = base;
         for (int c = 0; c < nc; ++c) {
             const int tb = (int)((long long)t * c / nc), te = (int)((long long)t * (c + 1) / nc);
