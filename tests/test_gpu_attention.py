@@ -66,9 +66,9 @@ def test_tiny_config(war, kernel):
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
-@pytest.mark.parametrize("case", ["ragged16", "ragged32", "wide", "single", "deep"])
+@pytest.mark.parametrize("case", ["ragged16", "ragged32", "wide", "single", "deep", "many", "rows256"])
 def test_shapes_and_ragged_lengths(war, kernel, case):
-    rng = np.random.default_rng(["ragged16", "ragged32", "wide", "single", "deep"].index(case))
+    rng = np.random.default_rng(["ragged16", "ragged32", "wide", "single", "deep", "many", "rows256"].index(case))
     base = W.CONFIGS["tiny"]
     if case == "ragged16":       # lengths around page and tile edges, empty prefix, an unused request
         ctx = np.array([1, 2, 15, 16, 17, 113, 127, 128, 129, 1000, 1024, 1025, 2049, 3000])
@@ -87,6 +87,14 @@ def test_shapes_and_ragged_lengths(war, kernel, case):
         ctx = np.array([300, 4000, 9])
         cfg = W.scaled(base, B=len(ctx), N=8)
         nn, parent = _random_trees(rng, cfg.B, cfg.N, n_fixed=[1, 1, 1])
+    elif case == "many":         # more requests than one planning pass handles per thread, all short
+        ctx = rng.integers(1, 300, size=1500)
+        cfg = W.scaled(base, B=len(ctx), N=4)
+        nn, parent = _random_trees(rng, cfg.B, cfg.N)
+    elif case == "rows256":      # 4 heads per group x 64 slots: two row blocks per kv head, the second partly filled
+        ctx = np.array([900, 130, 2000])
+        cfg = W.scaled(base, B=len(ctx), N=64)
+        nn, parent = _random_trees(rng, cfg.B, cfg.N, n_fixed=[64, 40, 33])
     else:                        # chains as deep as the budget allows (every ancestor bit set)
         ctx = np.array([257, 1500])
         cfg = W.scaled(base, B=len(ctx), N=32)
@@ -137,6 +145,26 @@ def test_needle_key_and_large_logits(war, kernel):
     G = cfg.Hq // cfg.Hkv
     want = a.v_pool[page, :, pos % cfg.page_size, :].float().cpu().numpy()
     np.testing.assert_allclose(got[0, 1, ::G, :], want, atol=2e-2, rtol=2e-2)
+
+
+def test_lse_is_optional_and_scale_is_an_argument(war):
+    cfg = W.scaled(W.CONFIGS["tiny"], B=2, N=8)
+    ctx = np.array([1300, 77])
+    a = W.make_attention_inputs(cfg, ctx, device="cuda:0")
+    nn, parent = _random_trees(np.random.default_rng(3), cfg.B, cfg.N)
+    d_nn = torch.from_numpy(nn).to("cuda:0"); d_par = torch.from_numpy(parent).to("cuda:0")
+    for scale in (0.02, 0.3):
+        params = war.attn_params(a.q, a.k_pool, a.v_pool, a.page_table, scale, 0)
+        ws = war.new_workspace(params, "cuda:0")
+        out = torch.zeros_like(a.q)
+        war.war_verify_attn(a.q, a.k_pool, a.v_pool, a.page_table, a.prefix_len, d_nn, d_par, params, ws, out, None)
+        torch.cuda.synchronize()
+        want = A.verify_attention(a.q, a.k_pool, a.v_pool, a.page_table.cpu().numpy(), a.prefix_len.cpu().numpy(), nn, parent, scale)
+        for i in range(cfg.B):
+            n = int(nn[i])
+            np.testing.assert_allclose(out[i, :n].float().cpu().numpy(), want[i][0].astype(np.float32), atol=1e-2, rtol=1e-2)
+    params = war.attn_params(a.q, a.k_pool, a.v_pool, a.page_table, 0.0, 0)
+    assert war.war_verify_attn_workspace_bytes(params) == 0          # scale must be positive
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
