@@ -210,6 +210,16 @@ def main():
     t0 = time.perf_counter()
     ix = war.war_index_build(d_tok, off, cfg.vocab, cfg.P + cfg.N, len(tok) + cfg.n_traj)
     index_build_s = time.perf_counter() - t0
+    # the index the steps use is then made the way a rollout would make it: all but the last trajectories first, the
+    # rest appended as an RL step's worth of new trajectories (an appended index answers exactly like a fresh build)
+    ix.destroy()
+    k_new = max(1, cfg.n_traj // 32)
+    ix = war.war_index_build(d_tok, off[:cfg.n_traj - k_new + 1], cfg.vocab, cfg.P + cfg.N, len(tok) + cfg.n_traj)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    war.war_index_append(ix, d_tok, off[cfg.n_traj - k_new:])
+    index_append_s = time.perf_counter() - t0
+    index_append_tokens = int(off[-1] - off[cfg.n_traj - k_new])
     del d_tok
     attn = W.make_attention_inputs(cfg, ctx, device=dev)
     B, N = cfg.B, cfg.N
@@ -354,6 +364,7 @@ def main():
             "breakdown_ms": {"draft": draft_ms, "verify_attn": attn_ms, "accept": accept_ms},
             "slots_verified_per_s": slots_all / (ms_per_step * 1e-3),
             "accept_len_mean": float(h_alen.mean()), "index_build_s": index_build_s, "index_tokens": int(len(tok)),
+            "index_append": {"trajectories": k_new, "tokens": index_append_tokens, "seconds": index_append_s},
             "device_status": status,
         }
         if not args.no_cpu_baseline and world == 1:

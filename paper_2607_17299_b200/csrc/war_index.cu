@@ -87,32 +87,6 @@ __global__ void lcp_kernel(const int32_t* __restrict__ corpus, const int32_t* __
     lcp[i] = (uint8_t)l;
 }
 
-__global__ void histogram_kernel(const int32_t* __restrict__ corpus, int64_t M, int vocab, uint32_t* __restrict__ hist) {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= M) return;
-    const int32_t c = corpus[i];
-    if (c >= 0 && c < vocab) atomicAdd(&hist[c], 1u);
-}
-
-// bucket[v] = T + sum_{u<v} hist[u]  (the T separators sort first); single block
-__global__ void bucket_scan_kernel(const uint32_t* __restrict__ hist, int vocab, int T, int32_t* __restrict__ bucket) {
-    typedef cub::BlockScan<uint32_t, 1024> Scan;
-    __shared__ typename Scan::TempStorage tmp;
-    __shared__ uint32_t carry;
-    if (threadIdx.x == 0) carry = (uint32_t)T;
-    __syncthreads();
-    for (int base = 0; base < vocab + 1; base += 1024) {
-        const int v = base + threadIdx.x;
-        const uint32_t x = v < vocab ? hist[v] : 0u;
-        uint32_t excl, total;
-        Scan(tmp).ExclusiveSum(x, excl, total);
-        if (v <= vocab) bucket[v] = (int32_t)(carry + excl);
-        __syncthreads();
-        if (threadIdx.x == 0) carry += total;
-        __syncthreads();
-    }
-}
-
 struct Scratch {
     void* p = nullptr;
     ~Scratch() { if (p) cudaFree(p); }
@@ -120,15 +94,12 @@ struct Scratch {
 
 inline dim3 grid_for(int64_t n) { return dim3((unsigned)((n + kThreads - 1) / kThreads)); }
 
-// (Re)builds sa / lcp / bucket from ix->corpus[0 .. M).
-war_status_t rebuild(war_index* ix, cudaStream_t s) {
-    const int64_t M = ix->M;
-    if (M == 0) {
-        WAR_CUDA_TRY(cudaMemsetAsync(ix->bucket, 0, sizeof(int32_t) * (ix->vocab + 1), s));
-        return WAR_OK;
-    }
-    const int n = (int)M;
-    // scratch: key64 x2, val x2, rank, flag, hist, cub temp
+// Sorts the n suffixes of `corpus[0 .. n)` (a run of whole trajectories, each ending in its separator) to depth
+// max_depth by prefix doubling and writes their start positions, relative to `corpus`, to out_sa (device, n entries).
+// T_total shifts the symbols so that every separator -(t+1), t < T_total, maps to a non-negative key.
+war_status_t sort_suffixes(const int32_t* corpus, int64_t n64, int T_total, int vocab, int max_depth, int32_t* out_sa,
+                           cudaStream_t s) {
+    const int n = (int)n64;
     size_t temp_sort64 = 0, temp_sort32 = 0, temp_scan = 0;
     {
         cub::DoubleBuffer<uint64_t> k64(nullptr, nullptr);
@@ -141,9 +112,8 @@ war_status_t rebuild(war_index* ix, cudaStream_t s) {
     size_t temp_bytes = temp_sort64 > temp_sort32 ? temp_sort64 : temp_sort32;
     if (temp_scan > temp_bytes) temp_bytes = temp_scan;
     auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
-    const size_t b_key = align(sizeof(uint64_t) * M), b_val = align(sizeof(int32_t) * M), b_u32 = align(sizeof(uint32_t) * M);
-    const size_t b_hist = align(sizeof(uint32_t) * (ix->vocab + 1));
-    const size_t total = 2 * b_key + 2 * b_val + 2 * b_u32 + b_hist + align(temp_bytes);
+    const size_t b_key = align(sizeof(uint64_t) * n64), b_val = align(sizeof(int32_t) * n64), b_u32 = align(sizeof(uint32_t) * n64);
+    const size_t total = 2 * b_key + 2 * b_val + 2 * b_u32 + align(temp_bytes);
     Scratch scratch;
     WAR_CUDA_TRY(cudaMalloc(&scratch.p, total));
     char* at = (char*)scratch.p;
@@ -153,40 +123,154 @@ war_status_t rebuild(war_index* ix, cudaStream_t s) {
     int32_t* val_b = (int32_t*)at; at += b_val;
     uint32_t* rank = (uint32_t*)at; at += b_u32;
     uint32_t* flag = (uint32_t*)at; at += b_u32;
-    uint32_t* hist = (uint32_t*)at; at += b_hist;
     void* temp = at;
 
     int sym_bits = 1;
-    while (((int64_t)1 << sym_bits) < (int64_t)ix->vocab + ix->T) ++sym_bits;
+    while (((int64_t)1 << sym_bits) < (int64_t)vocab + T_total) ++sym_bits;
     int pos_bits = 1;
-    while (((int64_t)1 << pos_bits) < M + 1) ++pos_bits;
+    while (((int64_t)1 << pos_bits) < n64 + 1) ++pos_bits;
 
     // round 0: order by the first token
     cub::DoubleBuffer<int32_t> val(val_a, val_b);
     {
         cub::DoubleBuffer<uint32_t> k32((uint32_t*)key_a, (uint32_t*)key_b);
-        init_keys_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, M, ix->T, k32.Current(), val.Current());
+        init_keys_kernel<<<grid_for(n64), kThreads, 0, s>>>(corpus, n64, T_total, k32.Current(), val.Current());
         WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(temp, temp_bytes, k32, val, n, 0, sym_bits, s));
-        flag32_kernel<<<grid_for(M), kThreads, 0, s>>>(k32.Current(), M, flag);
+        flag32_kernel<<<grid_for(n64), kThreads, 0, s>>>(k32.Current(), n64, flag);
         WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, flag, flag, MaxOp(), n, s));
-        scatter_rank_kernel<<<grid_for(M), kThreads, 0, s>>>(val.Current(), flag, M, rank);
+        scatter_rank_kernel<<<grid_for(n64), kThreads, 0, s>>>(val.Current(), flag, n64, rank);
     }
-    for (int64_t h = 1; h < ix->max_depth; h <<= 1) {
+    for (int64_t h = 1; h < max_depth; h <<= 1) {
         cub::DoubleBuffer<uint64_t> k64(key_a, key_b);
-        make_pair_keys_kernel<<<grid_for(M), kThreads, 0, s>>>(val.Current(), rank, M, h, k64.Current());
+        make_pair_keys_kernel<<<grid_for(n64), kThreads, 0, s>>>(val.Current(), rank, n64, h, k64.Current());
         WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(temp, temp_bytes, k64, val, n, 0, 32 + pos_bits, s));
-        flag64_kernel<<<grid_for(M), kThreads, 0, s>>>(k64.Current(), M, flag);
+        flag64_kernel<<<grid_for(n64), kThreads, 0, s>>>(k64.Current(), n64, flag);
         WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, flag, flag, MaxOp(), n, s));
-        scatter_rank_kernel<<<grid_for(M), kThreads, 0, s>>>(val.Current(), flag, M, rank);
+        scatter_rank_kernel<<<grid_for(n64), kThreads, 0, s>>>(val.Current(), flag, n64, rank);
     }
-    WAR_CUDA_TRY(cudaMemcpyAsync(ix->sa, val.Current(), sizeof(int32_t) * M, cudaMemcpyDeviceToDevice, s));
+    WAR_CUDA_TRY(cudaMemcpyAsync(out_sa, val.Current(), sizeof(int32_t) * n64, cudaMemcpyDeviceToDevice, s));
+    WAR_LAUNCH_CHECK();
+    WAR_CUDA_TRY(cudaStreamSynchronize(s));          // the scratch is freed on return
+    return WAR_OK;
+}
+
+// bucket[v] = first suffix-array index whose suffix starts with a token >= v (tokens ascend along the suffix array,
+// the T separators come first); one thread per entry fills the gap between its predecessor's token and its own.
+__global__ void bucket_from_sa_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, int64_t M, int vocab,
+                                      int32_t* __restrict__ bucket) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i > M) return;
+    const int cur = i < M ? max(corpus[sa[i]], -1) : vocab;          // sentinel after the last suffix
+    const int prev = i > 0 ? max(corpus[sa[i - 1]], -1) : -1;
+    for (int v = prev + 1; v <= min(cur, vocab); ++v) bucket[v] = (int32_t)i;
+}
+
+// lcp and buckets from a finished suffix array
+war_status_t finish_index(war_index* ix, cudaStream_t s) {
+    const int64_t M = ix->M;
     lcp_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, ix->sa, M, ix->max_depth, ix->lcp);
-    WAR_CUDA_TRY(cudaMemsetAsync(hist, 0, b_hist, s));
-    histogram_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, M, ix->vocab, hist);
-    bucket_scan_kernel<<<1, 1024, 0, s>>>(hist, ix->vocab, ix->T, ix->bucket);
+    bucket_from_sa_kernel<<<grid_for(M + 1), kThreads, 0, s>>>(ix->corpus, ix->sa, M, ix->vocab, ix->bucket);
     WAR_LAUNCH_CHECK();
     WAR_CUDA_TRY(cudaStreamSynchronize(s));
     return WAR_OK;
+}
+
+// (Re)builds sa / lcp / bucket from ix->corpus[0 .. M).
+war_status_t rebuild(war_index* ix, cudaStream_t s) {
+    const int64_t M = ix->M;
+    if (M == 0) {
+        WAR_CUDA_TRY(cudaMemsetAsync(ix->bucket, 0, sizeof(int32_t) * (ix->vocab + 1), s));
+        return WAR_OK;
+    }
+    const war_status_t st = sort_suffixes(ix->corpus, M, ix->T, ix->vocab, ix->max_depth, ix->sa, s);
+    if (st != WAR_OK) return st;
+    return finish_index(ix, s);
+}
+
+// ---- incremental append -------------------------------------------------------------------------
+// Separators isolate trajectories, so appending never changes the relative order of the old suffixes.  The new
+// suffixes are sorted among themselves, each finds how many old suffixes precede it (binary search inside its first
+// token's old bucket, to the depth the index is ordered to), and the two sorted lists are merged by scatter.
+
+// pos[j] = number of old suffixes that sort before new suffix j (lower bound; equal-to-depth ties go after it)
+__global__ void insert_pos_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa_old,
+                                  const int32_t* __restrict__ bucket_old, const int32_t* __restrict__ new_sa, int64_t m, int64_t M_old,
+                                  int vocab, int depth, uint32_t* __restrict__ pos) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= m) return;
+    const int64_t p = M_old + new_sa[j];
+    const int c0 = corpus[p];
+    if (c0 < 0 || c0 >= vocab) { pos[j] = 0u; return; }     // new separators are smaller than every old entry
+    int a = bucket_old[c0], z = bucket_old[c0 + 1];
+    int ma = 1, mz = 1;                                     // tokens known equal at the current ends (bucket: token 0)
+    while (a < z) {
+        const int mid = a + ((z - a) >> 1);
+        const int64_t q = sa_old[mid];
+        int t = min(ma, mz);
+        int cmp = 0;                                        // sign of (old suffix - new suffix)
+        for (; t < depth; ++t) {
+            const int x = corpus[q + t], y = corpus[p + t];
+            if (x != y) { cmp = x < y ? -1 : 1; break; }
+        }
+        if (cmp < 0) { a = mid + 1; ma = t; } else { z = mid; mz = t; }
+    }
+    pos[j] = (uint32_t)a;
+}
+
+__global__ void count_pos_kernel(const uint32_t* __restrict__ pos, int64_t m, uint32_t* __restrict__ add) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < m) atomicAdd(&add[pos[j]], 1u);
+}
+
+// old suffix i moves behind the new suffixes that were inserted at or before it
+__global__ void scatter_old_kernel(const int32_t* __restrict__ sa_old, const uint32_t* __restrict__ shift, int64_t M_old,
+                                   int32_t* __restrict__ sa_out) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < M_old) sa_out[i + shift[i]] = sa_old[i];
+}
+
+__global__ void scatter_new_kernel(const int32_t* __restrict__ new_sa, const uint32_t* __restrict__ pos, int64_t m, int64_t M_old,
+                                   int32_t* __restrict__ sa_out) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < m) sa_out[(int64_t)pos[j] + j] = (int32_t)(M_old + new_sa[j]);
+}
+
+struct SumOp {
+    __device__ __forceinline__ uint32_t operator()(uint32_t a, uint32_t b) const { return a + b; }
+};
+
+war_status_t merge_new_suffixes(war_index* ix, int64_t M_old, cudaStream_t s) {
+    const int64_t M = ix->M, m = M - M_old;
+    auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    size_t temp_scan = 0, temp_scan2 = 0;
+    WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(nullptr, temp_scan, (uint32_t*)nullptr, (uint32_t*)nullptr, MaxOp(), (int)m, s));
+    WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(nullptr, temp_scan2, (uint32_t*)nullptr, (uint32_t*)nullptr, SumOp(), (int)(M_old + 1), s));
+    size_t temp_bytes = temp_scan > temp_scan2 ? temp_scan : temp_scan2;
+    const size_t b_new = align(sizeof(int32_t) * m), b_pos = align(sizeof(uint32_t) * m), b_add = align(sizeof(uint32_t) * (M_old + 1)),
+                 b_out = align(sizeof(int32_t) * M);
+    Scratch scratch;
+    WAR_CUDA_TRY(cudaMalloc(&scratch.p, b_new + b_pos + b_add + b_out + align(temp_bytes)));
+    char* at = (char*)scratch.p;
+    int32_t* new_sa = (int32_t*)at; at += b_new;
+    uint32_t* pos = (uint32_t*)at; at += b_pos;
+    uint32_t* add = (uint32_t*)at; at += b_add;
+    int32_t* sa_out = (int32_t*)at; at += b_out;
+    void* temp = at;
+
+    war_status_t st = sort_suffixes(ix->corpus + M_old, m, ix->T, ix->vocab, ix->max_depth, new_sa, s);
+    if (st != WAR_OK) return st;
+    insert_pos_kernel<<<grid_for(m), kThreads, 0, s>>>(ix->corpus, ix->sa, ix->bucket, new_sa, m, M_old, ix->vocab, ix->max_depth, pos);
+    // positions must not decrease along the sorted new suffixes (they cannot, up to ties at full depth): enforce it
+    WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, pos, pos, MaxOp(), (int)m, s));
+    WAR_CUDA_TRY(cudaMemsetAsync(add, 0, b_add, s));
+    count_pos_kernel<<<grid_for(m), kThreads, 0, s>>>(pos, m, add);
+    WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, add, add, SumOp(), (int)(M_old + 1), s));
+    scatter_old_kernel<<<grid_for(M_old), kThreads, 0, s>>>(ix->sa, add, M_old, sa_out);
+    scatter_new_kernel<<<grid_for(m), kThreads, 0, s>>>(new_sa, pos, m, M_old, sa_out);
+    WAR_CUDA_TRY(cudaMemcpyAsync(ix->sa, sa_out, sizeof(int32_t) * M, cudaMemcpyDeviceToDevice, s));
+    WAR_LAUNCH_CHECK();
+    st = finish_index(ix, s);
+    return st;
 }
 
 war_status_t check_offsets(const int64_t* h_offsets, int32_t T) {
@@ -268,8 +352,11 @@ extern "C" war_status_t war_index_append(war_index_t* ix, const int32_t* d_token
     war_status_t st = check_offsets(h_offsets, T);
     if (st != WAR_OK) return st;
     if (T == 0) return WAR_OK;
+    const int64_t M_old = ix->M;
     st = add_trajectories(ix, d_tokens, h_offsets, T, stream);
     if (st != WAR_OK) return st;
+    // merging pays when the addition is the smaller part; otherwise sort everything again
+    if (M_old > 0 && ix->M - M_old < M_old) return merge_new_suffixes(ix, M_old, stream);
     return rebuild(ix, stream);
 }
 

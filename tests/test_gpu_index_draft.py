@@ -183,6 +183,48 @@ def test_append_equals_rebuild_and_order_independence(war):
     ix2.destroy()
 
 
+@pytest.mark.parametrize("seed", range(3))
+def test_incremental_appends_keep_a_valid_suffix_array(war, seed):
+    """Small appends take the merge path (new suffixes sorted on their own, then merged into the old order).  After
+    every append the suffix array must be a depth-ordered permutation with correct LCP and buckets, and drafts must
+    equal the brute-force checker's on everything stored so far."""
+    rng = np.random.default_rng(40 + seed)
+    vocab = 5
+    trajs = [rng.integers(0, vocab, size=int(rng.integers(0, 400))).tolist() for _ in range(14)]
+    tok, off = _flat(trajs)
+    d_tok = torch.from_numpy(tok).to("cuda:0")
+    cap = len(tok) + len(trajs)
+    ix = U.build_index(war, tok[:off[6]], off[:7], vocab, max_depth=96, capacity=cap)
+    tails = rng.integers(0, vocab, size=(40, 12)).astype(np.int32)
+    tl = rng.integers(0, 13, size=40).astype(np.int32)
+    done = 6
+    for step in (1, 2, 1, 3, 1):                                        # each addition is smaller than what is stored
+        war.war_index_append(ix, d_tok, off[done:done + step + 1])
+        done += step
+        info = war.war_index_info(ix)
+        M = int(info.M)
+        assert M == off[done] + done and info.T == done
+        sa = _read_device(info.d_sa, M * 4).view(np.int32)
+        lcp = _read_device(info.d_lcp, M)
+        corpus = _read_device(info.d_corpus, M * 4).view(np.int32).tolist()
+        bucket = _read_device(info.d_bucket, (vocab + 1) * 4).view(np.int32)
+        assert sorted(sa.tolist()) == list(range(M))
+        key = lambda i: corpus[i:i + 128]
+        naive = sorted(range(M), key=lambda i: corpus[i:])
+        assert [key(i) for i in sa] == [key(i) for i in naive]
+        for i in range(1, M):
+            a, b = corpus[sa[i - 1]:], corpus[sa[i]:]
+            l = 0
+            while l < min(len(a), len(b), 96) and a[l] == b[l]:
+                l += 1
+            assert lcp[i] == l
+        firsts = np.array([corpus[i] for i in sa])
+        for v in range(vocab + 1):
+            assert bucket[v] == int((firsts < v).sum())
+        _compare_with_oracle(war, tok[:off[done]], off[:done + 1], vocab, tails, tl, 24, 4, ix=ix)
+    ix.destroy()
+
+
 def test_empty_and_degenerate_inputs(war):
     ix = U.build_index(war, np.zeros(0, np.int32), np.zeros(1, np.int64), vocab=10, capacity=64)   # no trajectories
     tails = np.array([[1, 2, 3, 4]], np.int32)
