@@ -320,8 +320,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
             for (int t = 0; t < T && ok; ++t) {
                 const uint32_t g = t & 1, tg = cg[g] + (uint32_t)(t >> 1);
                 const uint32_t sq = seq_v(ld0, t, T), slot = sq % kSlots;
+                const bool has_s = t + 2 < T;                        // S(t+2) goes out in the same burst as PV(t)
+                const uint32_t sq_k = has_s ? seq_k(ld0, t + 2) : 0u, slot_k = sq_k % kSlots;
                 ok = mbar_wait(&bars->p_ready[g], tg & 1u, bars, a.status_word) &&
                      mbar_wait(&bars->full[slot], (sq / kSlots) & 1u, bars, a.status_word);
+                if (ok && has_s) ok = mbar_wait(&bars->full[slot_k], (sq_k / kSlots) & 1u, bars, a.status_word);
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
@@ -330,11 +333,24 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
                         umma_bf16_ts(d_o, a_p + (uint32_t)ks * 8u, pack64(v_lo + (uint32_t)ks * (4096u >> 4), hi_kv), idesc_o, ks > 0 ? 1u : acc0);
+                    if (has_s) {
+                        // sixteen MMAs back to back; the completion signals follow the burst (the one the softmax group
+                        // waits for first)
+                        const uint32_t k_lo = ring_lo + slot_k * (kSlotBytes >> 4), d_s = tmem + g * 128u;
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            constexpr uint32_t kHalfQ = 16384u >> 4, kHalfK = 1024u >> 4;
+                            const uint32_t qo = (uint32_t)(ks >> 2) * kHalfQ + (uint32_t)(ks & 3) * 2u;
+                            const uint32_t ko = (uint32_t)(ks >> 2) * kHalfK + (uint32_t)(ks & 3) * 2u;
+                            umma_bf16(d_s, pack64(q_lo + qo, hi_q), pack64(k_lo + ko, hi_kv), idesc_s, ks > 0);
+                        }
+                        umma_commit(&bars->s_ready[g]);
+                    }
                     umma_commit(&bars->pv_done[g]);
                     umma_commit(&bars->empty[slot]);
+                    if (has_s) umma_commit(&bars->empty[slot_k]);
                 }
                 __syncwarp();
-                if (t + 2 < T) ok = issue_s(t + 2);
             }
             cg[0] += (uint32_t)(T + 1) >> 1;
             cg[1] += (uint32_t)T >> 1;
