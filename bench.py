@@ -52,7 +52,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -254,12 +254,20 @@ def main():
             attn_events[1].record()
         war.war_accept(d_ids, d_par, d_nn, d_target, 0, d_alen, d_path, d_bonus)
 
+    # nvidia-smi needs a few hundred ms to start reporting, so the sampler runs from the warm-up through the timed
+    # region (and is given a moment to produce its first lines while the GPU is already under load)
+    clocks = ClockSampler(local_rank)
+    clocks.__enter__()
+    t_warm = time.perf_counter()
     for _ in range(args.warmup):
         step()
+    while time.perf_counter() - t_warm < 0.6 and not clocks.rows:
+        step()
+        torch.cuda.synchronize()
     barrier()
     attn_ev = [(ev(), ev()) for _ in range(args.steps)]
     draft_ev = [ev() for _ in range(args.steps + 1)]
-    with ClockSampler(local_rank) as clocks:
+    if True:
         barrier()
         start, stop = ev(), ev()
         start.record()
@@ -270,6 +278,8 @@ def main():
         stop.record()
         barrier()
         total_ms = start.elapsed_time(stop)
+    time.sleep(0.06)                                       # let the sampler see the end of the timed region
+    clocks.__exit__(None, None, None)
     attn_ms = float(np.mean([a.elapsed_time(b) for a, b in attn_ev]))
     draft_ms = float(np.mean([draft_ev[s].elapsed_time(attn_ev[s][0]) for s in range(args.steps)]))
     accept_ms = float(np.mean([attn_ev[s][1].elapsed_time(draft_ev[s + 1]) for s in range(args.steps)]))

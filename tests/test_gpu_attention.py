@@ -184,6 +184,28 @@ def test_page_permutation_leaves_bits_unchanged(war, kernel):
     assert torch.equal(raw1, raw2)
 
 
+def test_kv_head_shards_equal_the_unsharded_call(war):
+    """Tensor-parallel replicas shard the kv heads (and their query-head groups): a rank calls the library on its
+    own slice of the pools and of q.  Outputs of the shards, put side by side, must equal the unsharded call bit for
+    bit (each kv head is an independent problem)."""
+    cfg = W.scaled(W.CONFIGS["tiny"], B=3, N=16)
+    ctx = np.array([2100, 400, 900])
+    rng = np.random.default_rng(5)
+    nn, parent = _random_trees(rng, cfg.B, cfg.N)
+    a = W.make_attention_inputs(cfg, ctx, device="cuda:0")
+    _, _, full = U.run_attn(war, a, nn, parent, 0.09, 0)
+    G = cfg.Hq // cfg.Hkv
+    shards = []
+    for r in range(2):                                                     # two ranks, four kv heads each
+        h0, h1 = r * cfg.Hkv // 2, (r + 1) * cfg.Hkv // 2
+        b = W.AttnInputs(q=a.q[:, :, h0 * G:h1 * G, :].contiguous(), k_pool=a.k_pool[:, h0:h1].contiguous(),
+                         v_pool=a.v_pool[:, h0:h1].contiguous(), page_table=a.page_table, prefix_len=a.prefix_len,
+                         num_pages=a.num_pages, max_pages=a.max_pages)
+        _, _, part = U.run_attn(war, b, nn, parent, 0.09, 0)
+        shards.append(part)
+    assert torch.equal(torch.cat(shards, dim=2), full)
+
+
 @pytest.mark.parametrize("kernel", KERNELS)
 def test_malformed_inputs_are_reported_not_faulted(war, kernel):
     cfg = W.scaled(W.CONFIGS["tiny"], B=2, N=8)
