@@ -24,7 +24,7 @@ constexpr int kMaxN = 64;
 constexpr int kMaxK = 8;
 constexpr int kMaxP = 32;
 constexpr int kPoolCap = kMaxN * kMaxK;
-constexpr int kBlockScanMin = 8192;          // intervals at least this long are scanned by every warp
+constexpr int kBlockScanMin = 1024;          // intervals at least this long are scanned by every warp (measured: 1024-2048 best)
 constexpr int kLongRunFirstMin = 1024;       // intervals at least this long first look for runs of 16 or more only
 
 struct TopK {                                 // warp-uniform, sorted by (cnt desc, start asc)
