@@ -57,7 +57,8 @@ typedef struct war_index war_index_t;          /* opaque; lives on the device th
 /* ------------------------------------------------------------------------------------------------
  * Trajectory cache (paper Section 3.2: SuffixDecoding "caches token-sequence patterns from previously
  * generated trajectories"; the "external update interface" adds newly generated trajectories after each
- * RL step).  Trajectory t is d_tokens[h_offsets[t] .. h_offsets[t+1]); token ids lie in [0, vocab).
+ * RL step).  Trajectory t is d_tokens[h_offsets[t] .. h_offsets[t+1]); token ids must lie in [0, vocab)
+ * (checked on the device: WAR_ERR_INVALID_ARG, nothing added).
  * Inside the index the trajectories are joined with one unique negative separator each, so no match ever
  * straddles two trajectories.  The suffix array is ordered to depth max_depth (>= P + N of every later
  * war_draft call; <= 128) and LCP values are capped there.

@@ -19,8 +19,10 @@ struct MaxOp {
 };
 
 // corpus[dst_base + off[t] + t + i] = tokens[off[t] + i]; separator -(t0 + t + 1) after each trajectory.
+// A token id outside [0, vocab) raises *bad (such ids would collide with separators or overflow the sort keys).
 __global__ void scatter_corpus_kernel(const int32_t* __restrict__ tokens, const int64_t* __restrict__ off, int T,
-                                      int t0, int64_t dst_base, int32_t* __restrict__ corpus, int64_t n_out) {
+                                      int t0, int64_t dst_base, int32_t* __restrict__ corpus, int64_t n_out, int vocab,
+                                      int* __restrict__ bad) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_out) return;
     // trajectory t covers output positions [off[t] + t, off[t+1] + t]; the last one is its separator
@@ -32,7 +34,12 @@ __global__ void scatter_corpus_kernel(const int32_t* __restrict__ tokens, const 
     const int t = lo;
     const int64_t local = i - (off[t] + t);
     const int64_t len = off[t + 1] - off[t];
-    corpus[dst_base + i] = local < len ? tokens[off[t] + local] : -(t0 + t + 1);
+    int32_t v = -(t0 + t + 1);
+    if (local < len) {
+        v = tokens[off[t] + local];
+        if (v < 0 || v >= vocab) *bad = 1;
+    }
+    corpus[dst_base + i] = v;
 }
 
 // first-round key: separators (negative, unique) below every token
@@ -294,17 +301,22 @@ war_status_t add_trajectories(war_index* ix, const int32_t* d_tokens, const int6
     int64_t* rel = new (std::nothrow) int64_t[T + 1];
     if (!rel) return WAR_ERR_OOM;
     for (int t = 0; t <= T; ++t) rel[t] = h_offsets[t] - h_offsets[0];
-    Scratch off;
-    cudaError_t e = cudaMalloc(&off.p, sizeof(int64_t) * (T + 1));
+    Scratch off;                                             // offsets, then one int: the bad-token flag
+    int bad = 0;
+    cudaError_t e = cudaMalloc(&off.p, sizeof(int64_t) * (T + 2));
+    int* d_bad = e == cudaSuccess ? (int*)((int64_t*)off.p + (T + 1)) : nullptr;
     if (e == cudaSuccess) e = cudaMemcpyAsync(off.p, rel, sizeof(int64_t) * (T + 1), cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(d_bad, 0, sizeof(int), s);
     if (e == cudaSuccess) {
         scatter_corpus_kernel<<<grid_for(n_out), kThreads, 0, s>>>(d_tokens + h_offsets[0], (const int64_t*)off.p, T, ix->T,
-                                                                  ix->M, ix->corpus, n_out);
+                                                                  ix->M, ix->corpus, n_out, ix->vocab, d_bad);
         e = cudaGetLastError();
     }
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     delete[] rel;
     if (e != cudaSuccess) { (void)cudaGetLastError(); return e == cudaErrorMemoryAllocation ? WAR_ERR_OOM : WAR_ERR_CUDA; }
+    if (bad) return WAR_ERR_INVALID_ARG;                     // nothing was committed: M and T are unchanged
     ix->M += n_out;
     ix->T += T;
     return WAR_OK;

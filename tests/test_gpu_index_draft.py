@@ -234,4 +234,11 @@ def test_empty_and_degenerate_inputs(war):
     war.war_index_append(ix, d_tok, np.array([0, 0, 5, 5]))            # empty trajectories around a real one
     ml, nn, ids, par, cnt = U.run_draft(war, ix, tails, np.array([4]), 8, 4, with_count=False)
     assert ml[0] == 4 and nn[0] == 2 and ids[0, :2].tolist() == [4, 5] and cnt is None
+    for bad in (10, -1):                                               # ids outside [0, vocab) are refused, nothing changes
+        with pytest.raises(war.WarError) as e:
+            war.war_index_append(ix, torch.tensor([1, bad, 3], dtype=torch.int32, device="cuda:0"), np.array([0, 3]))
+        assert e.value.code == 1
+    assert war.war_index_info(ix).M == 8 and war.war_index_info(ix).T == 3
+    ml, nn, ids, par, cnt = U.run_draft(war, ix, tails, np.array([4]), 8, 4)
+    assert ml[0] == 4 and nn[0] == 2 and ids[0, :2].tolist() == [4, 5]
     ix.destroy()
