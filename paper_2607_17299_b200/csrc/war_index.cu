@@ -3,8 +3,9 @@
 // Only ordering to depth max_depth (<= 128) is ever needed by the draft kernel (it compares at most P pattern
 // tokens and descends at most N-1 further), so prefix doubling stops after ceil(log2(max_depth)) rounds.
 // Round r sorts 64-bit keys (rank of the first 2^r tokens, rank of the next 2^r tokens) with a device radix
-// sort and re-ranks by adjacent difference + scan.  Suffixes that still tie after the last round keep the
-// order the stable sort left them in; no output of the library depends on that order.
+// sort and re-ranks by adjacent difference + scan; suffixes whose rank is already unique drop out of later rounds.
+// Suffixes that still tie after the last round keep the order the stable sort left them in; no output of the
+// library depends on that order.
 #include <cub/cub.cuh>
 #include <new>
 #include "war_common.cuh"
@@ -57,28 +58,12 @@ __global__ void flag32_kernel(const uint32_t* __restrict__ key, int64_t M, uint3
     flag[i] = (i > 0 && key[i] != key[i - 1]) ? (uint32_t)i : 0u;
 }
 
-__global__ void flag64_kernel(const uint64_t* __restrict__ key, int64_t M, uint32_t* __restrict__ flag) {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= M) return;
-    flag[i] = (i > 0 && key[i] != key[i - 1]) ? (uint32_t)i : 0u;
-}
-
 // rank[sa[i]] = index of the first suffix of i's group
 __global__ void scatter_rank_kernel(const int32_t* __restrict__ sa, const uint32_t* __restrict__ group_start, int64_t M,
                                     uint32_t* __restrict__ rank) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= M) return;
     rank[sa[i]] = group_start[i];
-}
-
-__global__ void make_pair_keys_kernel(const int32_t* __restrict__ sa, const uint32_t* __restrict__ rank, int64_t M, int64_t h,
-                                      uint64_t* __restrict__ key) {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= M) return;
-    const int64_t s = sa[i];
-    const uint64_t hi = rank[s];
-    const uint64_t lo = (s + h < M) ? (uint64_t)rank[s + h] + 1u : 0u;
-    key[i] = (hi << 32) | lo;
 }
 
 __global__ void lcp_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, int64_t M, int max_depth,
@@ -101,35 +86,88 @@ struct Scratch {
 
 inline dim3 grid_for(int64_t n) { return dim3((unsigned)((n + kThreads - 1) / kThreads)); }
 
+// ---- prefix doubling over the suffixes that are still tied ---------------------------------------
+// After a round, a suffix whose rank is unique is final.  Later rounds only touch the slots of groups that still
+// hold two or more suffixes (`act`, ascending slot numbers): their (rank, rank at +h) keys are sorted on their own
+// and written back into the same slots, because a group occupies a contiguous slot range and the key's upper word
+// (the group's rank) keeps groups in slot order.
+
+__global__ void active_keys_kernel(const int32_t* __restrict__ act, const int32_t* __restrict__ sa, const uint32_t* __restrict__ rank,
+                                   int64_t n, int64_t h, int64_t m, uint64_t* __restrict__ key, int32_t* __restrict__ val) {
+    const int64_t a = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (a >= m) return;
+    const int64_t s = sa[act[a]];
+    const uint64_t hi = rank[s];
+    const uint64_t lo = (s + h < n) ? (uint64_t)rank[s + h] + 1u : 0u;
+    key[a] = (hi << 32) | lo;
+    val[a] = (int32_t)s;
+}
+
+// writes the sorted suffixes back into their slots; head[a] = slot number if a starts a new (sub)group, else 0
+__global__ void active_writeback_kernel(const int32_t* __restrict__ act, const uint64_t* __restrict__ key, const int32_t* __restrict__ val,
+                                        int64_t m, int32_t* __restrict__ sa, uint32_t* __restrict__ head) {
+    const int64_t a = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (a >= m) return;
+    sa[act[a]] = val[a];
+    head[a] = (a == 0 || key[a] != key[a - 1]) ? (uint32_t)act[a] : 0u;
+}
+
+__global__ void active_rank_kernel(const int32_t* __restrict__ val, const uint32_t* __restrict__ grp, int64_t m, uint32_t* __restrict__ rank) {
+    const int64_t a = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (a < m) rank[val[a]] = grp[a];
+}
+
+// keep[a] = 1 unless the suffix in slot act[a] is alone in its group (grp = slot of the group's first suffix)
+__global__ void active_keep_kernel(const int32_t* __restrict__ act, const uint32_t* __restrict__ grp, int64_t m, uint8_t* __restrict__ keep) {
+    const int64_t a = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (a >= m) return;
+    const bool is_head = grp[a] == (uint32_t)act[a];
+    const bool next_is_head = a + 1 == m || grp[a + 1] == (uint32_t)act[a + 1];
+    keep[a] = (is_head && next_is_head) ? 0 : 1;
+}
+
+__global__ void iota_kernel(int32_t* __restrict__ x, int64_t n) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) x[i] = (int32_t)i;
+}
+
 // Sorts the n suffixes of `corpus[0 .. n)` (a run of whole trajectories, each ending in its separator) to depth
 // max_depth by prefix doubling and writes their start positions, relative to `corpus`, to out_sa (device, n entries).
 // T_total shifts the symbols so that every separator -(t+1), t < T_total, maps to a non-negative key.
 war_status_t sort_suffixes(const int32_t* corpus, int64_t n64, int T_total, int vocab, int max_depth, int32_t* out_sa,
                            cudaStream_t s) {
     const int n = (int)n64;
-    size_t temp_sort64 = 0, temp_sort32 = 0, temp_scan = 0;
+    size_t t_sort64 = 0, t_sort32 = 0, t_scan = 0, t_sel = 0;
     {
         cub::DoubleBuffer<uint64_t> k64(nullptr, nullptr);
         cub::DoubleBuffer<uint32_t> k32(nullptr, nullptr);
         cub::DoubleBuffer<int32_t> v(nullptr, nullptr);
-        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(nullptr, temp_sort64, k64, v, n, 0, 64, s));
-        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(nullptr, temp_sort32, k32, v, n, 0, 32, s));
-        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(nullptr, temp_scan, (uint32_t*)nullptr, (uint32_t*)nullptr, MaxOp(), n, s));
+        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(nullptr, t_sort64, k64, v, n, 0, 64, s));
+        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(nullptr, t_sort32, k32, v, n, 0, 32, s));
+        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(nullptr, t_scan, (uint32_t*)nullptr, (uint32_t*)nullptr, MaxOp(), n, s));
+        WAR_CUDA_TRY(cub::DeviceSelect::Flagged(nullptr, t_sel, (int32_t*)nullptr, (uint8_t*)nullptr, (int32_t*)nullptr, (int*)nullptr, n, s));
     }
-    size_t temp_bytes = temp_sort64 > temp_sort32 ? temp_sort64 : temp_sort32;
-    if (temp_scan > temp_bytes) temp_bytes = temp_scan;
+    size_t temp_bytes = t_sort64;
+    if (t_sort32 > temp_bytes) temp_bytes = t_sort32;
+    if (t_scan > temp_bytes) temp_bytes = t_scan;
+    if (t_sel > temp_bytes) temp_bytes = t_sel;
     auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
-    const size_t b_key = align(sizeof(uint64_t) * n64), b_val = align(sizeof(int32_t) * n64), b_u32 = align(sizeof(uint32_t) * n64);
-    const size_t total = 2 * b_key + 2 * b_val + 2 * b_u32 + align(temp_bytes);
+    const size_t b_key = align(sizeof(uint64_t) * n64), b_i32 = align(sizeof(int32_t) * n64), b_u8 = align((size_t)n64);
+    // key x2, val x2, rank, head/group, act x2, keep, one counter, cub temp
+    const size_t total = 2 * b_key + 2 * b_i32 + 2 * b_i32 + 2 * b_i32 + b_u8 + 256 + align(temp_bytes);
     Scratch scratch;
     WAR_CUDA_TRY(cudaMalloc(&scratch.p, total));
     char* at = (char*)scratch.p;
     uint64_t* key_a = (uint64_t*)at; at += b_key;
     uint64_t* key_b = (uint64_t*)at; at += b_key;
-    int32_t* val_a = (int32_t*)at; at += b_val;
-    int32_t* val_b = (int32_t*)at; at += b_val;
-    uint32_t* rank = (uint32_t*)at; at += b_u32;
-    uint32_t* flag = (uint32_t*)at; at += b_u32;
+    int32_t* val_a = (int32_t*)at; at += b_i32;
+    int32_t* val_b = (int32_t*)at; at += b_i32;
+    uint32_t* rank = (uint32_t*)at; at += b_i32;
+    uint32_t* head = (uint32_t*)at; at += b_i32;
+    int32_t* act_a = (int32_t*)at; at += b_i32;
+    int32_t* act_b = (int32_t*)at; at += b_i32;
+    uint8_t* keep = (uint8_t*)at; at += b_u8;
+    int* d_count = (int*)at; at += 256;
     void* temp = at;
 
     int sym_bits = 1;
@@ -137,25 +175,40 @@ war_status_t sort_suffixes(const int32_t* corpus, int64_t n64, int T_total, int 
     int pos_bits = 1;
     while (((int64_t)1 << pos_bits) < n64 + 1) ++pos_bits;
 
-    // round 0: order by the first token
-    cub::DoubleBuffer<int32_t> val(val_a, val_b);
+    // round 0: order everything by the first token; out_sa holds the slots from here on
     {
         cub::DoubleBuffer<uint32_t> k32((uint32_t*)key_a, (uint32_t*)key_b);
+        cub::DoubleBuffer<int32_t> val(val_a, val_b);
         init_keys_kernel<<<grid_for(n64), kThreads, 0, s>>>(corpus, n64, T_total, k32.Current(), val.Current());
         WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(temp, temp_bytes, k32, val, n, 0, sym_bits, s));
-        flag32_kernel<<<grid_for(n64), kThreads, 0, s>>>(k32.Current(), n64, flag);
-        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, flag, flag, MaxOp(), n, s));
-        scatter_rank_kernel<<<grid_for(n64), kThreads, 0, s>>>(val.Current(), flag, n64, rank);
+        WAR_CUDA_TRY(cudaMemcpyAsync(out_sa, val.Current(), sizeof(int32_t) * n64, cudaMemcpyDeviceToDevice, s));
+        flag32_kernel<<<grid_for(n64), kThreads, 0, s>>>(k32.Current(), n64, head);
+        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, head, head, MaxOp(), n, s));
+        scatter_rank_kernel<<<grid_for(n64), kThreads, 0, s>>>(out_sa, head, n64, rank);
+        iota_kernel<<<grid_for(n64), kThreads, 0, s>>>(act_a, n64);
+        active_keep_kernel<<<grid_for(n64), kThreads, 0, s>>>(act_a, head, n64, keep);
+        WAR_CUDA_TRY(cub::DeviceSelect::Flagged(temp, temp_bytes, act_a, keep, act_b, d_count, n, s));
     }
-    for (int64_t h = 1; h < max_depth; h <<= 1) {
+    int32_t* act = act_b;
+    int32_t* act_other = act_a;
+    int m = 0;
+    WAR_CUDA_TRY(cudaMemcpyAsync(&m, d_count, sizeof(int), cudaMemcpyDeviceToHost, s));
+    WAR_CUDA_TRY(cudaStreamSynchronize(s));
+    for (int64_t h = 1; h < max_depth && m > 0; h <<= 1) {
         cub::DoubleBuffer<uint64_t> k64(key_a, key_b);
-        make_pair_keys_kernel<<<grid_for(n64), kThreads, 0, s>>>(val.Current(), rank, n64, h, k64.Current());
-        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(temp, temp_bytes, k64, val, n, 0, 32 + pos_bits, s));
-        flag64_kernel<<<grid_for(n64), kThreads, 0, s>>>(k64.Current(), n64, flag);
-        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, flag, flag, MaxOp(), n, s));
-        scatter_rank_kernel<<<grid_for(n64), kThreads, 0, s>>>(val.Current(), flag, n64, rank);
+        cub::DoubleBuffer<int32_t> val(val_a, val_b);
+        active_keys_kernel<<<grid_for(m), kThreads, 0, s>>>(act, out_sa, rank, n64, h, m, k64.Current(), val.Current());
+        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(temp, temp_bytes, k64, val, m, 0, 32 + pos_bits, s));
+        active_writeback_kernel<<<grid_for(m), kThreads, 0, s>>>(act, k64.Current(), val.Current(), m, out_sa, head);
+        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, head, head, MaxOp(), m, s));
+        active_rank_kernel<<<grid_for(m), kThreads, 0, s>>>(val.Current(), head, m, rank);
+        if ((h << 1) >= max_depth) break;                    // last round: nobody needs the next active list
+        active_keep_kernel<<<grid_for(m), kThreads, 0, s>>>(act, head, m, keep);
+        WAR_CUDA_TRY(cub::DeviceSelect::Flagged(temp, temp_bytes, act, keep, act_other, d_count, m, s));
+        WAR_CUDA_TRY(cudaMemcpyAsync(&m, d_count, sizeof(int), cudaMemcpyDeviceToHost, s));
+        WAR_CUDA_TRY(cudaStreamSynchronize(s));
+        int32_t* tmp = act; act = act_other; act_other = tmp;
     }
-    WAR_CUDA_TRY(cudaMemcpyAsync(out_sa, val.Current(), sizeof(int32_t) * n64, cudaMemcpyDeviceToDevice, s));
     WAR_LAUNCH_CHECK();
     WAR_CUDA_TRY(cudaStreamSynchronize(s));          // the scratch is freed on return
     return WAR_OK;
