@@ -199,7 +199,7 @@ struct Shared {
     int w_cnt[kWarps][kMaxK], w_start[kWarps][kMaxK];
     int st_cnt[32], st_start[32];               // runs that cross span edges (one per span) and the closing run
     int fin_cnt[kMaxK], fin_start[kMaxK], fin_tok[kMaxK];
-    int mode, cur, lo, cnt, depth, n_nodes, pool_n, thr_shared, long_runs_only;
+    int mode, cur, lo, cnt, depth, n_nodes, pool_n, thr_shared, long_runs_only, full_lo, full_cnt;
 };
 
 // Tokens from index `from` on of the suffix at s against the pattern; returns the sign and, in `matched`, how many
@@ -257,12 +257,13 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
     // Publishes the next node to expand: its token range (the interval minus the suffixes that end at this depth).
     auto publish = [&](int slot, int lo, int cnt, int depth) {          // warp 0, all lanes
         if (cnt <= 32) {                                                // handled in registers, one suffix per lane
-            if (lane == 0) { sh.cur = slot; sh.lo = lo; sh.cnt = cnt; sh.depth = depth; sh.long_runs_only = 0; sh.mode = 3; }
+            if (lane == 0) { sh.cur = slot; sh.lo = lo; sh.cnt = cnt; sh.depth = depth; sh.long_runs_only = 0; sh.mode = 3;
+                             sh.full_lo = lo; sh.full_cnt = cnt; }
             return;
         }
         const int e = count_ending(corpus, sa, lo, lo + cnt, depth, lane);
         if (lane == 0) {
-            sh.cur = slot; sh.lo = lo + e; sh.cnt = cnt - e; sh.depth = depth;
+            sh.cur = slot; sh.lo = lo + e; sh.cnt = cnt - e; sh.depth = depth; sh.full_lo = lo; sh.full_cnt = cnt;
             // Large nodes are first scanned for runs of 16 positions or more only (bar preset to 16): that pass never
             // walks the boundaries inside a lane.  It is exact whenever it finds k such runs; otherwise the node is
             // scanned again without the preset.
@@ -444,10 +445,43 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 }
             }
             __syncwarp();
-            if (sh.long_runs_only && n_fin < K) {                        // uniform: fewer than k long runs, look at all runs
+            int covered = 0;                                             // suffixes accounted for by the runs found
+            for (int e = 0; e < n_fin; ++e) covered += sh.fin_cnt[e];
+            if (sh.long_runs_only && n_fin < K && covered < cnt) {       // uniform: fewer than k long runs and more runs exist
                 __syncwarp();
                 if (lane == 0) { sh.long_runs_only = 0; sh.thr_shared = 0; }
                 continue;
+            }
+            // ---- chain shortcut ----
+            // If every occurrence of this node continues with the same token, that child has the node's own count; when
+            // no pooled offer reaches that count it is the strict best and becomes the next slot, and the same holds for
+            // its own single child, and so on for as long as the first and the last suffix of the interval agree (their
+            // common prefix is the common prefix of the whole interval).  All those slots are emitted at once.
+            if (n_fin == 1 && covered == sh.full_cnt) {
+                int pmax = 0;
+                for (int i = lane; i < sh.pool_n; i += 32) pmax = max(pmax, sh.pool_cnt[i]);
+                pmax = __reduce_max_sync(0xffffffffu, pmax);
+                const int c = sh.full_cnt, flo = sh.full_lo, j0 = sh.n_nodes, room = N - j0;
+                __syncwarp();
+                if (pmax < c && room > 0) {
+                    const int64_t s_first = sa[flo], s_last = sa[flo + c - 1];
+                    const int tf = lane < room ? corpus[s_first + d + lane] : -1;
+                    const int tl = lane < room ? corpus[s_last + d + lane] : -2;
+                    const unsigned eq = __ballot_sync(0xffffffffu, tf >= 0 && tf == tl);
+                    const int len = eq == 0xffffffffu ? 32 : __ffs(~eq) - 1;     // leading lanes that agree (>= 1 here)
+                    if (len >= 1) {
+                        if (lane < len) {
+                            o_ids[j0 + lane] = tf;
+                            o_par[j0 + lane] = j0 + lane - 1;                    // j0 - 1 is this node (the newest slot)
+                            if (o_cnt) o_cnt[j0 + lane] = c;
+                            sh.slot_depth[j0 + lane] = d + 1 + lane;
+                        }
+                        __syncwarp();
+                        if (lane == 0) { sh.n_nodes = j0 + len; sh.mode = 0; }
+                        if (j0 + len < N) publish(j0 + len - 1, flo, c, d + len);
+                        continue;
+                    }
+                }
             }
             // tokens of the winners, one lane each (the register path above already has them)
             if (mode != 3 && lane < n_fin) sh.fin_tok[lane] = corpus[(int64_t)sa[sh.fin_start[lane]] + d];
