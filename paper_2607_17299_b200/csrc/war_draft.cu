@@ -114,45 +114,62 @@ __device__ void warp_scan_span(const uint8_t* __restrict__ lcp, int d, int sb, i
             carry = max(carry, __shfl_sync(0xffffffffu, incl, 31));
             int thr = max(thr_local, *(volatile int*)thr_shared - 1);
             thr = __shfl_sync(0xffffffffu, thr, 0);                // one value for the whole warp
-            // candidates in ascending position order: lowest lane first, ascending inside a lane
-            bool have = false;
-            int c_cnt = 0, c_start = 0;
+            if (bits && prev < 0) my_first = pos0 + __ffs(bits) - 1;  // the span's very first boundary opens, closes nothing
             if (thr >= 15) {
-                // only the run that ends at this lane's first boundary can be long enough
-                if (bits) {
-                    const int bpos = pos0 + __ffs(bits) - 1;
-                    if (prev >= 0) {
-                        const int c = bpos - prev;
-                        if (c > thr) { c_cnt = c; c_start = prev; have = true; }
-                    } else {
-                        my_first = bpos;
+                // only the run that ends at a lane's first boundary can be long enough: one proposal per lane
+                int c = 0, st = 0;
+                if (bits && prev >= 0) { c = pos0 + __ffs(bits) - 1 - prev; st = prev; }
+                while (true) {
+                    // best proposal of the warp under (count desc, start asc)
+                    int bc = c > thr ? c : 0, bs = st;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const int oc = __shfl_xor_sync(0xffffffffu, bc, o), os = __shfl_xor_sync(0xffffffffu, bs, o);
+                        if (oc > bc || (oc == bc && oc > 0 && os < bs)) { bc = oc; bs = os; }
                     }
-                    bits = 0;
-                }
-            }
-            while (true) {
-                if (!have) {
-                    while (bits) {
-                        const int t = __ffs(bits) - 1;
-                        bits &= bits - 1;
-                        const int bpos = pos0 + t;
-                        if (prev >= 0) {
-                            const int c = bpos - prev;
-                            if (c > thr) { c_cnt = c; c_start = prev; prev = bpos; have = true; break; }
-                        } else {
-                            my_first = bpos;
-                        }
-                        prev = bpos;
+                    if (bc == 0) break;
+                    topk_insert(tk, k, bc, bs);
+                    if (c == bc && st == bs) c = 0;
+                    if (tk.n == k) {
+#pragma unroll
+                        for (int i = 0; i < kMaxK; ++i) if (i == k - 1) thr_local = tk.cnt[i];
+                        if (lane == 0) atomicMax(thr_shared, thr_local);
+                        thr = max(thr, thr_local);
                     }
                 }
-                const unsigned vote = __ballot_sync(0xffffffffu, have);
-                if (!vote) break;
-                const int src = __ffs(vote) - 1;
-                const int cc = __shfl_sync(0xffffffffu, c_cnt, src);
-                const int cs = __shfl_sync(0xffffffffu, c_start, src);
-                if (lane == src) have = false;
-                if (cc > thr) {
-                    topk_insert(tk, k, cc, cs);
+            } else {
+                // Dense case.  Every lane walks its own boundaries (all lanes at once) and proposes its best run that
+                // still beats the bar; the warp takes the best proposal, raises the bar, and asks again.  At most k
+                // rounds per chunk can succeed, so the cost stays bounded however many tiny runs there are.
+                // len[t]: length of the run that ends at this lane's position t (0: no boundary there, or nothing opened it)
+                int len[16];
+                {
+                    int p = prev;
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) {
+                        const bool bd = (bits >> t) & 1u;
+                        len[t] = (bd && p >= 0) ? pos0 + t - p : 0;
+                        p = bd ? pos0 + t : p;
+                    }
+                }
+                while (true) {
+                    int c = 0, ct = 0;
+#pragma unroll
+                    for (int t = 0; t < 16; ++t)
+                        if (len[t] > thr && len[t] > c) { c = len[t]; ct = t; }      // strict: the earliest of equal runs
+                    const int st = pos0 + ct - c;
+                    int bc = c, bs = st;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const int oc = __shfl_xor_sync(0xffffffffu, bc, o), os = __shfl_xor_sync(0xffffffffu, bs, o);
+                        if (oc > bc || (oc == bc && oc > 0 && os < bs)) { bc = oc; bs = os; }
+                    }
+                    if (bc == 0) break;
+                    topk_insert(tk, k, bc, bs);
+                    if (c == bc && st == bs) {
+#pragma unroll
+                        for (int t = 0; t < 16; ++t) if (t == ct) len[t] = 0;            // taken
+                    }
                     if (tk.n == k) {
 #pragma unroll
                         for (int i = 0; i < kMaxK; ++i) if (i == k - 1) thr_local = tk.cnt[i];
