@@ -402,19 +402,19 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                     if (lane == wl) c = 0;
                     ++n_fin;
                 }
-            } else if (cnt > 0) {
-                int nw = kWarps;
-                if (mode == 1) {
-                    TopK tk;
-                    int fb, lb;
-                    warp_scan_span(lcp, d, lo, hi, K, lane, tk, fb, lb, &sh.thr_shared);
-                    if (lane == 0) {
-                        sh.w_first[0] = fb; sh.w_last[0] = lb; sh.w_n[0] = tk.n;
+            } else if (cnt > 0 && mode == 1) {
+                // one warp saw the whole node: its list plus the closing run (last boundary to the end) is the answer
+                TopK tk;
+                int fb, lb;
+                warp_scan_span(lcp, d, lo, hi, K, lane, tk, fb, lb, &sh.thr_shared);
+                if (lb >= 0) topk_insert(tk, K, hi - lb, lb);
+                n_fin = tk.n;
+                if (lane == 0) {
 #pragma unroll
-                        for (int i = 0; i < kMaxK; ++i) { sh.w_cnt[0][i] = tk.cnt[i]; sh.w_start[0][i] = tk.start[i]; }
-                    }
-                    nw = 1;
+                    for (int i = 0; i < kMaxK; ++i) { sh.fin_cnt[i] = tk.cnt[i]; sh.fin_start[i] = tk.start[i]; }
                 }
+            } else if (cnt > 0) {
+                const int nw = kWarps;
                 __syncwarp();
                 // runs that cross span edges: span w's first boundary closes the run opened by the last boundary before it
                 const int wf = lane < nw ? sh.w_first[lane] : -1;
