@@ -132,6 +132,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kernel", type=int, default=0, help="0 = tensor-core verify attention, 1 = plain CUDA-core kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flush-l2", action="store_true",
+                    help="write a 256 MB scratch buffer before every timed step (for workloads whose KV cache fits L2); "
+                         "ms_per_step is then the mean of the per-step event intervals, the flush excluded")
     ap.add_argument("--requests", type=int, default=0,
                     help="run the workload's recipe with this many requests instead of its own count (profiling-size cases)")
     args = ap.parse_args()
@@ -150,7 +153,8 @@ def main():
                                f"{cfg.Hq}q/{cfg.Hkv}kv heads, d={cfg.D}, page {cfg.page_size}",
                    "requests_per_gpu": cfg.B, "parallelism": f"replica x{world}" if world > 1 else "single gpu",
                    "l2": "inputs (KV cache) far larger than L2, no flush needed" if cfg.name != "tiny" else
-                         "KV cache fits L2: value is an L2-resident number"}
+                         ("L2 flushed (256 MB written) before every step" if args.flush_l2 else
+                          "KV cache fits L2: value is an L2-resident number (--flush-l2 gives the cold one)")}
 
     # ------------------------------------------------------------------------------------------
     if args.impl == "reference":
@@ -266,23 +270,26 @@ def main():
         torch.cuda.synchronize()
     barrier()
     attn_ev = [(ev(), ev()) for _ in range(args.steps)]
-    draft_ev = [ev() for _ in range(args.steps + 1)]
-    if True:
-        barrier()
-        start, stop = ev(), ev()
-        start.record()
-        for s in range(args.steps):
-            draft_ev[s].record()
-            step(attn_ev[s])
-        draft_ev[args.steps].record()
-        stop.record()
-        barrier()
-        total_ms = start.elapsed_time(stop)
+    step_ev = [(ev(), ev()) for _ in range(args.steps)]
+    scratch = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if args.flush_l2 else None
+    barrier()
+    start, stop = ev(), ev()
+    start.record()
+    for s in range(args.steps):
+        if scratch is not None:
+            scratch.fill_(s & 0xFF)
+        step_ev[s][0].record()
+        step(attn_ev[s])
+        step_ev[s][1].record()
+    stop.record()
+    barrier()
+    per_step = np.array([a.elapsed_time(b) for a, b in step_ev])
+    total_ms = float(per_step.sum()) if args.flush_l2 else start.elapsed_time(stop)
     time.sleep(0.06)                                       # let the sampler see the end of the timed region
     clocks.__exit__(None, None, None)
     attn_ms = float(np.mean([a.elapsed_time(b) for a, b in attn_ev]))
-    draft_ms = float(np.mean([draft_ev[s].elapsed_time(attn_ev[s][0]) for s in range(args.steps)]))
-    accept_ms = float(np.mean([attn_ev[s][1].elapsed_time(draft_ev[s + 1]) for s in range(args.steps)]))
+    draft_ms = float(np.mean([step_ev[s][0].elapsed_time(attn_ev[s][0]) for s in range(args.steps)]))
+    accept_ms = float(np.mean([attn_ev[s][1].elapsed_time(step_ev[s][1]) for s in range(args.steps)]))
     status = war.war_device_status()
     h_alen = d_alen.cpu().numpy()
     verified = int((h_alen.astype(np.int64) + 1).sum())
@@ -372,6 +379,7 @@ def main():
             "roofline_kernel": {"name": "war_verify_attn (plan + attention + combine launches)", "bytes_per_launch": kvb,
                                 "ms_per_launch": attn_ms},
             "breakdown_ms": {"draft": draft_ms, "verify_attn": attn_ms, "accept": accept_ms},
+            "step_ms": {"median": float(np.median(per_step)), "min": float(per_step.min()), "max": float(per_step.max())},
             "slots_verified_per_s": slots_all / (ms_per_step * 1e-3),
             "accept_len_mean": float(h_alen.mean()), "index_build_s": index_build_s, "index_tokens": int(len(tok)),
             "index_append": {"trajectories": k_new, "tokens": index_append_tokens, "seconds": index_append_s},

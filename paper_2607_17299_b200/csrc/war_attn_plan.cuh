@@ -3,8 +3,8 @@
 // A unit = (request, kv head, row block, KV chunk).  The rows of a unit are the (slot, query head of the group)
 // pairs r = slot * G + g of one kv head, cut into row blocks of at most kRowBlock rows; its chunk is a range of
 // 128-key tiles.  A tiny planning kernel cuts every request into chunks so that about kTargetUnits units exist,
-// orders requests longest-first and writes the unit table; the attention kernel's CTAs pull units from an atomic
-// counter; units of a split request leave (max, sum, unnormalised output) partials that a combine kernel merges
+// orders requests longest-first and writes the unit table; the attention kernel's persistent CTAs take units in a
+// fixed snake order; units of a split request leave (max, sum, unnormalised output) partials that a combine kernel merges
 // in chunk order.  Everything lives in the caller's workspace, so no call allocates.
 #pragma once
 #include <stdint.h>

@@ -13,65 +13,95 @@ constexpr float kLn2 = 0.6931471805599453f;
 // ------------------------------------------------------------------------------------------------
 // plan: one CTA
 // ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t shfl64(uint64_t v, int src) {
+    const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)v, src);
+    const uint32_t hi = __shfl_sync(0xffffffffu, (uint32_t)(v >> 32), src);
+    return ((uint64_t)hi << 32) | lo;
+}
+
 __global__ void __launch_bounds__(1024)
 attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ num_nodes,
                  const int32_t* __restrict__ parent, int B, int N, int Hkv, int G, int page_size, int max_pages,
                  AttnWorkspace w, int* status_word) {
-    constexpr int kPer = kMaxPlanB / 1024;    // requests per thread, kept in registers through all phases
+    constexpr int kPer = kMaxPlanB / 1024;    // requests per thread in the per-request phases
     __shared__ int s_tiles[kMaxPlanB];
     __shared__ int s_units[kMaxPlanB];        // units per request, indexed by sorted position; then exclusive scan
+    __shared__ uint16_t s_order[kMaxPlanB];   // request at each sorted position
+    __shared__ uint8_t s_n[kMaxPlanB];        // validated slot count
     __shared__ int s_red[32];
     __shared__ long long s_sum[32];
-    __shared__ int s_chunk_tiles;
-    const int tid = threadIdx.x;
+    __shared__ int s_chunk_tiles, s_total;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // ---- per request, one warp: validate, ancestor masks by pointer jumping, tile count ----
+    // Lane l holds slots l and l + 32.  After round r a slot's mask covers its 2^r nearest ancestors-or-self and its
+    // pointer is the 2^r-th ancestor (the root points at itself), so 6 rounds cover any tree of 64 slots.
+    for (int i = warp; i < B; i += 32) {
+        int n = num_nodes[i];
+        const int pl = prefix_len[i];
+        bool bad = n < 0 || n > N || pl < 0;
+        if (!bad && n > 0) {
+            const int32_t* prow = parent + (size_t)i * N;
+            const int j0 = lane, j1 = lane + 32;
+            int p0 = (j0 > 0 && j0 < n) ? prow[j0] : 0;
+            int p1 = (j1 < n) ? prow[j1] : 0;
+            const bool bad_l = (j0 > 0 && j0 < n && (p0 < 0 || p0 >= j0)) || (j1 < n && (p1 < 0 || p1 >= j1));
+            bad = __any_sync(0xffffffffu, bad_l);
+            if (!bad) {
+                uint64_t a0 = 1ull << j0, a1 = 1ull << j1;
+                if (n <= 32) {
+#pragma unroll
+                    for (int r = 0; r < 5; ++r) {
+                        const uint64_t b = shfl64(a0, p0);
+                        const int q = __shfl_sync(0xffffffffu, p0, p0);
+                        a0 |= b; p0 = q;
+                    }
+                } else {
+#pragma unroll
+                    for (int r = 0; r < 6; ++r) {
+                        const uint64_t b00 = shfl64(a0, p0 & 31), b01 = shfl64(a1, p0 & 31);
+                        const uint64_t b10 = shfl64(a0, p1 & 31), b11 = shfl64(a1, p1 & 31);
+                        const int q00 = __shfl_sync(0xffffffffu, p0, p0 & 31), q01 = __shfl_sync(0xffffffffu, p1, p0 & 31);
+                        const int q10 = __shfl_sync(0xffffffffu, p0, p1 & 31), q11 = __shfl_sync(0xffffffffu, p1, p1 & 31);
+                        a0 |= p0 >= 32 ? b01 : b00;
+                        a1 |= p1 >= 32 ? b11 : b10;
+                        p0 = p0 >= 32 ? q01 : q00;
+                        p1 = p1 >= 32 ? q11 : q10;
+                    }
+                }
+                if (j0 < n) w.anc[(size_t)i * N + j0] = a0;
+                if (j1 < n) w.anc[(size_t)i * N + j1] = a1;
+            }
+        }
+        if (lane == 0) {
+            if (bad) { war_set_device_status(status_word, WAR_ERR_BAD_TREE); n = 0; }
+            int tiles = 0;
+            if (n > 0) {
+                const long long L = (long long)pl + n;
+                if ((L + page_size - 1) / page_size > max_pages) { war_set_device_status(status_word, WAR_ERR_BAD_PAGE); n = 0; }
+                else tiles = (int)((L + kTileKeys - 1) / kTileKeys);
+            }
+            s_tiles[i] = tiles;
+            s_n[i] = (uint8_t)n;
+        }
+    }
+    __syncthreads();
+
+    // ---- per request, one thread: weights, order, chunk counts ----
     int r_n[kPer], r_tiles[kPer], r_rbs[kPer], r_pos[kPer], r_nc[kPer];
-    // per request: validate, ancestor masks, tile count
     long long my_tiles = 0;
 #pragma unroll
     for (int k = 0; k < kPer; ++k) {
         const int i = tid + k * 1024;
         r_n[k] = 0; r_tiles[k] = 0; r_rbs[k] = 0; r_pos[k] = 0; r_nc[k] = 0;
         if (i >= B) continue;
-        int n = num_nodes[i];
-        const int pl = prefix_len[i];
-        bool bad = n < 0 || n > N || pl < 0;
-        if (!bad && n > 0) {
-            // all parent ids of the request are requested before any is used, so their latencies overlap
-            int pbuf[64];
-            const int4* prow = reinterpret_cast<const int4*>(parent + (size_t)i * N);
-            if ((N & 3) == 0 && (reinterpret_cast<uintptr_t>(parent) & 15) == 0) {
-                for (int j = 0; j < n; j += 4) {
-                    const int4 v = prow[j >> 2];
-                    pbuf[j] = v.x; pbuf[j + 1] = v.y; pbuf[j + 2] = v.z; pbuf[j + 3] = v.w;
-                }
-            } else {
-                for (int j = 0; j < n; ++j) pbuf[j] = parent[(size_t)i * N + j];
-            }
-            uint64_t local[64];
-            local[0] = 1ull;
-            for (int j = 1; j < n; ++j) {
-                const int p = pbuf[j];
-                if (p < 0 || p >= j) { bad = true; break; }
-                local[j] = local[p] | (1ull << j);
-            }
-            if (!bad)
-                for (int j = 0; j < n; ++j) w.anc[(size_t)i * N + j] = local[j];
-        }
-        if (bad) { war_set_device_status(status_word, WAR_ERR_BAD_TREE); n = 0; }
-        int tiles = 0;
-        if (n > 0) {
-            const long long L = (long long)pl + n;
-            if ((L + page_size - 1) / page_size > max_pages) { war_set_device_status(status_word, WAR_ERR_BAD_PAGE); n = 0; }
-            else tiles = (int)((L + kTileKeys - 1) / kTileKeys);
-        }
-        s_tiles[i] = tiles;
-        r_n[k] = n; r_tiles[k] = tiles;
-        r_rbs[k] = n > 0 ? (G * n + kRowBlock - 1) / kRowBlock : 0;
-        my_tiles += (long long)tiles * r_rbs[k];
+        r_n[k] = s_n[i]; r_tiles[k] = s_tiles[i];
+        r_rbs[k] = r_n[k] > 0 ? (G * r_n[k] + kRowBlock - 1) / kRowBlock : 0;
+        my_tiles += (long long)r_tiles[k] * r_rbs[k];
     }
     // block sum of tiles (weighted by row blocks and kv heads)
     for (int o = 16; o > 0; o >>= 1) my_tiles += __shfl_xor_sync(0xffffffffu, my_tiles, o);
-    if ((tid & 31) == 0) s_sum[tid >> 5] = my_tiles;
+    if (lane == 0) s_sum[warp] = my_tiles;
     __syncthreads();
     if (tid == 0) {
         long long tot = 0;
@@ -99,6 +129,7 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         r_pos[k] = pos;
         r_nc[k] = t > 0 ? (t + chunk_tiles - 1) / chunk_tiles : 0;
         s_units[pos] = r_nc[k] * Hkv * r_rbs[k];
+        s_order[pos] = (uint16_t)i;
     }
     __syncthreads();
     // exclusive scan of s_units: per-thread serial segments + warp scans
@@ -108,40 +139,49 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         int sum = 0;
         for (int q = b0; q < b1; ++q) sum += s_units[q];
         int incl = sum;
-        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if ((tid & 31) >= o) incl += y; }
-        if ((tid & 31) == 31) s_red[tid >> 5] = incl;
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+        if (lane == 31) s_red[warp] = incl;
         __syncthreads();
         if (tid < 32) {
             int x = s_red[tid], xi = x;
             for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, xi, o); if (tid >= o) xi += y; }
             s_red[tid] = xi - x;
-            if (tid == 31) w.counters[1] = xi;     // total number of units
+            if (tid == 31) { w.counters[1] = xi; s_total = xi; }     // total number of units
         }
         __syncthreads();
-        int run = s_red[tid >> 5] + incl - sum;
+        int run = s_red[warp] + incl - sum;
         for (int q = b0; q < b1; ++q) { const int u = s_units[q]; s_units[q] = run; run += u; }
     }
     __syncthreads();
-    // unit table: per request, chunks balanced to within one tile, order (chunk, kv head, row block)
 #pragma unroll
     for (int k = 0; k < kPer; ++k) {
         const int i = tid + k * 1024;
         if (i >= B) continue;
-        const int base = s_units[r_pos[k]];
-        const int nc = r_nc[k], t = r_tiles[k], rbs = r_rbs[k];
         AttnReq rq;
-        rq.base_unit = base; rq.n_chunks = nc; rq.n_tiles = t; rq.n_nodes = r_n[k];
+        rq.base_unit = s_units[r_pos[k]]; rq.n_chunks = r_nc[k]; rq.n_tiles = r_tiles[k]; rq.n_nodes = r_n[k];
         w.req[i] = rq;
-        int u = base;
-        for (int c = 0; c < nc; ++c) {
-            const int tb = (int)((long long)t * c / nc), te = (int)((long long)t * (c + 1) / nc);
-            for (int h = 0; h < Hkv; ++h)
-                for (int rb = 0; rb < rbs; ++rb, ++u) {
-                    AttnUnit x;
-                    x.req = i; x.kvh = h; x.rb = rb; x.tile_begin = tb; x.tile_end = te; x.n_chunks = nc; x.chunk = c; x.pad = 0;
-                    w.units[u] = x;
-                }
+    }
+    // ---- unit table, one thread per unit: per request, chunks balanced to within one tile, order (chunk, kv head,
+    // row block).  Requests with units come first in the order and their offsets increase strictly, so the request of
+    // unit u is the last position whose offset is <= u.
+    const int total = s_total;
+    for (int u = tid; u < total; u += 1024) {
+        int lo = 0, hi = B - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (s_units[mid] <= u) lo = mid; else hi = mid - 1;
         }
+        const int i = s_order[lo];
+        const int t = s_tiles[i], n = s_n[i];
+        const int rbs = (G * n + kRowBlock - 1) / kRowBlock;
+        const int nc = (t + chunk_tiles - 1) / chunk_tiles;
+        const int local = u - s_units[lo];
+        const int c = local / (Hkv * rbs), rem = local % (Hkv * rbs);
+        AttnUnit x;
+        x.req = i; x.kvh = rem / rbs; x.rb = rem % rbs;
+        x.tile_begin = (int)((long long)t * c / nc); x.tile_end = (int)((long long)t * (c + 1) / nc);
+        x.n_chunks = nc; x.chunk = c; x.pad = 0;
+        w.units[u] = x;
     }
 }
 
