@@ -321,6 +321,19 @@ def main():
     barrier()
     e2e_ms = 1e3 * (time.perf_counter() - t0)
 
+    # ---- commit (the accepted tokens become context), timed on its own: it is what a caller runs between two
+    # steps, not part of the step metric.  Run last: it moves K/V rows of the resident cache.
+    c_pl, c_tails, c_tl = attn.prefix_len.clone(), d_tails.clone(), d_tl.clone()
+    war.war_commit(d_ids, d_alen, d_path, d_bonus, attn.k_pool, attn.v_pool, attn.page_table, c_pl, c_tails, c_tl)
+    c_pl.copy_(attn.prefix_len); c_tails.copy_(d_tails); c_tl.copy_(d_tl)
+    c0, c1 = ev(), ev()
+    torch.cuda.synchronize()
+    c0.record()
+    war.war_commit(d_ids, d_alen, d_path, d_bonus, attn.k_pool, attn.v_pool, attn.page_table, c_pl, c_tails, c_tl)
+    c1.record()
+    torch.cuda.synchronize()
+    commit_ms = c0.elapsed_time(c1)
+
     # ---- max over ranks, totals over ranks ----
     agg = torch.tensor([total_ms, e2e_ms, attn_ms], dtype=torch.float64, device=dev)
     tot = torch.tensor([verified, slots], dtype=torch.float64, device=dev)
@@ -379,6 +392,7 @@ def main():
             "roofline_kernel": {"name": "war_verify_attn (plan + attention + combine launches)", "bytes_per_launch": kvb,
                                 "ms_per_launch": attn_ms},
             "breakdown_ms": {"draft": draft_ms, "verify_attn": attn_ms, "accept": accept_ms},
+            "commit_ms": commit_ms,
             "step_ms": {"median": float(np.median(per_step)), "min": float(per_step.min()), "max": float(per_step.max())},
             "slots_verified_per_s": slots_all / (ms_per_step * 1e-3),
             "accept_len_mean": float(h_alen.mean()), "index_build_s": index_build_s, "index_tokens": int(len(tok)),

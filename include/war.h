@@ -12,6 +12,7 @@
  *   war_draft                            longest-suffix match + frequency-ranked draft token tree
  *   war_verify_attn                      tree-masked GQA decode attention over a paged bf16 KV cache
  *   war_accept                           longest root path of the tree that equals the target's tokens
+ *   war_commit                           the accepted tokens become context: KV rows, prefix length, tail window
  *
  * Conventions shared by every call
  *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller owns every buffer it
@@ -183,6 +184,38 @@ war_status_t war_verify_attn_noalloc(const void* d_q, const void* d_kpool, const
 war_status_t war_accept(const int32_t* d_ids, const int32_t* d_parent, const int32_t* d_num_nodes,
                         const int32_t* d_target_ids, int32_t B, int32_t N, int32_t target_mode,
                         int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, war_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Commit (completes the step of paper Section 3.2: the rollout advances "by multiple tokens in a single forward
+ * pass when the drafts are accepted"; the paper does not spell the bookkeeping out).  After war_accept, makes the
+ * accepted path the end of each request's context, so that the next war_draft / war_verify_attn can run on the
+ * same buffers:
+ *   KV cache    the K/V rows of the accepted slots (logical positions prefix_len + slot) move to positions
+ *               prefix_len + 1 .. prefix_len + accept_len, in path order, inside the paged pool; no page is
+ *               allocated or freed and rows of rejected slots are left as they are (dead)
+ *   context     context' = context ++ ids[path[0]] .. ids[path[accept_len-1]] ++ bonus (when bonus >= 0)
+ *   d_tail      [B, P] in/out, right-aligned: the last min(P, length) tokens of context'; entries left of the
+ *               window are set to 0.  d_tail_len [B] in/out.
+ *   d_prefix_len[B] in/out: the last token of context' is the next root.  bonus >= 0: += accept_len + 1 (the new
+ *               root's K/V does not exist yet); bonus < 0 (per-node targets): += accept_len (the last accepted
+ *               token, or the old root, stays the root).
+ * d_accept_path [B, N] as written by war_accept (slots strictly increasing).  Pools: bf16, D = 128, strides in
+ * elements as in war_attn_params_t with unit stride along d and the others multiples of 8 (rows are moved 16
+ * bytes at a time); both pools are modified in place.
+ * A request whose path is malformed or whose rows lie beyond max_pages_per_req is left untouched and
+ * WAR_ERR_BAD_TREE is recorded in the device status word; a page id outside [0, num_pages) records
+ * WAR_ERR_BAD_PAGE and that row is skipped.  Enqueues two kernels on `stream`; does not synchronise.
+ * ------------------------------------------------------------------------------------------------ */
+typedef struct {
+    int32_t B, N, P;                 /* requests, slots per tree, tail window */
+    int32_t Hkv, D, page_size, max_pages_per_req, reserved;
+    int64_t num_pages;
+    int64_t k_strides[4], v_strides[4];   /* [page, head, token, d] in elements */
+} war_commit_params_t;
+war_status_t war_commit(const int32_t* d_ids, const int32_t* d_accept_len, const int32_t* d_accept_path,
+                        const int32_t* d_bonus, void* d_kpool, void* d_vpool, const int32_t* d_page_table,
+                        const war_commit_params_t* params, int32_t* d_prefix_len, int32_t* d_tail,
+                        int32_t* d_tail_len, war_stream_t stream);
 
 /* Reads and clears the sticky device status word (synchronises `stream`).  *h_status receives a
  * war_status_t value: WAR_OK, or the first device-side problem seen since the last read. */

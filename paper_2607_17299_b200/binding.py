@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "WAR_OK", 1: "WAR_ERR_INVALID_ARG", 2: "WAR_ERR_OOM", 3: "WAR
                 5: "WAR_ERR_TIMEOUT", 6: "WAR_ERR_UNSUPPORTED", 7: "WAR_ERR_BAD_TREE", 8: "WAR_ERR_BAD_PAGE"}
 
 EXPORTS = ["war_index_build", "war_index_append", "war_index_info", "war_index_destroy", "war_draft",
-           "war_verify_attn_workspace_bytes", "war_verify_attn", "war_verify_attn_noalloc", "war_accept", "war_device_status",
+           "war_verify_attn_workspace_bytes", "war_verify_attn", "war_verify_attn_noalloc", "war_accept", "war_commit", "war_device_status",
            "war_status_string"]
 
 
@@ -227,6 +227,35 @@ def war_accept(d_ids: torch.Tensor, d_parent: torch.Tensor, d_num_nodes: torch.T
                            _ptr(d_target_ids, torch.int32), B, N, target_mode, _ptr(d_accept_len, torch.int32),
                            _ptr(d_accept_path, torch.int32), _ptr(d_bonus, torch.int32), _stream())
     _check("war_accept", code)
+
+
+class CommitParams(C.Structure):
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("P", C.c_int32), ("Hkv", C.c_int32), ("D", C.c_int32),
+                ("page_size", C.c_int32), ("max_pages_per_req", C.c_int32), ("reserved", C.c_int32),
+                ("num_pages", C.c_int64), ("k_strides", C.c_int64 * 4), ("v_strides", C.c_int64 * 4)]
+
+
+_lib.war_commit.restype = C.c_int
+_lib.war_commit.argtypes = [C.c_void_p] * 7 + [C.POINTER(CommitParams)] + [C.c_void_p] * 4
+
+
+def war_commit(d_ids: torch.Tensor, d_accept_len: torch.Tensor, d_accept_path: torch.Tensor, d_bonus: torch.Tensor,
+               k_pool: torch.Tensor, v_pool: torch.Tensor, page_table: torch.Tensor, d_prefix_len: torch.Tensor,
+               d_tail: torch.Tensor, d_tail_len: torch.Tensor) -> None:
+    """Pools are [pages, Hkv, page_size, D] bf16 views (any strides the library accepts); updated in place."""
+    B, N = d_ids.shape
+    p = CommitParams()
+    p.B, p.N, p.P = B, N, d_tail.shape[1]
+    p.Hkv, p.D, p.page_size = k_pool.shape[1], k_pool.shape[3], k_pool.shape[2]
+    p.max_pages_per_req, p.num_pages = page_table.shape[1], k_pool.shape[0]
+    for i in range(4):
+        p.k_strides[i] = k_pool.stride(i)
+        p.v_strides[i] = v_pool.stride(i)
+    code = _lib.war_commit(_ptr(d_ids, torch.int32), _ptr(d_accept_len, torch.int32), _ptr(d_accept_path, torch.int32),
+                           _ptr(d_bonus, torch.int32), C.c_void_p(k_pool.data_ptr()), C.c_void_p(v_pool.data_ptr()),
+                           _ptr(page_table, torch.int32), C.byref(p), _ptr(d_prefix_len, torch.int32),
+                           _ptr(d_tail, torch.int32), _ptr(d_tail_len, torch.int32), _stream())
+    _check("war_commit", code)
 
 
 def war_device_status() -> int:
