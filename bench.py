@@ -135,6 +135,9 @@ def main():
     ap.add_argument("--flush-l2", action="store_true",
                     help="write a 256 MB scratch buffer before every timed step (for workloads whose KV cache fits L2); "
                          "ms_per_step is then the mean of the per-step event intervals, the flush excluded")
+    ap.add_argument("--spec-batch-limit", type=int, default=0,
+                    help="workload-aware switch of war_draft: above this many running requests the step is a plain decode "
+                         "step (root-only trees); 0 = always speculate")
     ap.add_argument("--requests", type=int, default=0,
                     help="run the workload's recipe with this many requests instead of its own count (profiling-size cases)")
     args = ap.parse_args()
@@ -240,7 +243,7 @@ def main():
     ws = war.new_workspace(params, dev)
 
     # targets depend on the trees; the trees are a deterministic function of the inputs, so draft once to make them
-    war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt)
+    war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt, args.spec_batch_limit)
     torch.cuda.synchronize()
     h_ids, h_par, h_nn = d_ids.cpu().numpy(), d_par.cpu().numpy(), d_nn.cpu().numpy()
     targets = W.make_targets(cfg, h_ids, h_par, h_nn, 0)
@@ -249,7 +252,7 @@ def main():
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
     def step(attn_events=None):
-        war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt)
+        war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt, args.spec_batch_limit)
         if attn_events is not None:
             attn_events[0].record()
         war.war_verify_attn(attn.q, attn.k_pool, attn.v_pool, attn.page_table, attn.prefix_len, d_nn, d_par, params, ws,
@@ -377,7 +380,8 @@ def main():
             "metric": METRIC, "value": verified_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": dict(base_config, kernel="tcgen05" if args.kernel == 0 else "cuda-core"),
+            "config": dict(base_config, kernel="tcgen05" if args.kernel == 0 else "cuda-core",
+                           **({"spec_batch_limit": args.spec_batch_limit} if args.spec_batch_limit else {})),
             "clocks": clocks.summary(),
             "e2e": {"value": verified_all / (e2e_ms / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},

@@ -105,9 +105,18 @@ war_status_t war_index_destroy(war_index_t* ix);
  * entries are read.  Tail tokens outside [0, vocab) never match.
  * Outputs: d_match_len [B], d_num_nodes [B], d_ids / d_parent / d_count [B, N] (d_count may be NULL).
  * Unused slots are written as ids = -1, parent = -1, count = 0.
+ * Workload-aware switch (paper Section 3.2, "adaptive enabling and disabling" of speculation "according to the
+ * current batch size", with "stateless mode switching"; Section 5.3: beyond a batch of about 16 speculation
+ * costs more than it gains).  A request with tail_len[b] < 0 is not running: num_nodes = 0, match_len = 0.  The
+ * effective batch size is the number of running requests, counted on the device in this call.  When
+ * spec_batch_limit > 0 and the effective batch size exceeds it, nothing is looked up and every running request
+ * gets the root alone (num_nodes = 1, match_len = 0, count = 0), so the step that follows is a plain decode step
+ * through the same calls: no state is kept between calls and one captured CUDA graph serves both modes.
+ * spec_batch_limit = 0 always speculates.
  * ------------------------------------------------------------------------------------------------ */
 typedef struct {
     int32_t B, P, N, topk, min_match;
+    int32_t spec_batch_limit;
 } war_draft_params_t;
 war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, const int32_t* d_tail_len,
                        const war_draft_params_t* params,

@@ -171,15 +171,28 @@ def build_draft_tree(corpus: Corpus, tail: np.ndarray, match_len: int, ends: np.
     return np.array(ids, np.int32), np.array(parent, np.int32), np.array(count, np.int32)
 
 
-def draft_batch(corpus: Corpus, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, min_match: int = 1):
-    """Batched form with the library's output convention: unused slots hold ids = -1, parent = -1, count = 0."""
+def draft_batch(corpus: Corpus, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, min_match: int = 1,
+                spec_batch_limit: int = 0):
+    """Batched form with the library's output convention: unused slots hold ids = -1, parent = -1, count = 0.
+
+    Workload-aware switch (paper, Section 3.2, "adaptive enabling and disabling" by the current batch size, and
+    Section 5.3: beyond a batch of about 16 speculation costs more than it gains): a request with
+    tail_len < 0 is not running (no tree at all); the effective batch size is the number of running requests;
+    when spec_batch_limit > 0 and the effective batch size exceeds it, nothing is looked up and every running
+    request gets the root alone (match_len 0, count 0), which makes the step a plain decode step."""
     B = tails.shape[0]
     match_len = np.zeros(B, np.int32)
     num_nodes = np.zeros(B, np.int32)
     ids = np.full((B, N), -1, np.int32)
     parent = np.full((B, N), -1, np.int32)
     count = np.zeros((B, N), np.int32)
-    for i in range(B):
+    running = [i for i in range(B) if int(tail_len[i]) >= 0]
+    plain = spec_batch_limit > 0 and len(running) > spec_batch_limit
+    for i in running:
+        if plain:
+            num_nodes[i] = 1
+            ids[i, 0] = tails[i, -1]
+            continue
         ml, ends = longest_suffix_match(corpus, tails[i], int(tail_len[i]))
         a, b, c = build_draft_tree(corpus, tails[i], ml, ends, N, k, min_match)
         n = len(a)

@@ -217,6 +217,7 @@ struct Shared {
     int st_cnt[32], st_start[32];               // runs that cross span edges (one per span) and the closing run
     int fin_cnt[kMaxK], fin_start[kMaxK], fin_tok[kMaxK];
     int mode, cur, lo, cnt, depth, n_nodes, pool_n, thr_shared, long_runs_only, full_lo, full_cnt;
+    int n_running;
 };
 
 // Tokens from index `from` on of the suffix at s against the pattern; returns the sign and, in `matched`, how many
@@ -258,7 +259,7 @@ __device__ __forceinline__ int compare_suffix(const int32_t* __restrict__ corpus
 __global__ void __launch_bounds__(kThreads, 2)
 war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, const uint8_t* __restrict__ lcp,
                  const int32_t* __restrict__ bucket, int vocab, const int32_t* __restrict__ tail,
-                 const int32_t* __restrict__ tail_len, int P, int N, int K, int min_match,
+                 const int32_t* __restrict__ tail_len, int B, int P, int N, int K, int min_match, int spec_batch_limit,
                  int32_t* __restrict__ match_len, int32_t* __restrict__ num_nodes, int32_t* __restrict__ ids,
                  int32_t* __restrict__ parent, int32_t* __restrict__ count) {
     __shared__ Shared sh;
@@ -269,7 +270,35 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
     int32_t* o_cnt = count ? count + (size_t)b * N : nullptr;
 
     if (tid < P) sh.pat[tid] = tail[(size_t)b * P + tid];
+    // Workload-aware switch: a request with tail_len < 0 is not running; when more requests run than the limit,
+    // nothing is looked up and every running request gets the root alone (a plain decode step through the same
+    // calls).  Every CTA counts the running requests itself: no extra launch, no state between calls.
+    bool plain = false;
+    if (spec_batch_limit > 0) {
+        int c = 0;
+        for (int i = tid; i < B; i += kThreads) c += tail_len[i] >= 0;
+        if (tid == 0) sh.n_running = 0;
+        __syncthreads();
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+        if (lane == 0 && c) atomicAdd(&sh.n_running, c);
+        __syncthreads();
+        plain = sh.n_running > spec_batch_limit;
+    }
     __syncthreads();
+    const int my_tl = tail_len[b];
+    if (my_tl < 0 || plain) {
+        const int n = my_tl < 0 ? 0 : 1;
+        if (tid == 0) {
+            match_len[b] = 0; num_nodes[b] = n;
+            if (n) { o_ids[0] = sh.pat[P - 1]; o_par[0] = -1; if (o_cnt) o_cnt[0] = 0; }
+        }
+        for (int j = n + tid; j < N; j += kThreads) {
+            o_ids[j] = -1; o_par[j] = -1;
+            if (o_cnt) o_cnt[j] = 0;
+        }
+        return;
+    }
 
     // Publishes the next node to expand: its token range (the interval minus the suffixes that end at this depth).
     auto publish = [&](int slot, int lo, int cnt, int depth) {          // warp 0, all lanes
@@ -561,14 +590,15 @@ extern "C" war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, 
                                   const war_draft_params_t* p, int32_t* d_match_len, int32_t* d_num_nodes,
                                   int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream) {
     if (!ix || !p) return WAR_ERR_INVALID_ARG;
-    if (p->B < 0 || p->P < 1 || p->P > kMaxP || p->N < 1 || p->N > kMaxN || p->topk < 1 || p->topk > kMaxK || p->min_match < 0)
+    if (p->B < 0 || p->P < 1 || p->P > kMaxP || p->N < 1 || p->N > kMaxN || p->topk < 1 || p->topk > kMaxK || p->min_match < 0 ||
+        p->spec_batch_limit < 0)
         return WAR_ERR_INVALID_ARG;
     if (p->P + p->N > ix->max_depth) return WAR_ERR_INVALID_ARG;     // the index is not ordered deep enough
     if (p->B == 0) return WAR_OK;
     if (!d_tail || !d_tail_len || !d_match_len || !d_num_nodes || !d_ids || !d_parent) return WAR_ERR_INVALID_ARG;
     war_draft_kernel<<<p->B, kThreads, 0, stream>>>(ix->corpus, ix->sa, ix->lcp, ix->bucket, ix->vocab, d_tail, d_tail_len,
-                                                   p->P, p->N, p->topk, p->min_match, d_match_len, d_num_nodes, d_ids,
-                                                   d_parent, d_count);
+                                                   p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, d_match_len,
+                                                   d_num_nodes, d_ids, d_parent, d_count);
     WAR_LAUNCH_CHECK();
     return WAR_OK;
 }

@@ -72,3 +72,60 @@ def test_step_replays_from_a_cuda_graph(war):
     assert not torch.equal(replayed[2], eager[2])
     assert war.war_device_status() == 0
     ix.destroy()
+
+
+def test_one_graph_serves_speculative_and_plain_steps(war):
+    """Workload-aware switch inside a captured step (paper Section 3.2: adaptive enabling by batch size, stateless
+    switching, CUDA-graph compatibility): the number of running requests is read on the device, so the same graph
+    speculates while few requests run and does plain decode steps (root-only trees) when many do."""
+    from oracle import draft_oracle as D
+    dev = torch.device("cuda:0")
+    cfg = W.scaled(W.CONFIGS["tiny"], B=12, N=16)
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(cfg)
+    corpus = D.Corpus(tok, off)
+    ix = U.build_index(war, tok, off, cfg.vocab, max_depth=cfg.P + cfg.N)
+    a = W.make_attention_inputs(cfg, W.context_lengths(cfg)[:cfg.B] // 4 + 100, device=dev)
+    B, N, limit = cfg.B, cfg.N, 8
+    i32 = dict(dtype=torch.int32, device=dev)
+    d_tails, d_tl = torch.from_numpy(tails).to(dev), torch.from_numpy(tl).to(dev)
+    ml, nn = torch.zeros(B, **i32), torch.zeros(B, **i32)
+    ids, par, cnt = torch.zeros((B, N), **i32), torch.zeros((B, N), **i32), torch.zeros((B, N), **i32)
+    alen, path, bonus = torch.zeros(B, **i32), torch.zeros((B, N), **i32), torch.zeros(B, **i32)
+    target = torch.randint(0, cfg.vocab, (B, N), dtype=torch.int32, device=dev)
+    out = torch.zeros_like(a.q)
+    params = war.attn_params(a.q, a.k_pool, a.v_pool, a.page_table, 1.0 / np.sqrt(cfg.D), 0)
+    ws = war.new_workspace(params, dev)
+
+    def step():
+        war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, ml, nn, ids, par, cnt, limit)
+        war.war_verify_attn(a.q, a.k_pool, a.v_pool, a.page_table, a.prefix_len, nn, par, params, ws, out, None)
+        war.war_accept(ids, par, nn, target, 0, alen, path, bonus)
+
+    step()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    with torch.cuda.graph(g):
+        step()
+    for running in (12, 8, 3, 9):                                     # above, at, below, above the limit again
+        h_tl = tl.copy(); h_tl[running:] = -1
+        d_tl.copy_(torch.from_numpy(h_tl).to(dev))
+        out.fill_(7.0)
+        g.replay()
+        torch.cuda.synchronize()
+        want = D.draft_batch(corpus, tails, h_tl, N, cfg.topk, spec_batch_limit=limit)
+        for got, w in zip((ml, nn, ids, par, cnt), want):
+            assert np.array_equal(got.cpu().numpy(), w), running
+        h_nn = nn.cpu().numpy()
+        assert (h_nn.max() > 1) == (running <= limit)
+        assert (alen.cpu().numpy()[h_nn <= 1] == 0).all()
+        o = out.float().cpu().numpy()
+        for i in range(B):                                             # rows beyond num_nodes are never written
+            assert (o[i, h_nn[i]:] == 7.0).all() and (h_nn[i] == 0 or (o[i, 0] != 7.0).any())
+    assert war.war_device_status() == 0
+    ix.destroy()

@@ -242,3 +242,21 @@ def test_empty_and_degenerate_inputs(war):
     ml, nn, ids, par, cnt = U.run_draft(war, ix, tails, np.array([4]), 8, 4)
     assert ml[0] == 4 and nn[0] == 2 and ids[0, :2].tolist() == [4, 5]
     ix.destroy()
+
+
+def test_workload_aware_switch(war):
+    """Requests with tail_len < 0 are not running; above the limit every running request gets the root alone."""
+    cfg = W.scaled(W.CONFIGS["tiny"], B=24)
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(cfg)
+    tl = tl.copy(); tl[[3, 11, 17]] = -1                               # 21 running
+    corpus = D.Corpus(tok, off)
+    ix = U.build_index(war, tok, off, cfg.vocab, max_depth=cfg.P + cfg.N)
+    for limit in (0, 21, 20, 1):
+        got = U.run_draft(war, ix, tails, tl, cfg.N, cfg.topk, spec_batch_limit=limit)
+        want = D.draft_batch(corpus, tails, tl, cfg.N, cfg.topk, spec_batch_limit=limit)
+        for g, w in zip(got, want):
+            assert np.array_equal(g, w), limit
+        assert (got[1][[3, 11, 17]] == 0).all()
+        assert (got[1].max() > 1) == (limit in (0, 21))
+    ix.destroy()

@@ -218,3 +218,26 @@ def test_min_match_and_budget_edges():
     ids, parent, count = D.build_draft_tree(corpus, tail, ml, ends, 3, 1)
     assert ids.tolist() == [2, 3, 1] and parent.tolist() == [-1, 0, 1]   # k=1: chain along the smaller id on ties
     assert D.longest_suffix_match(corpus, tail, 0)[0] == 0
+
+
+def test_workload_aware_switch():
+    """Effective batch size = running requests (tail_len >= 0).  At or below the limit nothing changes; above it
+    every running request gets the root alone; a request that is not running gets no tree in either mode."""
+    rng = np.random.default_rng(3)
+    toks = [rng.integers(0, 6, 40).astype(np.int32) for _ in range(5)]
+    off = np.concatenate([[0], np.cumsum([len(t) for t in toks])]).astype(np.int64)
+    corpus = D.Corpus(np.concatenate(toks), off)
+    B, P, N = 6, 4, 5
+    tails = rng.integers(0, 6, (B, P)).astype(np.int32)
+    tl = np.array([4, 4, -1, 2, 0, 4], np.int32)                      # request 2 is not running: 5 running
+    base = D.draft_batch(corpus, tails, tl, N, 2)
+    for limit in (0, 5, 9):                                            # no limit, exactly at the limit, above
+        got = D.draft_batch(corpus, tails, tl, N, 2, spec_batch_limit=limit)
+        for g, w in zip(got, base):
+            assert np.array_equal(g, w)
+    assert base[1][2] == 0 and (base[2][2] == -1).all()                # not running: no slots
+    assert base[1].max() > 1                                           # the speculative mode does draft here
+    ml, nn, ids, par, cnt = D.draft_batch(corpus, tails, tl, N, 2, spec_batch_limit=4)
+    assert nn.tolist() == [1, 1, 0, 1, 1, 1] and (ml == 0).all() and (cnt == 0).all()
+    for i in (0, 1, 3, 4, 5):
+        assert ids[i, 0] == tails[i, -1] and par[i, 0] == -1 and (ids[i, 1:] == -1).all()
