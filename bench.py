@@ -219,8 +219,12 @@ def main():
     index_build_s = time.perf_counter() - t0
     # the index the steps use is then made the way a rollout would make it: all but the last trajectories first, the
     # rest appended as an RL step's worth of new trajectories (an appended index answers exactly like a fresh build)
-    ix.destroy()
     k_new = max(1, cfg.n_traj // 32)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    war.war_index_evict(ix, k_new)                         # sliding window: the oldest 1/32 of the trajectories leave
+    index_evict_s = time.perf_counter() - t0
+    ix.destroy()
     ix = war.war_index_build(d_tok, off[:cfg.n_traj - k_new + 1], cfg.vocab, cfg.P + cfg.N, len(tok) + cfg.n_traj)
     torch.cuda.synchronize()
     t0 = time.perf_counter()
@@ -401,6 +405,7 @@ def main():
             "slots_verified_per_s": slots_all / (ms_per_step * 1e-3),
             "accept_len_mean": float(h_alen.mean()), "index_build_s": index_build_s, "index_tokens": int(len(tok)),
             "index_append": {"trajectories": k_new, "tokens": index_append_tokens, "seconds": index_append_s},
+            "index_evict": {"trajectories": k_new, "seconds": index_evict_s},
             "device_status": status,
         }
         if not args.no_cpu_baseline and world == 1:

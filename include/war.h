@@ -75,6 +75,13 @@ war_status_t war_index_build(const int32_t* d_tokens, const int64_t* h_offsets, 
 war_status_t war_index_append(war_index_t* ix, const int32_t* d_tokens, const int64_t* h_offsets, int32_t T,
                               war_stream_t stream);
 
+/* Windowed cache (the paper keeps the cache's "memory overhead" modest, Section 3.2, without naming a policy; this
+ * is the simplest one): removes the n_oldest trajectories that were added first.  Afterwards every query answers
+ * exactly as a fresh build on the remaining trajectories would.  The suffix array is filtered, not sorted again
+ * (the remaining suffixes keep their order); LCP and buckets are recomputed.  Synchronises `stream`; allocates
+ * and frees scratch of 4 bytes per stored token.  n_oldest must be in [0, T]. */
+war_status_t war_index_evict(war_index_t* ix, int32_t n_oldest, war_stream_t stream);
+
 typedef struct {
     int64_t M;                  /* corpus entries in use: tokens + one separator per trajectory */
     int64_t capacity_tokens;

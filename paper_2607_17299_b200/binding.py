@@ -25,7 +25,7 @@ WAR_OK = 0
 STATUS_NAMES = {0: "WAR_OK", 1: "WAR_ERR_INVALID_ARG", 2: "WAR_ERR_OOM", 3: "WAR_ERR_CAPACITY", 4: "WAR_ERR_CUDA",
                 5: "WAR_ERR_TIMEOUT", 6: "WAR_ERR_UNSUPPORTED", 7: "WAR_ERR_BAD_TREE", 8: "WAR_ERR_BAD_PAGE"}
 
-EXPORTS = ["war_index_build", "war_index_append", "war_index_info", "war_index_destroy", "war_draft",
+EXPORTS = ["war_index_build", "war_index_append", "war_index_evict", "war_index_info", "war_index_destroy", "war_draft",
            "war_verify_attn_workspace_bytes", "war_verify_attn", "war_verify_attn_noalloc", "war_accept", "war_commit", "war_device_status",
            "war_status_string"]
 
@@ -61,6 +61,8 @@ _lib.war_index_build.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C
                                  C.POINTER(C.c_void_p)]
 _lib.war_index_append.restype = C.c_int
 _lib.war_index_append.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+_lib.war_index_evict.restype = C.c_int
+_lib.war_index_evict.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
 _lib.war_index_info.restype = C.c_int
 _lib.war_index_info.argtypes = [C.c_void_p, C.POINTER(IndexInfo)]
 _lib.war_index_destroy.restype = C.c_int
@@ -146,6 +148,10 @@ def war_index_append(ix: Index, d_tokens: torch.Tensor, h_offsets) -> None:
     off = _offsets(h_offsets)
     _check("war_index_append", _lib.war_index_append(ix.handle, _ptr(d_tokens, torch.int32), off.ctypes.data,
                                                      len(off) - 1, _stream()))
+
+
+def war_index_evict(ix: Index, n_oldest: int) -> None:
+    _check("war_index_evict", _lib.war_index_evict(ix.handle, int(n_oldest), _stream()))
 
 
 def war_index_info(ix: Index) -> IndexInfo:

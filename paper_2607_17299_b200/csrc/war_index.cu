@@ -370,9 +370,70 @@ war_status_t add_trajectories(war_index* ix, const int32_t* d_tokens, const int6
     delete[] rel;
     if (e != cudaSuccess) { (void)cudaGetLastError(); return e == cudaErrorMemoryAllocation ? WAR_ERR_OOM : WAR_ERR_CUDA; }
     if (bad) return WAR_ERR_INVALID_ARG;                     // nothing was committed: M and T are unchanged
+    try {
+        for (int t = 1; t <= T; ++t) ix->bounds.push_back(ix->M + (h_offsets[t] - h_offsets[0]) + t);
+    } catch (...) {
+        ix->bounds.resize((size_t)ix->T + 1);
+        return WAR_ERR_OOM;
+    }
     ix->M += n_out;
     ix->T += T;
     return WAR_OK;
+}
+
+// ---- eviction of the oldest trajectories ----------------------------------------------------------
+// Suffixes of the remaining trajectories keep their relative order (separators isolate trajectories and keep their
+// own order when all of them are renumbered by the same amount), so the suffix array is filtered, not sorted again.
+struct KeepFrom {
+    int32_t cut;
+    __device__ __forceinline__ bool operator()(const int32_t& x) const { return x >= cut; }
+};
+
+__global__ void shift_sa_kernel(int32_t* __restrict__ sa, int64_t n, int32_t cut) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) sa[i] -= cut;
+}
+
+// dst[i] = src[cut + i], separators renumbered from -(1) again
+__global__ void shift_corpus_kernel(const int32_t* __restrict__ src, int64_t n, int64_t cut, int32_t n_evicted, int32_t* __restrict__ dst) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int32_t v = src[cut + i];
+    dst[i] = v < 0 ? v + n_evicted : v;
+}
+
+war_status_t evict_oldest(war_index* ix, int32_t n, cudaStream_t s) {
+    const int64_t cut = ix->bounds[(size_t)n], M_old = ix->M, M = M_old - cut;
+    if (M > 0) {
+        size_t temp_bytes = 0;
+        WAR_CUDA_TRY(cub::DeviceSelect::If(nullptr, temp_bytes, (int32_t*)nullptr, (int32_t*)nullptr, (int32_t*)nullptr, (int)M_old,
+                                           KeepFrom{(int32_t)cut}, s));
+        auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
+        Scratch scratch;
+        WAR_CUDA_TRY(cudaMalloc(&scratch.p, align(sizeof(int32_t) * M_old) + align(sizeof(int32_t)) + align(temp_bytes)));
+        int32_t* tmp = (int32_t*)scratch.p;
+        int32_t* d_n = (int32_t*)((char*)scratch.p + align(sizeof(int32_t) * M_old));
+        void* temp = (char*)d_n + align(sizeof(int32_t));
+        WAR_CUDA_TRY(cub::DeviceSelect::If(temp, temp_bytes, ix->sa, tmp, d_n, (int)M_old, KeepFrom{(int32_t)cut}, s));
+        WAR_CUDA_TRY(cudaMemcpyAsync(ix->sa, tmp, sizeof(int32_t) * M, cudaMemcpyDeviceToDevice, s));
+        shift_sa_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->sa, M, (int32_t)cut);
+        shift_corpus_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, M, cut, n, tmp);
+        WAR_CUDA_TRY(cudaMemcpyAsync(ix->corpus, tmp, sizeof(int32_t) * M, cudaMemcpyDeviceToDevice, s));
+        WAR_LAUNCH_CHECK();
+        WAR_CUDA_TRY(cudaStreamSynchronize(s));
+    }
+    // the vacated end reads as "no token" again (readable slack behind the last separator)
+    WAR_CUDA_TRY(cudaMemsetAsync(ix->corpus + M, 0xff, sizeof(int32_t) * (size_t)(M_old - M), s));
+    ix->bounds.erase(ix->bounds.begin(), ix->bounds.begin() + n);
+    for (auto& b : ix->bounds) b -= cut;
+    ix->M = M;
+    ix->T -= n;
+    if (M == 0) {
+        WAR_CUDA_TRY(cudaMemsetAsync(ix->bucket, 0, sizeof(int32_t) * (ix->vocab + 1), s));
+        WAR_CUDA_TRY(cudaStreamSynchronize(s));
+        return WAR_OK;
+    }
+    return finish_index(ix, s);
 }
 
 }  // namespace
@@ -423,6 +484,12 @@ extern "C" war_status_t war_index_append(war_index_t* ix, const int32_t* d_token
     // merging pays when the addition is the smaller part; otherwise sort everything again
     if (M_old > 0 && ix->M - M_old < M_old) return merge_new_suffixes(ix, M_old, stream);
     return rebuild(ix, stream);
+}
+
+extern "C" war_status_t war_index_evict(war_index_t* ix, int32_t n_oldest, war_stream_t stream) {
+    if (!ix || n_oldest < 0 || n_oldest > ix->T) return WAR_ERR_INVALID_ARG;
+    if (n_oldest == 0) return WAR_OK;
+    return evict_oldest(ix, n_oldest, stream);
 }
 
 extern "C" war_status_t war_index_info(const war_index_t* ix, war_index_info_t* out) {

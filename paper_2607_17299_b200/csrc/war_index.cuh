@@ -1,6 +1,7 @@
 // The index object behind war_index_t (library-internal).
 #pragma once
 #include <stdint.h>
+#include <vector>
 
 struct war_index {
     int32_t* corpus = nullptr;   // [capacity + slack] trajectories joined by unique negative separators
@@ -13,4 +14,5 @@ struct war_index {
     int32_t vocab = 0;
     int32_t max_depth = 0;
     int device = 0;
+    std::vector<int64_t> bounds{0};   // host: corpus position where each stored trajectory starts, then M
 };

@@ -52,11 +52,27 @@ def gather_trajectories(tokens: np.ndarray, offsets: np.ndarray, device: torch.d
     return out_tok, out_off
 
 
+def window_eviction(stored: int, incoming: int, window: int) -> int:
+    """How many of the oldest stored trajectories must go so that stored + incoming <= window (a sliding window
+    over the trajectory stream; every rank computes the same number because it appends the same trajectories)."""
+    if window <= 0:
+        return 0
+    return max(0, min(stored, stored + incoming - window))
+
+
 def append_step_trajectories(ix, tokens: np.ndarray, offsets: np.ndarray, device: torch.device,
-                             group: Optional[dist.ProcessGroup] = None) -> Tuple[np.ndarray, np.ndarray]:
-    """End-of-step synchronisation on a GPU rank: gather everybody's new trajectories, append them to this rank's index."""
+                             group: Optional[dist.ProcessGroup] = None, window: int = 0) -> Tuple[np.ndarray, np.ndarray]:
+    """End-of-step synchronisation on a GPU rank: gather everybody's new trajectories and append them to this rank's
+    index; with `window` > 0 the oldest trajectories are evicted first so that at most `window` stay stored."""
     from . import binding as war
     all_tok, all_off = gather_trajectories(tokens, offsets, device, group)
-    if len(all_off) > 1:
-        war.war_index_append(ix, torch.from_numpy(all_tok).to(device), all_off)
+    n_new = len(all_off) - 1
+    if n_new > 0:
+        if window > 0:
+            n_new_kept = min(n_new, window)                       # more new ones than the window holds: keep the latest
+            all_tok, all_off = all_tok[all_off[n_new - n_new_kept]:], all_off[n_new - n_new_kept:] - all_off[n_new - n_new_kept]
+            n_evict = window_eviction(int(war.war_index_info(ix).T), n_new_kept, window)
+            if n_evict:
+                war.war_index_evict(ix, n_evict)
+        war.war_index_append(ix, torch.from_numpy(np.ascontiguousarray(all_tok)).to(device), all_off)
     return all_tok, all_off

@@ -260,3 +260,60 @@ def test_workload_aware_switch(war):
         assert (got[1][[3, 11, 17]] == 0).all()
         assert (got[1].max() > 1) == (limit in (0, 21))
     ix.destroy()
+
+
+@pytest.mark.parametrize("seed", range(2))
+def test_evicting_the_oldest_trajectories_equals_a_fresh_build(war, seed):
+    """A sliding window over the trajectory stream: append, evict the oldest, append again.  After every change the
+    suffix array must be a depth-ordered permutation of what is stored, with exact LCP and buckets and separators
+    numbered from the first stored trajectory, and drafts must equal the brute-force checker's on the window."""
+    rng = np.random.default_rng(70 + seed)
+    vocab = 5
+    trajs = [rng.integers(0, vocab, size=int(rng.integers(0, 300))).tolist() for _ in range(16)]
+    tok, off = _flat(trajs)
+    d_tok = torch.from_numpy(tok).to("cuda:0")
+    ix = U.build_index(war, tok[:off[8]], off[:9], vocab, max_depth=96, capacity=len(tok) + len(trajs))
+    tails = rng.integers(0, vocab, size=(40, 12)).astype(np.int32)
+    tl = rng.integers(0, 13, size=40).astype(np.int32)
+    first, done = 0, 8
+
+    def check():
+        info = war.war_index_info(ix)
+        M = int(info.M)
+        assert info.T == done - first and M == (off[done] - off[first]) + (done - first)
+        wtok, woff = tok[off[first]:off[done]], off[first:done + 1] - off[first]
+        if M:
+            sa = _read_device(info.d_sa, M * 4).view(np.int32)
+            lcp = _read_device(info.d_lcp, M)
+            corpus = _read_device(info.d_corpus, (M + 8) * 4).view(np.int32).tolist()
+            assert corpus[M:] == [-1] * 8                                # the vacated end reads as "no token"
+            corpus = corpus[:M]
+            assert [v for v in corpus if v < 0] == [-(t + 1) for t in range(done - first)]
+            assert [v for v in corpus if v >= 0] == wtok.tolist()
+            assert sorted(sa.tolist()) == list(range(M))
+            naive = sorted(range(M), key=lambda i: corpus[i:])
+            assert [corpus[i:i + 128] for i in sa] == [corpus[i:i + 128] for i in naive]
+            for i in range(1, M):
+                a, b = corpus[sa[i - 1]:], corpus[sa[i]:]
+                l = 0
+                while l < min(len(a), len(b), 96) and a[l] == b[l]:
+                    l += 1
+                assert lcp[i] == l
+            bucket = _read_device(info.d_bucket, (vocab + 1) * 4).view(np.int32)
+            firsts = np.array([corpus[i] for i in sa])
+            for v in range(vocab + 1):
+                assert bucket[v] == int((firsts < v).sum())
+        _compare_with_oracle(war, wtok, woff, vocab, tails, tl, 24, 4, ix=ix)
+
+    for evict, add in ((3, 2), (0, 1), (4, 3), (1, 2)):
+        war.war_index_evict(ix, evict); first += evict
+        check()
+        war.war_index_append(ix, d_tok, off[done:done + add + 1]); done += add
+        check()
+    with pytest.raises(war.WarError):
+        war.war_index_evict(ix, done - first + 1)                        # more than is stored
+    war.war_index_evict(ix, done - first); first = done                  # everything: an empty index still answers
+    check()
+    war.war_index_append(ix, d_tok, off[0:3]); first, done = 0, 2       # and can be filled again
+    check()
+    ix.destroy()

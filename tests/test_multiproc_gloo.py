@@ -71,3 +71,18 @@ def test_trajectory_exchange_and_sharding(tmp_path):
     assert (res[2] == r0["ids"]).all() and (res[3] == r0["parent"]).all() and (res[4] == r0["count"]).all()
     shards = [np.load(tmp_path / f"shard{r}.npy") for r in range(world)]
     assert np.concatenate(shards).tolist() == list(range(11)) and abs(len(shards[0]) - len(shards[1])) <= 1
+
+
+def test_window_eviction_policy():
+    """Host logic of the sliding window: stored + incoming never exceeds the window, never evicts more than stored."""
+    assert replica.window_eviction(10, 3, 0) == 0                  # no window
+    assert replica.window_eviction(10, 3, 20) == 0
+    assert replica.window_eviction(10, 3, 13) == 0
+    assert replica.window_eviction(10, 3, 12) == 1
+    assert replica.window_eviction(10, 3, 3) == 10
+    assert replica.window_eviction(2, 9, 4) == 2                   # more incoming than the window holds
+    for stored in range(0, 12):
+        for incoming in range(0, 12):
+            for window in range(1, 12):
+                e = replica.window_eviction(stored, incoming, window)
+                assert 0 <= e <= stored and (stored - e + min(incoming, window) <= window or e == stored)
