@@ -120,10 +120,19 @@ war_status_t war_index_destroy(war_index_t* ix);
  * gets the root alone (num_nodes = 1, match_len = 0, count = 0), so the step that follows is a plain decode step
  * through the same calls: no state is kept between calls and one captured CUDA graph serves both modes.
  * spec_batch_limit = 0 always speculates.
+ * Two thresholds of the SuffixDecoding method the paper builds on (Section 3.2 takes that method's code base; the
+ * paper itself names neither), both exact integer rules, both off when their numerator is 0:
+ *   spec_factor_num / spec_factor_den   the tree has at most 1 + floor(match_len * num / den) slots, so a longer
+ *                                       match earns a larger tree (den >= 1)
+ *   min_prob_num / min_prob_den         a continuation is offered only if count(child) * den >= num * count(parent),
+ *                                       i.e. its empirical probability after the parent's string is at least
+ *                                       num / den (0 < num <= den)
  * ------------------------------------------------------------------------------------------------ */
 typedef struct {
     int32_t B, P, N, topk, min_match;
     int32_t spec_batch_limit;
+    int32_t spec_factor_num, spec_factor_den;
+    int32_t min_prob_num, min_prob_den;
 } war_draft_params_t;
 war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, const int32_t* d_tail_len,
                        const war_draft_params_t* params,

@@ -135,9 +135,18 @@ def longest_suffix_match(corpus: Corpus, tail: np.ndarray, tail_len: int) -> Tup
 
 
 def build_draft_tree(corpus: Corpus, tail: np.ndarray, match_len: int, ends: np.ndarray, N: int, k: int,
-                     min_match: int = 1):
-    """Returns (ids, parent, count) int32 arrays of length num_nodes (see module docstring for the rules)."""
+                     min_match: int = 1, spec_factor=(0, 1), min_prob=(0, 1)):
+    """Returns (ids, parent, count) int32 arrays of length num_nodes (see module docstring for the rules).
+
+    Two thresholds of the SuffixDecoding method the paper builds on (Section 3.2 takes that method's code base;
+    the paper itself names neither), both exact integer rules:
+      spec_factor (a, b), a > 0: the tree has at most 1 + floor(match_len * a / b) slots (a longer match earns a
+                  larger tree); (0, .) = no such cap.
+      min_prob (a, b), a > 0:    a continuation is offered only if count(child) * b >= a * count(parent), i.e. its
+                  empirical probability after the parent's string is at least a / b; (0, .) = every one is."""
     P = len(tail)
+    if spec_factor[0] > 0:
+        N = min(N, 1 + (match_len * spec_factor[0]) // spec_factor[1])
     tok = corpus.tokens
     ids, parent, count = [int(tail[P - 1])], [-1], [int(len(ends)) if match_len > 0 else 0]
     if match_len < max(1, min_match) or N <= 1:
@@ -154,7 +163,8 @@ def build_draft_tree(corpus: Corpus, tail: np.ndarray, match_len: int, ends: np.
             return []
         uniq, cnt = np.unique(t, return_counts=True)
         order = np.lexsort((uniq, -cnt))[:k]              # count descending, token id ascending
-        return [(int(cnt[o]), slot, int(uniq[o])) for o in order]
+        return [(int(cnt[o]), slot, int(uniq[o])) for o in order
+                if min_prob[0] == 0 or int(cnt[o]) * min_prob[1] >= min_prob[0] * len(nxt[slot])]
 
     frontier = offers(0)
     while len(ids) < N and frontier:
@@ -172,7 +182,7 @@ def build_draft_tree(corpus: Corpus, tail: np.ndarray, match_len: int, ends: np.
 
 
 def draft_batch(corpus: Corpus, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, min_match: int = 1,
-                spec_batch_limit: int = 0):
+                spec_batch_limit: int = 0, spec_factor=(0, 1), min_prob=(0, 1)):
     """Batched form with the library's output convention: unused slots hold ids = -1, parent = -1, count = 0.
 
     Workload-aware switch (paper, Section 3.2, "adaptive enabling and disabling" by the current batch size, and
@@ -194,7 +204,7 @@ def draft_batch(corpus: Corpus, tails: np.ndarray, tail_len: np.ndarray, N: int,
             ids[i, 0] = tails[i, -1]
             continue
         ml, ends = longest_suffix_match(corpus, tails[i], int(tail_len[i]))
-        a, b, c = build_draft_tree(corpus, tails[i], ml, ends, N, k, min_match)
+        a, b, c = build_draft_tree(corpus, tails[i], ml, ends, N, k, min_match, spec_factor, min_prob)
         n = len(a)
         match_len[i], num_nodes[i] = ml, n
         ids[i, :n], parent[i, :n], count[i, :n] = a, b, c

@@ -44,7 +44,8 @@ class IndexInfo(C.Structure):
 
 class DraftParams(C.Structure):
     _fields_ = [("B", C.c_int32), ("P", C.c_int32), ("N", C.c_int32), ("topk", C.c_int32), ("min_match", C.c_int32),
-                ("spec_batch_limit", C.c_int32)]
+                ("spec_batch_limit", C.c_int32), ("spec_factor_num", C.c_int32), ("spec_factor_den", C.c_int32),
+                ("min_prob_num", C.c_int32), ("min_prob_den", C.c_int32)]
 
 
 class AttnParams(C.Structure):
@@ -166,9 +167,10 @@ def war_index_destroy(ix: Index) -> None:
 
 def war_draft(ix: Index, d_tail: torch.Tensor, d_tail_len: torch.Tensor, N: int, topk: int, min_match: int,
               d_match_len: torch.Tensor, d_num_nodes: torch.Tensor, d_ids: torch.Tensor, d_parent: torch.Tensor,
-              d_count: Optional[torch.Tensor], spec_batch_limit: int = 0) -> None:
+              d_count: Optional[torch.Tensor], spec_batch_limit: int = 0, spec_factor=(0, 1), min_prob=(0, 1)) -> None:
+    """spec_factor / min_prob are (numerator, denominator) pairs; a numerator of 0 switches the rule off."""
     B, P = d_tail.shape
-    p = DraftParams(B, P, N, topk, min_match, spec_batch_limit)
+    p = DraftParams(B, P, N, topk, min_match, spec_batch_limit, spec_factor[0], spec_factor[1], min_prob[0], min_prob[1])
     code = _lib.war_draft(ix.handle, _ptr(d_tail, torch.int32), _ptr(d_tail_len, torch.int32), C.byref(p),
                           _ptr(d_match_len, torch.int32), _ptr(d_num_nodes, torch.int32), _ptr(d_ids, torch.int32),
                           _ptr(d_parent, torch.int32), _ptr(d_count, torch.int32), _stream())

@@ -217,7 +217,7 @@ struct Shared {
     int st_cnt[32], st_start[32];               // runs that cross span edges (one per span) and the closing run
     int fin_cnt[kMaxK], fin_start[kMaxK], fin_tok[kMaxK];
     int mode, cur, lo, cnt, depth, n_nodes, pool_n, thr_shared, long_runs_only, full_lo, full_cnt;
-    int n_running;
+    int n_running, n_cap;
 };
 
 // Tokens from index `from` on of the suffix at s against the pattern; returns the sign and, in `matched`, how many
@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, 2)
 war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, const uint8_t* __restrict__ lcp,
                  const int32_t* __restrict__ bucket, int vocab, const int32_t* __restrict__ tail,
                  const int32_t* __restrict__ tail_len, int B, int P, int N, int K, int min_match, int spec_batch_limit,
-                 int32_t* __restrict__ match_len, int32_t* __restrict__ num_nodes, int32_t* __restrict__ ids,
+                 int fac_num, int fac_den, int prob_num, int prob_den, int32_t* __restrict__ match_len, int32_t* __restrict__ num_nodes, int32_t* __restrict__ ids,
                  int32_t* __restrict__ parent, int32_t* __restrict__ count) {
     __shared__ Shared sh;
     const int b = blockIdx.x;
@@ -371,8 +371,11 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             hi = a;
         }
         const int c0 = ml > 0 ? hi - lo : 0;
-        const bool expand = ml >= max(1, min_match) && N > 1;
+        // node budget: a longer match earns a larger tree (at most 1 + floor(match_len * fac_num / fac_den) slots)
+        const int n_cap = fac_num > 0 ? min(N, 1 + (int)(((long long)ml * fac_num) / fac_den)) : N;
+        const bool expand = ml >= max(1, min_match) && n_cap > 1;
         if (lane == 0) {
+            sh.n_cap = n_cap;
             match_len[b] = ml;
             o_ids[0] = sh.pat[P - 1];
             o_par[0] = -1;
@@ -507,7 +510,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 int pmax = 0;
                 for (int i = lane; i < sh.pool_n; i += 32) pmax = max(pmax, sh.pool_cnt[i]);
                 pmax = __reduce_max_sync(0xffffffffu, pmax);
-                const int c = sh.full_cnt, flo = sh.full_lo, j0 = sh.n_nodes, room = N - j0;
+                const int c = sh.full_cnt, flo = sh.full_lo, j0 = sh.n_nodes, room = sh.n_cap - j0;
                 __syncwarp();
                 if (pmax < c && room > 0) {
                     const int64_t s_first = sa[flo], s_last = sa[flo + c - 1];
@@ -524,7 +527,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                         }
                         __syncwarp();
                         if (lane == 0) { sh.n_nodes = j0 + len; sh.mode = 0; }
-                        if (j0 + len < N) publish(j0 + len - 1, flo, c, d + len);
+                        if (j0 + len < sh.n_cap) publish(j0 + len - 1, flo, c, d + len);
                         continue;
                     }
                 }
@@ -534,8 +537,11 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             __syncwarp();
             if (lane == 0) {
                 int pn = sh.pool_n;
-                for (int e = 0; e < n_fin && pn < kPoolCap; ++e, ++pn) {
+                const long long need = (long long)prob_num * sh.full_cnt;      // count(child) * den >= num * count(parent)
+                for (int e = 0; e < n_fin && pn < kPoolCap; ++e) {
+                    if (prob_num > 0 && (long long)sh.fin_cnt[e] * prob_den < need) continue;
                     sh.pool_cnt[pn] = sh.fin_cnt[e]; sh.pool_par[pn] = cur; sh.pool_tok[pn] = sh.fin_tok[e]; sh.pool_lo[pn] = sh.fin_start[e];
+                    ++pn;
                 }
                 sh.pool_n = pn;
             }
@@ -572,7 +578,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                     sh.n_nodes = j + 1;
                     sh.mode = 0;
                 }
-                if (j + 1 < N) publish(j, slo, bc, depth);
+                if (j + 1 < sh.n_cap) publish(j, slo, bc, depth);
             }
         }
     }
@@ -591,13 +597,16 @@ extern "C" war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, 
                                   int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream) {
     if (!ix || !p) return WAR_ERR_INVALID_ARG;
     if (p->B < 0 || p->P < 1 || p->P > kMaxP || p->N < 1 || p->N > kMaxN || p->topk < 1 || p->topk > kMaxK || p->min_match < 0 ||
-        p->spec_batch_limit < 0)
+        p->spec_batch_limit < 0 || p->spec_factor_num < 0 || (p->spec_factor_num > 0 && p->spec_factor_den < 1) ||
+        p->min_prob_num < 0 || (p->min_prob_num > 0 && (p->min_prob_den < 1 || p->min_prob_num > p->min_prob_den)))
         return WAR_ERR_INVALID_ARG;
     if (p->P + p->N > ix->max_depth) return WAR_ERR_INVALID_ARG;     // the index is not ordered deep enough
     if (p->B == 0) return WAR_OK;
     if (!d_tail || !d_tail_len || !d_match_len || !d_num_nodes || !d_ids || !d_parent) return WAR_ERR_INVALID_ARG;
     war_draft_kernel<<<p->B, kThreads, 0, stream>>>(ix->corpus, ix->sa, ix->lcp, ix->bucket, ix->vocab, d_tail, d_tail_len,
-                                                   p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, d_match_len,
+                                                   p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, p->spec_factor_num,
+                                                   p->spec_factor_num > 0 ? p->spec_factor_den : 1, p->min_prob_num,
+                                                   p->min_prob_num > 0 ? p->min_prob_den : 1, d_match_len,
                                                    d_num_nodes, d_ids, d_parent, d_count);
     WAR_LAUNCH_CHECK();
     return WAR_OK;

@@ -14,7 +14,7 @@ def build_index(war, tokens: np.ndarray, offsets: np.ndarray, vocab: int, max_de
 
 
 def run_draft(war, ix, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, min_match: int = 1, with_count=True,
-              spec_batch_limit: int = 0):
+              spec_batch_limit: int = 0, spec_factor=(0, 1), min_prob=(0, 1)):
     B = tails.shape[0]
     d = dev()
     t = torch.from_numpy(np.ascontiguousarray(tails, dtype=np.int32)).to(d)
@@ -24,7 +24,7 @@ def run_draft(war, ix, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, 
     ids = torch.full((B, N), -7, dtype=torch.int32, device=d)
     par = torch.full((B, N), -7, dtype=torch.int32, device=d)
     cnt = torch.full((B, N), -7, dtype=torch.int32, device=d) if with_count else None
-    war.war_draft(ix, t, tl, N, k, min_match, ml, nn, ids, par, cnt, spec_batch_limit)
+    war.war_draft(ix, t, tl, N, k, min_match, ml, nn, ids, par, cnt, spec_batch_limit, spec_factor, min_prob)
     torch.cuda.synchronize()
     out = [ml.cpu().numpy(), nn.cpu().numpy(), ids.cpu().numpy(), par.cpu().numpy()]
     out.append(cnt.cpu().numpy() if with_count else None)

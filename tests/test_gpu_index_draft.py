@@ -317,3 +317,33 @@ def test_evicting_the_oldest_trajectories_equals_a_fresh_build(war, seed):
     war.war_index_append(ix, d_tok, off[0:3]); first, done = 0, 2       # and can be filled again
     check()
     ix.destroy()
+
+
+@pytest.mark.parametrize("spec_factor,min_prob", [((1, 1), (0, 1)), ((2, 3), (0, 1)), ((0, 1), (1, 2)), ((0, 1), (1, 10)),
+                                                  ((3, 1), (1, 4)), ((1, 8), (1, 1))])
+def test_node_budget_and_probability_threshold(war, spec_factor, min_prob):
+    """The two thresholds against the brute-force checker: the Tiny workload (template matches and junk matches) and
+    a tiny alphabet with heavy ties and large intervals (block-wide scans, chains)."""
+    cfg = W.CONFIGS["tiny"]
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(W.scaled(cfg, B=48))
+    ix = U.build_index(war, tok, off, cfg.vocab, max_depth=cfg.P + 64)
+    corpus = D.Corpus(tok, off)
+    for N, k in ((16, 4), (64, 8)):
+        got = U.run_draft(war, ix, tails, tl, N, k, spec_factor=spec_factor, min_prob=min_prob)
+        want = D.draft_batch(corpus, tails, tl, N, k, spec_factor=spec_factor, min_prob=min_prob)
+        for g, w in zip(got, want):
+            assert np.array_equal(g, w)
+    ix.destroy()
+    rng = np.random.default_rng(17)
+    trajs = [rng.integers(0, 3, size=int(rng.integers(50, 3000))).tolist() for _ in range(12)]
+    tok2, off2 = _flat(trajs)
+    tails2 = rng.integers(0, 3, size=(40, 10)).astype(np.int32)
+    tl2 = rng.integers(0, 11, size=40).astype(np.int32)
+    ix2 = U.build_index(war, tok2, off2, 3, max_depth=96)
+    got = U.run_draft(war, ix2, tails2, tl2, 32, 3, spec_factor=spec_factor, min_prob=min_prob)
+    want = D.draft_batch(D.Corpus(tok2, off2), tails2, tl2, 32, 3, spec_factor=spec_factor, min_prob=min_prob)
+    for g, w in zip(got, want):
+        assert np.array_equal(g, w)
+    assert war.war_device_status() == 0
+    ix2.destroy()

@@ -241,3 +241,45 @@ def test_workload_aware_switch():
     assert nn.tolist() == [1, 1, 0, 1, 1, 1] and (ml == 0).all() and (cnt == 0).all()
     for i in (0, 1, 3, 4, 5):
         assert ids[i, 0] == tails[i, -1] and par[i, 0] == -1 and (ids[i, 1:] == -1).all()
+
+
+def test_node_budget_and_probability_threshold():
+    """spec_factor caps the tree at 1 + floor(match_len * a / b) slots; min_prob keeps a continuation only when
+    count(child) / count(parent) >= a / b.  Checked on the hand-worked corpus and by properties on random ones."""
+    with open(os.path.join(GOLD, "draft_case1.json")) as f:
+        g = json.load(f)
+    trajs = [np.array(t, np.int32) for t in g["trajectories"]]
+    off = np.concatenate([[0], np.cumsum([len(t) for t in trajs])]).astype(np.int64)
+    corpus = D.Corpus(np.concatenate(trajs), off)
+    tail = np.array(g["tail"], np.int32)
+    ml, ends = D.longest_suffix_match(corpus, tail, len(tail))
+    assert ml == 3
+    full = D.build_draft_tree(corpus, tail, ml, ends, 16, 4)
+    # factor 1/1: 1 + 3 slots; 2/3: 1 + 2; the capped tree is a prefix of the uncapped one (best-first order)
+    for fac, n in (((1, 1), 4), ((2, 3), 3), ((5, 1), 14), ((1, 4), 1)):
+        ids, par, cnt = D.build_draft_tree(corpus, tail, ml, ends, 16, 4, spec_factor=fac)
+        assert len(ids) == n and ids.tolist() == full[0][:n].tolist() and par.tolist() == full[1][:n].tolist()
+    # min_prob 1/2: after [1,2,3] the continuations are 4 (2 of 3) and 5 (1 of 3): only 4 survives, then its own
+    # continuations 1 and 8 have 1 of 2 each = exactly 1/2: both stay
+    ids, par, cnt = D.build_draft_tree(corpus, tail, ml, ends, 6, 4, min_prob=(1, 2))
+    assert ids.tolist()[:4] == [3, 4, 1, 8] and par.tolist()[:4] == [-1, 0, 1, 1] and 5 not in ids.tolist()[1:2]
+    ids2, _, _ = D.build_draft_tree(corpus, tail, ml, ends, 6, 4, min_prob=(2, 3))
+    assert ids2.tolist() == [3, 4]                                  # 2/3: 4 stays (2 of 3), its continuations (1 of 2) do not
+    rng = np.random.default_rng(9)
+    toks = [rng.integers(0, 4, 60).astype(np.int32) for _ in range(6)]
+    off = np.concatenate([[0], np.cumsum([len(t) for t in toks])]).astype(np.int64)
+    corpus = D.Corpus(np.concatenate(toks), off)
+    for _ in range(50):
+        tail = rng.integers(0, 4, 6).astype(np.int32)
+        ml, ends = D.longest_suffix_match(corpus, tail, 6)
+        a, b = int(rng.integers(1, 4)), int(rng.integers(1, 5))
+        ids, par, cnt = D.build_draft_tree(corpus, tail, ml, ends, 20, 3, spec_factor=(a, b))
+        assert len(ids) <= max(1, 1 + ml * a // b)
+        pa, pb = int(rng.integers(1, 4)), 4
+        ids, par, cnt = D.build_draft_tree(corpus, tail, ml, ends, 20, 3, min_prob=(pa, pb))
+        for j in range(1, len(ids)):
+            assert cnt[j] * pb >= pa * cnt[par[j]]
+        # thresholds off = the plain rule
+        x = D.build_draft_tree(corpus, tail, ml, ends, 20, 3, spec_factor=(0, 1), min_prob=(0, 1))
+        y = D.build_draft_tree(corpus, tail, ml, ends, 20, 3)
+        assert all(np.array_equal(p, q) for p, q in zip(x, y))
