@@ -310,10 +310,28 @@ def main():
     h2d = sum(t.numel() * t.element_size() for t in (h_q, h_tails, h_tl, h_target))
     d2h = sum(t.numel() * t.element_size() for t in (r_alen, r_path, r_bonus, r_ids, r_par, r_nn, r_out))
 
+    # the queries are only needed by the verification: their copy runs on a second stream beside the draft call
+    copy_stream = torch.cuda.Stream()
+    q_ready = torch.cuda.Event()
+    main_stream = torch.cuda.current_stream()
+    overlap_q = h_q.numel() * h_q.element_size() >= (4 << 20)   # for a small batch the extra stream costs more than it hides
+
     def e2e_step():
-        attn.q.copy_(h_q, non_blocking=True); d_tails.copy_(h_tails, non_blocking=True)
-        d_tl.copy_(h_tl, non_blocking=True); d_target.copy_(h_target, non_blocking=True)
-        step()
+        d_tails.copy_(h_tails, non_blocking=True); d_tl.copy_(h_tl, non_blocking=True)
+        if overlap_q:
+            copy_stream.wait_stream(main_stream)            # the previous step's readers of q are done
+            with torch.cuda.stream(copy_stream):
+                attn.q.copy_(h_q, non_blocking=True)
+                q_ready.record(copy_stream)
+        else:
+            attn.q.copy_(h_q, non_blocking=True)
+        d_target.copy_(h_target, non_blocking=True)
+        war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt, args.spec_batch_limit)
+        if overlap_q:
+            main_stream.wait_event(q_ready)
+        war.war_verify_attn(attn.q, attn.k_pool, attn.v_pool, attn.page_table, attn.prefix_len, d_nn, d_par, params, ws,
+                            d_out, d_lse)
+        war.war_accept(d_ids, d_par, d_nn, d_target, 0, d_alen, d_path, d_bonus)
         for dst, src in ((r_alen, d_alen), (r_path, d_path), (r_bonus, d_bonus), (r_ids, d_ids), (r_par, d_par),
                          (r_nn, d_nn), (r_out, d_out)):
             dst.copy_(src, non_blocking=True)
