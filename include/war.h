@@ -68,6 +68,14 @@ typedef struct war_index war_index_t;          /* opaque; lives on the device th
  * war_index_append leaves the index answering every query exactly as a fresh build over the old
  * trajectories followed by the new ones would.  Exceeding the capacity returns WAR_ERR_CAPACITY and
  * leaves the index unchanged.  Both calls synchronise `stream` before returning.
+ * Updating without blocking the drafts (the paper updates the cache "asynchronously" so that it does not block
+ * the pipeline, Section 3.2): the index keeps two sets of (suffix array, LCP, buckets).  war_index_append builds
+ * the new set beside the published one and publishes it just before it returns; the corpus is only written
+ * behind what the published set refers to.  So ONE thread may run war_index_append (on its own stream) while other
+ * threads keep calling war_draft on other streams: a war_draft call uses the set that is published at the moment
+ * it is called, and that set stays intact until the NEXT update starts.  The caller makes sure that update does
+ * not start before those drafts have finished (an event, or one update per step).  Two updates must not
+ * overlap each other.  Cost: 5 more bytes per token of capacity.
  * ------------------------------------------------------------------------------------------------ */
 war_status_t war_index_build(const int32_t* d_tokens, const int64_t* h_offsets, int32_t T,
                              int32_t vocab, int32_t max_depth, int64_t capacity_tokens,
@@ -79,7 +87,8 @@ war_status_t war_index_append(war_index_t* ix, const int32_t* d_tokens, const in
  * is the simplest one): removes the n_oldest trajectories that were added first.  Afterwards every query answers
  * exactly as a fresh build on the remaining trajectories would.  The suffix array is filtered, not sorted again
  * (the remaining suffixes keep their order); LCP and buckets are recomputed.  Synchronises `stream`; allocates
- * and frees scratch of 4 bytes per stored token.  n_oldest must be in [0, T]. */
+ * and frees scratch of 4 bytes per stored token.  n_oldest must be in [0, T].  Unlike an append it moves the
+ * corpus itself, so no war_draft call may be in flight on this index while it runs. */
 war_status_t war_index_evict(war_index_t* ix, int32_t n_oldest, war_stream_t stream);
 
 typedef struct {

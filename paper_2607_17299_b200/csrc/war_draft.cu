@@ -603,7 +603,8 @@ extern "C" war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, 
     if (p->P + p->N > ix->max_depth) return WAR_ERR_INVALID_ARG;     // the index is not ordered deep enough
     if (p->B == 0) return WAR_OK;
     if (!d_tail || !d_tail_len || !d_match_len || !d_num_nodes || !d_ids || !d_parent) return WAR_ERR_INVALID_ARG;
-    war_draft_kernel<<<p->B, kThreads, 0, stream>>>(ix->corpus, ix->sa, ix->lcp, ix->bucket, ix->vocab, d_tail, d_tail_len,
+    const war_index_arrays arr = const_cast<war_index_t*>(ix)->published();       // a complete index, also during an update
+    war_draft_kernel<<<p->B, kThreads, 0, stream>>>(ix->corpus, arr.sa, arr.lcp, arr.bucket, ix->vocab, d_tail, d_tail_len,
                                                    p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, p->spec_factor_num,
                                                    p->spec_factor_num > 0 ? p->spec_factor_den : 1, p->min_prob_num,
                                                    p->min_prob_num > 0 ? p->min_prob_den : 1, d_match_len,

@@ -225,24 +225,28 @@ __global__ void bucket_from_sa_kernel(const int32_t* __restrict__ corpus, const 
     for (int v = prev + 1; v <= min(cur, vocab); ++v) bucket[v] = (int32_t)i;
 }
 
-// lcp and buckets from a finished suffix array
+// lcp and buckets of the shadow set from its finished suffix array; then the shadow set is published
 war_status_t finish_index(war_index* ix, cudaStream_t s) {
     const int64_t M = ix->M;
-    lcp_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, ix->sa, M, ix->max_depth, ix->lcp);
-    bucket_from_sa_kernel<<<grid_for(M + 1), kThreads, 0, s>>>(ix->corpus, ix->sa, M, ix->vocab, ix->bucket);
+    war_index_arrays& a = ix->shadow();
+    lcp_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, a.sa, M, ix->max_depth, a.lcp);
+    bucket_from_sa_kernel<<<grid_for(M + 1), kThreads, 0, s>>>(ix->corpus, a.sa, M, ix->vocab, a.bucket);
     WAR_LAUNCH_CHECK();
     WAR_CUDA_TRY(cudaStreamSynchronize(s));
+    ix->publish();
     return WAR_OK;
 }
 
-// (Re)builds sa / lcp / bucket from ix->corpus[0 .. M).
+// (Re)builds sa / lcp / bucket from ix->corpus[0 .. M) in the shadow set and publishes it.
 war_status_t rebuild(war_index* ix, cudaStream_t s) {
     const int64_t M = ix->M;
     if (M == 0) {
-        WAR_CUDA_TRY(cudaMemsetAsync(ix->bucket, 0, sizeof(int32_t) * (ix->vocab + 1), s));
+        WAR_CUDA_TRY(cudaMemsetAsync(ix->shadow().bucket, 0, sizeof(int32_t) * (ix->vocab + 1), s));
+        WAR_CUDA_TRY(cudaStreamSynchronize(s));
+        ix->publish();
         return WAR_OK;
     }
-    const war_status_t st = sort_suffixes(ix->corpus, M, ix->T, ix->vocab, ix->max_depth, ix->sa, s);
+    const war_status_t st = sort_suffixes(ix->corpus, M, ix->T, ix->vocab, ix->max_depth, ix->shadow().sa, s);
     if (st != WAR_OK) return st;
     return finish_index(ix, s);
 }
@@ -301,33 +305,32 @@ struct SumOp {
 
 war_status_t merge_new_suffixes(war_index* ix, int64_t M_old, cudaStream_t s) {
     const int64_t M = ix->M, m = M - M_old;
+    const war_index_arrays old = ix->published();
+    int32_t* sa_out = ix->shadow().sa;
     auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
     size_t temp_scan = 0, temp_scan2 = 0;
     WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(nullptr, temp_scan, (uint32_t*)nullptr, (uint32_t*)nullptr, MaxOp(), (int)m, s));
     WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(nullptr, temp_scan2, (uint32_t*)nullptr, (uint32_t*)nullptr, SumOp(), (int)(M_old + 1), s));
     size_t temp_bytes = temp_scan > temp_scan2 ? temp_scan : temp_scan2;
-    const size_t b_new = align(sizeof(int32_t) * m), b_pos = align(sizeof(uint32_t) * m), b_add = align(sizeof(uint32_t) * (M_old + 1)),
-                 b_out = align(sizeof(int32_t) * M);
+    const size_t b_new = align(sizeof(int32_t) * m), b_pos = align(sizeof(uint32_t) * m), b_add = align(sizeof(uint32_t) * (M_old + 1));
     Scratch scratch;
-    WAR_CUDA_TRY(cudaMalloc(&scratch.p, b_new + b_pos + b_add + b_out + align(temp_bytes)));
+    WAR_CUDA_TRY(cudaMalloc(&scratch.p, b_new + b_pos + b_add + align(temp_bytes)));
     char* at = (char*)scratch.p;
     int32_t* new_sa = (int32_t*)at; at += b_new;
     uint32_t* pos = (uint32_t*)at; at += b_pos;
     uint32_t* add = (uint32_t*)at; at += b_add;
-    int32_t* sa_out = (int32_t*)at; at += b_out;
     void* temp = at;
 
     war_status_t st = sort_suffixes(ix->corpus + M_old, m, ix->T, ix->vocab, ix->max_depth, new_sa, s);
     if (st != WAR_OK) return st;
-    insert_pos_kernel<<<grid_for(m), kThreads, 0, s>>>(ix->corpus, ix->sa, ix->bucket, new_sa, m, M_old, ix->vocab, ix->max_depth, pos);
+    insert_pos_kernel<<<grid_for(m), kThreads, 0, s>>>(ix->corpus, old.sa, old.bucket, new_sa, m, M_old, ix->vocab, ix->max_depth, pos);
     // positions must not decrease along the sorted new suffixes (they cannot, up to ties at full depth): enforce it
     WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, pos, pos, MaxOp(), (int)m, s));
     WAR_CUDA_TRY(cudaMemsetAsync(add, 0, b_add, s));
     count_pos_kernel<<<grid_for(m), kThreads, 0, s>>>(pos, m, add);
     WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, add, add, SumOp(), (int)(M_old + 1), s));
-    scatter_old_kernel<<<grid_for(M_old), kThreads, 0, s>>>(ix->sa, add, M_old, sa_out);
+    scatter_old_kernel<<<grid_for(M_old), kThreads, 0, s>>>(old.sa, add, M_old, sa_out);
     scatter_new_kernel<<<grid_for(m), kThreads, 0, s>>>(new_sa, pos, m, M_old, sa_out);
-    WAR_CUDA_TRY(cudaMemcpyAsync(ix->sa, sa_out, sizeof(int32_t) * M, cudaMemcpyDeviceToDevice, s));
     WAR_LAUNCH_CHECK();
     st = finish_index(ix, s);
     return st;
@@ -404,19 +407,20 @@ __global__ void shift_corpus_kernel(const int32_t* __restrict__ src, int64_t n, 
 
 war_status_t evict_oldest(war_index* ix, int32_t n, cudaStream_t s) {
     const int64_t cut = ix->bounds[(size_t)n], M_old = ix->M, M = M_old - cut;
+    const war_index_arrays old = ix->published();
     if (M > 0) {
         size_t temp_bytes = 0;
         WAR_CUDA_TRY(cub::DeviceSelect::If(nullptr, temp_bytes, (int32_t*)nullptr, (int32_t*)nullptr, (int32_t*)nullptr, (int)M_old,
                                            KeepFrom{(int32_t)cut}, s));
         auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
         Scratch scratch;
-        WAR_CUDA_TRY(cudaMalloc(&scratch.p, align(sizeof(int32_t) * M_old) + align(sizeof(int32_t)) + align(temp_bytes)));
+        WAR_CUDA_TRY(cudaMalloc(&scratch.p, align(sizeof(int32_t) * M) + align(sizeof(int32_t)) + align(temp_bytes)));
         int32_t* tmp = (int32_t*)scratch.p;
-        int32_t* d_n = (int32_t*)((char*)scratch.p + align(sizeof(int32_t) * M_old));
+        int32_t* d_n = (int32_t*)((char*)scratch.p + align(sizeof(int32_t) * M));
         void* temp = (char*)d_n + align(sizeof(int32_t));
-        WAR_CUDA_TRY(cub::DeviceSelect::If(temp, temp_bytes, ix->sa, tmp, d_n, (int)M_old, KeepFrom{(int32_t)cut}, s));
-        WAR_CUDA_TRY(cudaMemcpyAsync(ix->sa, tmp, sizeof(int32_t) * M, cudaMemcpyDeviceToDevice, s));
-        shift_sa_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->sa, M, (int32_t)cut);
+        int32_t* sa_new = ix->shadow().sa;
+        WAR_CUDA_TRY(cub::DeviceSelect::If(temp, temp_bytes, old.sa, sa_new, d_n, (int)M_old, KeepFrom{(int32_t)cut}, s));
+        shift_sa_kernel<<<grid_for(M), kThreads, 0, s>>>(sa_new, M, (int32_t)cut);
         shift_corpus_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, M, cut, n, tmp);
         WAR_CUDA_TRY(cudaMemcpyAsync(ix->corpus, tmp, sizeof(int32_t) * M, cudaMemcpyDeviceToDevice, s));
         WAR_LAUNCH_CHECK();
@@ -429,8 +433,9 @@ war_status_t evict_oldest(war_index* ix, int32_t n, cudaStream_t s) {
     ix->M = M;
     ix->T -= n;
     if (M == 0) {
-        WAR_CUDA_TRY(cudaMemsetAsync(ix->bucket, 0, sizeof(int32_t) * (ix->vocab + 1), s));
+        WAR_CUDA_TRY(cudaMemsetAsync(ix->shadow().bucket, 0, sizeof(int32_t) * (ix->vocab + 1), s));
         WAR_CUDA_TRY(cudaStreamSynchronize(s));
+        ix->publish();
         return WAR_OK;
     }
     return finish_index(ix, s);
@@ -455,11 +460,14 @@ extern "C" war_status_t war_index_build(const int32_t* d_tokens, const int64_t* 
     cudaGetDevice(&ix->device);
     const int64_t cap = capacity_tokens > 0 ? capacity_tokens : 1;
     cudaError_t e = cudaMalloc((void**)&ix->corpus, sizeof(int32_t) * (cap + 128));   // +128: readable slack behind the last separator
-    if (e == cudaSuccess) e = cudaMalloc((void**)&ix->sa, sizeof(int32_t) * cap);
-    if (e == cudaSuccess) e = cudaMalloc((void**)&ix->lcp, cap + 64);
-    if (e == cudaSuccess) e = cudaMalloc((void**)&ix->bucket, sizeof(int32_t) * (vocab + 1));
+    for (int k = 0; k < 2; ++k) {
+        if (e == cudaSuccess) e = cudaMalloc((void**)&ix->set[k].sa, sizeof(int32_t) * cap);
+        if (e == cudaSuccess) e = cudaMalloc((void**)&ix->set[k].lcp, cap + 64);
+        if (e == cudaSuccess) e = cudaMalloc((void**)&ix->set[k].bucket, sizeof(int32_t) * (vocab + 1));
+        if (e == cudaSuccess) e = cudaMemsetAsync(ix->set[k].lcp, 0, cap + 64, stream);
+        if (e == cudaSuccess) e = cudaMemsetAsync(ix->set[k].bucket, 0, sizeof(int32_t) * (vocab + 1), stream);
+    }
     if (e == cudaSuccess) e = cudaMemsetAsync(ix->corpus, 0xff, sizeof(int32_t) * (cap + 128), stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(ix->lcp, 0, cap + 64, stream);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         war_index_destroy(ix);
@@ -479,11 +487,17 @@ extern "C" war_status_t war_index_append(war_index_t* ix, const int32_t* d_token
     if (st != WAR_OK) return st;
     if (T == 0) return WAR_OK;
     const int64_t M_old = ix->M;
+    const int32_t T_old = ix->T;
     st = add_trajectories(ix, d_tokens, h_offsets, T, stream);
     if (st != WAR_OK) return st;
     // merging pays when the addition is the smaller part; otherwise sort everything again
-    if (M_old > 0 && ix->M - M_old < M_old) return merge_new_suffixes(ix, M_old, stream);
-    return rebuild(ix, stream);
+    st = (M_old > 0 && ix->M - M_old < M_old) ? merge_new_suffixes(ix, M_old, stream) : rebuild(ix, stream);
+    if (st != WAR_OK) {                                      // nothing was published: forget the addition
+        ix->M = M_old;
+        ix->T = T_old;
+        ix->bounds.resize((size_t)T_old + 1);
+    }
+    return st;
 }
 
 extern "C" war_status_t war_index_evict(war_index_t* ix, int32_t n_oldest, war_stream_t stream) {
@@ -500,19 +514,22 @@ extern "C" war_status_t war_index_info(const war_index_t* ix, war_index_info_t* 
     out->vocab = ix->vocab;
     out->max_depth = ix->max_depth;
     out->reserved = 0;
+    const war_index_arrays a = const_cast<war_index*>(ix)->published();
     out->d_corpus = ix->corpus;
-    out->d_sa = ix->sa;
-    out->d_lcp = ix->lcp;
-    out->d_bucket = ix->bucket;
+    out->d_sa = a.sa;
+    out->d_lcp = a.lcp;
+    out->d_bucket = a.bucket;
     return WAR_OK;
 }
 
 extern "C" war_status_t war_index_destroy(war_index_t* ix) {
     if (!ix) return WAR_OK;
     if (ix->corpus) cudaFree(ix->corpus);
-    if (ix->sa) cudaFree(ix->sa);
-    if (ix->lcp) cudaFree(ix->lcp);
-    if (ix->bucket) cudaFree(ix->bucket);
+    for (int k = 0; k < 2; ++k) {
+        if (ix->set[k].sa) cudaFree(ix->set[k].sa);
+        if (ix->set[k].lcp) cudaFree(ix->set[k].lcp);
+        if (ix->set[k].bucket) cudaFree(ix->set[k].bucket);
+    }
     delete ix;
     return WAR_OK;
 }

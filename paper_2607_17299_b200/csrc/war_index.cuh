@@ -1,13 +1,23 @@
 // The index object behind war_index_t (library-internal).
 #pragma once
 #include <stdint.h>
+#include <mutex>
 #include <vector>
 
-struct war_index {
-    int32_t* corpus = nullptr;   // [capacity + slack] trajectories joined by unique negative separators
+// The arrays a query reads.  There are two sets: queries read the published one, every update writes the other one
+// and publishes it when it is complete, so a query that was enqueued before an update returned keeps reading a
+// complete index.  The corpus is shared by both sets: an append only writes behind what the old set refers to.
+struct war_index_arrays {
     int32_t* sa = nullptr;       // [capacity]
     uint8_t* lcp = nullptr;      // [capacity + slack]
     int32_t* bucket = nullptr;   // [vocab + 1]
+};
+
+struct war_index {
+    int32_t* corpus = nullptr;   // [capacity + slack] trajectories joined by unique negative separators
+    war_index_arrays set[2];
+    int cur = 0;                 // published set; guarded by `lock` together with the pointers handed to queries
+    std::mutex lock;
     int64_t M = 0;               // corpus entries in use
     int64_t capacity = 0;
     int32_t T = 0;
@@ -15,4 +25,8 @@ struct war_index {
     int32_t max_depth = 0;
     int device = 0;
     std::vector<int64_t> bounds{0};   // host: corpus position where each stored trajectory starts, then M
+
+    war_index_arrays published() { std::lock_guard<std::mutex> g(lock); return set[cur]; }
+    war_index_arrays& shadow() { return set[cur ^ 1]; }                  // only the (single) updater touches it
+    void publish() { std::lock_guard<std::mutex> g(lock); cur ^= 1; }
 };

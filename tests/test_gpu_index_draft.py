@@ -347,3 +347,58 @@ def test_node_budget_and_probability_threshold(war, spec_factor, min_prob):
         assert np.array_equal(g, w)
     assert war.war_device_status() == 0
     ix2.destroy()
+
+
+def test_drafts_keep_running_while_the_index_is_updated(war):
+    """war_index_append builds the new arrays beside the published ones and publishes them when they are complete
+    (the paper updates the cache asynchronously so that the update does not block the pipeline, Section 3.2).  One
+    thread drafts in a loop on its own stream while another appends twice; every draft result must equal the
+    brute-force checker's answer on one of the three corpus states, and the states must appear in order."""
+    import threading
+    cfg = W.CONFIGS["tiny"]
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(W.scaled(cfg, B=32))
+    T = cfg.n_traj
+    cuts = [T - 24, T - 10, T]
+    d_tok = torch.from_numpy(tok).to("cuda:0")
+    ix = U.build_index(war, tok[:off[cuts[0]]], off[:cuts[0] + 1], cfg.vocab, max_depth=cfg.P + cfg.N, capacity=len(tok) + T)
+    wants = [D.draft_batch(D.Corpus(tok[:off[c]], off[:c + 1]), tails, tl, cfg.N, cfg.topk) for c in cuts]
+    assert not all(np.array_equal(a, b) for a, b in zip(wants[0], wants[2]))     # the appends change some draft
+    results, errors, stop = [], [], threading.Event()
+
+    def drafter():
+        try:
+            s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                while not stop.is_set() or len(results) < 3:
+                    results.append(U.run_draft(war, ix, tails, tl, cfg.N, cfg.topk))
+                    if len(results) > 4000:
+                        break
+        except Exception as e:                                       # noqa: BLE001
+            errors.append(e)
+
+    th = threading.Thread(target=drafter)
+    th.start()
+    s2 = torch.cuda.Stream()
+    with torch.cuda.stream(s2):
+        while len(results) < 5 and th.is_alive():
+            pass
+        war.war_index_append(ix, d_tok, off[cuts[0]:cuts[1] + 1])
+        n1 = len(results)
+        while len(results) < n1 + 5 and th.is_alive():
+            pass
+        war.war_index_append(ix, d_tok, off[cuts[1]:cuts[2] + 1])
+        n2 = len(results)
+        while len(results) < n2 + 5 and th.is_alive():
+            pass
+    stop.set()
+    th.join(timeout=60)
+    assert not errors and not th.is_alive()
+    state = 0
+    for got in results:
+        while state < 3 and not all(np.array_equal(g, w) for g, w in zip(got, wants[state])):
+            state += 1
+        assert state < 3, "a draft matched none of the corpus states (or went back to an older one)"
+    assert state == 2                                                 # the last drafts saw everything
+    assert war.war_device_status() == 0
+    ix.destroy()
