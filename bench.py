@@ -212,6 +212,14 @@ def main():
     tok, off = W.make_corpus(cfg)
     tails, tl = W.make_request_tails(cfg)
     ctx = W.context_lengths(cfg)
+    # the GPUs are shared: make sure the workload fits in what is free before allocating anything large
+    need = (int(((ctx - 1 + cfg.N + cfg.page_size - 1) // cfg.page_size).sum()) * cfg.Hkv * cfg.page_size * cfg.D * 2 * 2   # K and V pools
+            + (len(tok) + cfg.n_traj) * (14 + 44)                                                                        # index + build scratch
+            + 3 * cfg.B * cfg.N * cfg.Hq * cfg.D * 2 + (1 << 30))                                                        # q, out, workspace, slack
+    free, _total = torch.cuda.mem_get_info(dev)
+    if free < need:
+        raise SystemExit(f"bench.py: workload {cfg.name} needs about {need / 2**30:.1f} GiB of device memory, "
+                         f"{free / 2**30:.1f} GiB are free on cuda:{local_rank}")
     d_tok = torch.from_numpy(tok).to(dev)
     torch.cuda.synchronize()
     t0 = time.perf_counter()
