@@ -368,7 +368,9 @@ war_status_t check_params(const war_attn_params_t* p) {
     if (p->B < 0 || p->N < 1 || p->N > 64 || p->Hq < 1 || p->Hkv < 1 || p->Hq % p->Hkv != 0 || p->max_pages_per_req < 0 ||
         p->num_pages < 0 || p->kernel < 0 || p->kernel > 1 || !(p->scale > 0.f))
         return WAR_ERR_INVALID_ARG;
-    if (p->D != 128 || (p->page_size != 16 && p->page_size != 32)) return WAR_ERR_UNSUPPORTED;
+    // a 128-key tile is a whole number of pages, and a page is a whole number of 8-token groups of the tile layout
+    if (p->D != 128 || (p->page_size != 8 && p->page_size != 16 && p->page_size != 32 && p->page_size != 64 && p->page_size != 128))
+        return WAR_ERR_UNSUPPORTED;
     if ((p->Hq / p->Hkv) * p->N > 512 || p->B > kMaxPlanB) return WAR_ERR_UNSUPPORTED;
     if (!contiguous_head_major(p->k_strides, p) || !contiguous_head_major(p->v_strides, p)) return WAR_ERR_UNSUPPORTED;
     return WAR_OK;

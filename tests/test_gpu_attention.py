@@ -66,9 +66,9 @@ def test_tiny_config(war, kernel):
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
-@pytest.mark.parametrize("case", ["ragged16", "ragged32", "wide", "single", "deep", "many", "rows256"])
+@pytest.mark.parametrize("case", ["ragged16", "ragged32", "wide", "single", "deep", "many", "rows256", "page8", "page64", "page128"])
 def test_shapes_and_ragged_lengths(war, kernel, case):
-    rng = np.random.default_rng(["ragged16", "ragged32", "wide", "single", "deep", "many", "rows256"].index(case))
+    rng = np.random.default_rng(["ragged16", "ragged32", "wide", "single", "deep", "many", "rows256", "page8", "page64", "page128"].index(case))
     base = W.CONFIGS["tiny"]
     if case == "ragged16":       # lengths around page and tile edges, empty prefix, an unused request
         ctx = np.array([1, 2, 15, 16, 17, 113, 127, 128, 129, 1000, 1024, 1025, 2049, 3000])
@@ -78,6 +78,11 @@ def test_shapes_and_ragged_lengths(war, kernel, case):
     elif case == "ragged32":     # page size 32, 24 slots (96 rows)
         ctx = np.array([1, 31, 33, 500, 2047, 5000])
         cfg = W.scaled(base, B=len(ctx), N=24, page_size=32)
+        nn, parent = _random_trees(rng, cfg.B, cfg.N)
+    elif case in ("page8", "page64", "page128"):    # the other page sizes a 128-key tile can be cut into
+        pg = int(case[4:])
+        ctx = np.array([1, pg - 1, pg, pg + 1, 127, 129, 700, 2049, 4100])
+        cfg = W.scaled(base, B=len(ctx), N=16, page_size=pg)
         nn, parent = _random_trees(rng, cfg.B, cfg.N)
     elif case == "wide":         # 64 query heads on 8 kv heads, 64 slots: 512 rows per kv head, four row blocks
         ctx = np.array([700, 2500, 40])
