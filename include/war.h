@@ -159,8 +159,10 @@ war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, const int32
  * KV layout: logical position p of request b is row p % page_size of physical page
  * d_page_table[b, p / page_size]; slot a's K/V are at logical position prefix_len[b] + a (the caller writes
  * them before the call).  Pools are bf16 [num_pages, Hkv, page_size, D]; k_strides / v_strides give the
- * element strides of (page, head, token, d).  This build requires the contiguous head-major layout
- * (strides = {Hkv*page_size*D, page_size*D, D, 1}), page_size 8, 16, 32, 64 or 128, D == 128, Hq % Hkv == 0,
+ * element strides of (page, head, token, d).  Two memory layouts are accepted, the same one for both pools:
+ * head-major (strides = {Hkv*page_size*D, page_size*D, D, 1}; one copy per page and head, the faster one) and
+ * token-major (a page stored as [token][head][d]: strides = {page_size*Hkv*D, D, Hkv*D, 1}).
+ * Further: page_size 8, 16, 32, 64 or 128, D == 128, Hq % Hkv == 0,
  * (Hq/Hkv) * N <= 512, scale > 0; anything else returns WAR_ERR_UNSUPPORTED / WAR_ERR_INVALID_ARG.
  * Rows j >= num_nodes[b] of d_out / d_lse are left untouched.
  * d_workspace: war_verify_attn_workspace_bytes(params) bytes of device memory, 256-byte aligned, private to

@@ -34,6 +34,18 @@ struct AttnWorkspace {
     size_t bytes;
 };
 
+// Memory layout of a pool [num_pages, Hkv, page_size, D] as given by its element strides:
+//   0  head-major  (page, head, token, d contiguous in this order)
+//   1  token-major (page, token, head, d: the layout of engines that store a page as [block_size, heads, head_size])
+//  -1  anything else
+inline int war_attn_pool_layout(const int64_t* s, const war_attn_params_t* p) {
+    const int64_t D = p->D, pg = p->page_size, H = p->Hkv;
+    if (s[3] != 1) return -1;
+    if (s[2] == D && s[1] == pg * D && s[0] == H * pg * D) return 0;
+    if (s[1] == D && s[2] == H * D && s[0] == pg * H * D) return 1;
+    return -1;
+}
+
 inline AttnWorkspace war_attn_workspace_layout(const war_attn_params_t* p, void* base) {
     AttnWorkspace w;
     const int G = p->Hq / p->Hkv;

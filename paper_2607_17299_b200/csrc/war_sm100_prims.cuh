@@ -59,6 +59,13 @@ __device__ __forceinline__ void tma_load_block(uint32_t dst, const CUtensorMap* 
         ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(block) : "memory");
 }
 
+// token-major pools: tensor (d, token, head, page); one copy brings 64 dims of every token of one (page, head)
+__device__ __forceinline__ void tma_load_half_page(uint32_t dst, const CUtensorMap* map, int d0, int head, int page, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(d0), "r"(0), "r"(head), "r"(page) : "memory");
+}
+
 // shared-memory matrix descriptors: 128-byte swizzle, sm_100 version field.
 // The upper word of a descriptor (stride between 8-row groups, version, swizzle) is fixed per operand kind and the
 // lower word is an address plus a constant, so the issuing thread only adds small constants between MMAs: it is a

@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(128)
 attn_simple_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ kpool,
                    const __nv_bfloat16* __restrict__ vpool, const int32_t* __restrict__ page_table,
                    const int32_t* __restrict__ prefix_len, int N, int Hq, int Hkv, int G, int page_size, int max_pages,
-                   long long num_pages, float scale_log2, AttnWorkspace w, __nv_bfloat16* __restrict__ out,
+                   long long s_page, long long s_head, long long s_tok, long long num_pages, float scale_log2, AttnWorkspace w, __nv_bfloat16* __restrict__ out,
                    float* __restrict__ lse, int* status_word) {
     __shared__ __align__(16) __nv_bfloat16 sK[kSimpleTile][128];
     __shared__ __align__(16) __nv_bfloat16 sV[kSimpleTile][128];
@@ -293,7 +293,7 @@ attn_simple_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
                     long long page = page_table[(size_t)i * max_pages + pos / page_size];
                     if (page < 0 || page >= num_pages) { war_set_device_status(status_word, WAR_ERR_BAD_PAGE); page = 0; }
                     const __nv_bfloat16* pool = which ? vpool : kpool;
-                    const size_t off = (((size_t)page * Hkv + un.kvh) * page_size + pos % page_size) * 128 + piece * 8;
+                    const size_t off = (size_t)(page * s_page + un.kvh * s_head + (pos % page_size) * s_tok) + piece * 8;
                     val = *reinterpret_cast<const uint4*>(pool + off);
                 }
                 *reinterpret_cast<uint4*>(&(which ? sV : sK)[row][piece * 8]) = val;
@@ -358,11 +358,6 @@ attn_simple_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
     }
 }
 
-bool contiguous_head_major(const int64_t* s, const war_attn_params_t* p) {
-    return s[3] == 1 && s[2] == p->D && s[1] == (int64_t)p->page_size * p->D &&
-           s[0] == (int64_t)p->Hkv * p->page_size * p->D;
-}
-
 war_status_t check_params(const war_attn_params_t* p) {
     if (!p) return WAR_ERR_INVALID_ARG;
     if (p->B < 0 || p->N < 1 || p->N > 64 || p->Hq < 1 || p->Hkv < 1 || p->Hq % p->Hkv != 0 || p->max_pages_per_req < 0 ||
@@ -372,7 +367,8 @@ war_status_t check_params(const war_attn_params_t* p) {
     if (p->D != 128 || (p->page_size != 8 && p->page_size != 16 && p->page_size != 32 && p->page_size != 64 && p->page_size != 128))
         return WAR_ERR_UNSUPPORTED;
     if ((p->Hq / p->Hkv) * p->N > 512 || p->B > kMaxPlanB) return WAR_ERR_UNSUPPORTED;
-    if (!contiguous_head_major(p->k_strides, p) || !contiguous_head_major(p->v_strides, p)) return WAR_ERR_UNSUPPORTED;
+    const int layout = war_attn_pool_layout(p->k_strides, p);                 // both pools in the same one of the two layouts
+    if (layout < 0 || war_attn_pool_layout(p->v_strides, p) != layout) return WAR_ERR_UNSUPPORTED;
     return WAR_OK;
 }
 
@@ -384,6 +380,7 @@ war_status_t war_attn_launch_simple(const void* q, const void* k, const void* v,
     const int G = p->Hq / p->Hkv;
     attn_simple_kernel<<<148 * 4, 128, 0, s>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, page_table,
                                               prefix_len, p->N, p->Hq, p->Hkv, G, p->page_size, p->max_pages_per_req,
+                                              (long long)p->k_strides[0], (long long)p->k_strides[1], (long long)p->k_strides[2],
                                               (long long)p->num_pages, p->scale * kLog2e, w, (__nv_bfloat16*)out, lse, status_word);
     WAR_LAUNCH_CHECK();
     return WAR_OK;

@@ -16,8 +16,11 @@
 //                       as packed bf16; O is rescaled in TMEM only when the running max grows by more than 2^8
 //              The softmax warpgroups take registers from the third one (setmaxnreg) so a row of S fits.
 // Shared-memory operand layouts are the canonical 128-byte-swizzled ones: K-major for Q and K, MN-major for V.
-// A (page, head) block lands as [token/8][d/64][token%8][d%64], which serves both K (K-major, 8-row groups 2 KB
-// apart) and V (MN-major, 64-wide column blocks 1 KB apart, 8-key groups 2 KB apart) with one copy per block.
+// Head-major pools: a (page, head) block lands as [token/8][d/64][token%8][d%64], which serves both K (K-major,
+// 8-row groups 2 KB apart) and V (MN-major, 64-wide column blocks 1 KB apart, 8-key groups 2 KB apart) with one
+// copy per block.  Token-major pools (a page stored as [token][head][d]) cannot be copied that way in one piece (it
+// would take a 6-dimensional tensor map), so there a tile is laid out as [d/64][token][d%64] (8-row groups 1 KB
+// apart, the two 64-wide halves 16 KB apart) and every (page, head) takes two copies, one per half.
 // Every wait is bounded: on expiry the kernel records WAR_ERR_TIMEOUT, raises a CTA-wide abort flag and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -73,6 +76,7 @@ struct KernelArgs {
     int N, Hq, Hkv, G, page_size, max_pages;
 };
 
+template <bool kTokenMajor>                         // pool layout: false = (page, head, token, d), true = (page, token, head, d)
 __global__ void __launch_bounds__(kThreads, 1)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const KernelArgs a) {
     extern __shared__ uint8_t smem_raw[];
@@ -138,8 +142,14 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                 if (lane < n_valid) {
                     long long pg = page;
                     if (pg < 0 || pg >= a.num_pages) { war_set_device_status(a.status_word, WAR_ERR_BAD_PAGE); pg = 0; }
-                    tma_load_block(sRing + slot * kSlotBytes + lane * page_bytes, is_v ? &v_map : &k_map,
-                                   (int)(pg * a.Hkv + un.kvh), &bars->full[slot]);
+                    const CUtensorMap* map = is_v ? &v_map : &k_map;
+                    if (!kTokenMajor) {
+                        tma_load_block(sRing + slot * kSlotBytes + lane * page_bytes, map, (int)(pg * a.Hkv + un.kvh), &bars->full[slot]);
+                    } else {
+                        const uint32_t dst = sRing + slot * kSlotBytes + lane * (page_bytes >> 1);
+                        tma_load_half_page(dst, map, 0, un.kvh, (int)pg, &bars->full[slot]);
+                        tma_load_half_page(dst + 16384u, map, 64, un.kvh, (int)pg, &bars->full[slot]);
+                    }
                 }
                 return true;
             };
@@ -157,10 +167,15 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         uint32_t ld0 = 0, cg[2] = {0, 0}, units_done = 0;
         constexpr uint32_t idesc_s = umma_idesc(128, 128, 0);
         constexpr uint32_t idesc_o = umma_idesc(128, 128, 1);
-        constexpr uint32_t hi_q = umma_desc_hi(1024), hi_kv = umma_desc_hi(2048);
+        constexpr uint32_t hi_q = umma_desc_hi(1024);
         const uint32_t q_lo = umma_desc_lo(sQ, 16);                  // Q: K-major, 8-row groups 1 KB apart
-        const uint32_t ring_lo = umma_desc_lo(sRing, 16);             // K: K-major, 8-row groups 2 KB apart
-        const uint32_t ring_lo_v = umma_desc_lo(sRing, 1024);         // V: MN-major, 64-wide column blocks 1 KB apart
+        // K: K-major; V: MN-major.  Head-major tiles: 8-row groups 2 KB apart, the 64-wide halves 1 KB apart.
+        // Token-major tiles: 8-row groups 1 KB apart, the halves 16 KB apart.
+        const uint32_t hi_kv = kTokenMajor ? umma_desc_hi(1024) : umma_desc_hi(2048);
+        const uint32_t ring_lo = umma_desc_lo(sRing, 16);
+        const uint32_t ring_lo_v = umma_desc_lo(sRing, kTokenMajor ? 16384 : 1024);
+        const uint32_t k_half = (kTokenMajor ? 16384u : 1024u) >> 4;             // second 64 dims of K
+        const uint32_t v_step = (kTokenMajor ? 2048u : 4096u) >> 4;              // 16 keys of V
         bool ok = true;
         for (int k = 0; ok; ++k) {
             const int u = snake_unit(k, blockIdx.x, gridDim.x);
@@ -175,9 +190,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                     const uint32_t k_lo = ring_lo + slot * (kSlotBytes >> 4), d_s = tmem + g * 128u;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
-                        constexpr uint32_t kHalfQ = 16384u >> 4, kHalfK = 1024u >> 4;
+                        constexpr uint32_t kHalfQ = 16384u >> 4;
                         const uint32_t qo = (uint32_t)(ks >> 2) * kHalfQ + (uint32_t)(ks & 3) * 2u;
-                        const uint32_t ko = (uint32_t)(ks >> 2) * kHalfK + (uint32_t)(ks & 3) * 2u;
+                        const uint32_t ko = (uint32_t)(ks >> 2) * k_half + (uint32_t)(ks & 3) * 2u;
                         umma_bf16(d_s, pack64(q_lo + qo, hi_q), pack64(k_lo + ko, hi_kv), idesc_s, ks > 0);
                     }
                     umma_commit(&bars->s_ready[g]);
@@ -204,16 +219,16 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                     const uint32_t acc0 = t > 1 ? 1u : 0u;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
-                        umma_bf16_ts(d_o, a_p + (uint32_t)ks * 8u, pack64(v_lo + (uint32_t)ks * (4096u >> 4), hi_kv), idesc_o, ks > 0 ? 1u : acc0);
+                        umma_bf16_ts(d_o, a_p + (uint32_t)ks * 8u, pack64(v_lo + (uint32_t)ks * v_step, hi_kv), idesc_o, ks > 0 ? 1u : acc0);
                     if (has_s) {
                         // sixteen MMAs back to back; the completion signals follow the burst (the one the softmax group
                         // waits for first)
                         const uint32_t k_lo = ring_lo + slot_k * (kSlotBytes >> 4), d_s = tmem + g * 128u;
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {
-                            constexpr uint32_t kHalfQ = 16384u >> 4, kHalfK = 1024u >> 4;
+                            constexpr uint32_t kHalfQ = 16384u >> 4;
                             const uint32_t qo = (uint32_t)(ks >> 2) * kHalfQ + (uint32_t)(ks & 3) * 2u;
-                            const uint32_t ko = (uint32_t)(ks >> 2) * kHalfK + (uint32_t)(ks & 3) * 2u;
+                            const uint32_t ko = (uint32_t)(ks >> 2) * k_half + (uint32_t)(ks & 3) * 2u;
                             umma_bf16(d_s, pack64(q_lo + qo, hi_q), pack64(k_lo + ko, hi_kv), idesc_s, ks > 0);
                         }
                         umma_commit(&bars->s_ready[g]);
@@ -354,12 +369,14 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                     ok = mbar_wait(&bars->full[slot], (sq / kSlots) & 1u, bars, a.status_word);
                     if (!ok) break;
                     if (row >= L - key0) {
-                        const uint32_t base = sRing + slot * kSlotBytes + (uint32_t)(row >> 3) * 2048u + (uint32_t)(row & 7) * 128u;
+                        const uint32_t base = sRing + slot * kSlotBytes +
+                                              (kTokenMajor ? (uint32_t)row * 128u : (uint32_t)(row >> 3) * 2048u + (uint32_t)(row & 7) * 128u);
+                        const uint32_t half = kTokenMajor ? 16384u : 1024u;
 #pragma unroll
                         for (int h = 0; h < 2; ++h)
 #pragma unroll
                             for (int c = 0; c < 8; ++c)
-                                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + h * 1024u + c * 16u), "r"(0) : "memory");
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + h * half + c * 16u), "r"(0) : "memory");
                     }
                     fence_async_proxy();
                 }
@@ -466,14 +483,23 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// A pool [num_pages, Hkv, page_size, 128] bf16 seen as blocks of (page, head): [blocks][token/8][d/64][token%8][d%64].
-bool make_pool_map(CUtensorMap* map, const void* pool, long long num_pages, int Hkv, int page_size) {
+// A head-major pool [num_pages, Hkv, page_size, 128] bf16 seen as blocks of (page, head): [blocks][token/8][d/64][token%8][d%64].
+// A token-major pool (page, token, head, d) seen as (d, token, head, page) with a box of 64 dims x all tokens of one head.
+bool make_pool_map(CUtensorMap* map, const void* pool, long long num_pages, int Hkv, int page_size, int token_major) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    if (token_major) {
+        const cuuint64_t dims[4] = {128, (cuuint64_t)page_size, (cuuint64_t)Hkv, (cuuint64_t)num_pages};
+        const cuuint64_t strides[3] = {(cuuint64_t)Hkv * 256, 256, (cuuint64_t)page_size * Hkv * 256};
+        const cuuint32_t box[4] = {64, (cuuint32_t)page_size, 1, 1};
+        return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    }
     const cuuint64_t dims[5] = {64, 8, 2, (cuuint64_t)(page_size / 8), (cuuint64_t)(num_pages * Hkv)};
     const cuuint64_t strides[4] = {256, 128, 2048, (cuuint64_t)page_size * 256};
     const cuuint32_t box[5] = {64, 8, 2, (cuuint32_t)(page_size / 8), 1};
-    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(pool), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -491,19 +517,23 @@ war_status_t war_attn_launch_sm100(const void* q, const void* k, const void* v, 
     if (dev < 0 || dev >= 64) return WAR_ERR_UNSUPPORTED;
     if (!sm_count[dev]) WAR_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
     if (!attr_set[dev]) {
-        WAR_CUDA_TRY(cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        WAR_CUDA_TRY(cudaFuncSetAttribute(attn_sm100_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        WAR_CUDA_TRY(cudaFuncSetAttribute(attn_sm100_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
         attr_set[dev] = true;
     }
     if (p->num_pages == 0) return WAR_ERR_INVALID_ARG;
     CUtensorMap k_map, v_map;
-    if (!make_pool_map(&k_map, k, p->num_pages, p->Hkv, p->page_size) || !make_pool_map(&v_map, v, p->num_pages, p->Hkv, p->page_size))
+    const int token_major = war_attn_pool_layout(p->k_strides, p) == 1;
+    if (!make_pool_map(&k_map, k, p->num_pages, p->Hkv, p->page_size, token_major) ||
+        !make_pool_map(&v_map, v, p->num_pages, p->Hkv, p->page_size, token_major))
         return WAR_ERR_CUDA;
     KernelArgs a;
     a.q = (const __nv_bfloat16*)q; a.page_table = page_table; a.prefix_len = prefix_len;
     a.out = (__nv_bfloat16*)out; a.lse = lse; a.status_word = status_word; a.w = w;
     a.num_pages = p->num_pages; a.scale_log2 = p->scale * kLog2e;
     a.N = p->N; a.Hq = p->Hq; a.Hkv = p->Hkv; a.G = p->Hq / p->Hkv; a.page_size = p->page_size; a.max_pages = p->max_pages_per_req;
-    attn_sm100_kernel<<<sm_count[dev], kThreads, kSmemBytes, s>>>(k_map, v_map, a);
+    if (token_major) attn_sm100_kernel<true><<<sm_count[dev], kThreads, kSmemBytes, s>>>(k_map, v_map, a);
+    else attn_sm100_kernel<false><<<sm_count[dev], kThreads, kSmemBytes, s>>>(k_map, v_map, a);
     WAR_LAUNCH_CHECK();
     return WAR_OK;
 }

@@ -225,3 +225,26 @@ def test_malformed_inputs_are_reported_not_faulted(war, kernel):
     a.page_table[1, 2] = a.num_pages + 5                                     # a page index outside the pool
     U.run_attn(war, a, np.array([0, 3], np.int32), parent, 0.1, kernel)
     assert war.war_device_status() == 8
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("pg", [16, 32, 128])
+def test_token_major_pools(war, kernel, pg):
+    """Engines that store a page as [token][head][d] pass the same logical tensor with other strides.  The result
+    must equal the head-major call bit for bit (same arithmetic, other addressing) and the checker within tolerance."""
+    cfg = W.scaled(W.CONFIGS["tiny"], B=5, N=24, page_size=pg)
+    ctx = np.array([1, pg + 1, 900, 2049, 5000])
+    rng = np.random.default_rng(31 + pg)
+    nn, parent = _random_trees(rng, cfg.B, cfg.N)
+    a = W.make_attention_inputs(cfg, ctx, device="cuda:0")
+    _, _, head_major = U.run_attn(war, a, nn, parent, 0.088, kernel)
+    tm = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)       # same shape, (page, token, head, d) in memory
+    b = W.AttnInputs(q=a.q, k_pool=tm(a.k_pool), v_pool=tm(a.v_pool), page_table=a.page_table, prefix_len=a.prefix_len,
+                     num_pages=a.num_pages, max_pages=a.max_pages)
+    assert b.k_pool.stride() == (pg * cfg.Hkv * cfg.D, cfg.D, cfg.Hkv * cfg.D, 1)
+    _, raw = _check(war, cfg, ctx, nn, parent, kernel, scale=0.088, a=b)
+    assert torch.equal(raw, head_major)
+    # mixed layouts are refused
+    c = W.AttnInputs(q=a.q, k_pool=b.k_pool, v_pool=a.v_pool, page_table=a.page_table, prefix_len=a.prefix_len,
+                     num_pages=a.num_pages, max_pages=a.max_pages)
+    assert war.war_verify_attn_workspace_bytes(war.attn_params(c.q, c.k_pool, c.v_pool, c.page_table, 0.088, kernel)) == 0

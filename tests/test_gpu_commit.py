@@ -65,13 +65,17 @@ def _dense(k_pool, v_pool, pt_row, n):
     return A.gather_request_kv(k_pool, v_pool, pt_row, n)
 
 
-@pytest.mark.parametrize("N,pg,mode", [(8, 16, 0), (64, 16, 0), (24, 32, 0), (16, 16, 1), (1, 16, 0)])
-def test_commit_matches_checker(war, N, pg, mode):
+@pytest.mark.parametrize("N,pg,mode,token_major", [(8, 16, 0, False), (64, 16, 0, False), (24, 32, 0, False), (16, 16, 1, False),
+                                                   (1, 16, 0, False), (32, 16, 0, True), (16, 64, 0, True)])
+def test_commit_matches_checker(war, N, pg, mode, token_major):
     rng = np.random.default_rng(100 + N + pg + mode)
     B, Hkv, P = 37, 4, 32
     pl = rng.integers(0, 300, B).astype(np.int32)
     pl[:4] = [0, pg - 1, pg, 2 * pg - 1]                                       # page-boundary cases
     k_pool, v_pool, pt = _pool(rng, B, pl + N, Hkv, pg)
+    if token_major:                                                            # same logical tensors, (page, token, head, d) in memory
+        k_pool = k_pool.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        v_pool = v_pool.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
     nn, parent, ids = _random_trees(rng, B, N)
     target = _targets(rng, nn, parent, ids, mode)
     alen, path, bonus = U.run_accept(war, ids, parent, nn, target, mode)
