@@ -24,6 +24,7 @@ constexpr int kMaxN = 64;
 constexpr int kMaxK = 8;
 constexpr int kMaxP = 32;
 constexpr int kPoolCap = kMaxN * kMaxK;
+constexpr int kMemoMinCount = 33;        // nodes with at least this many occurrences go through the index's memo
 constexpr int kBlockScanMin = 1024;          // intervals at least this long are scanned by every warp (measured: 1024-2048 best)
 constexpr int kLongRunFirstMin = 1024;       // intervals at least this long first look for runs of 16 or more only
 
@@ -218,26 +219,27 @@ struct Shared {
     int fin_cnt[kMaxK], fin_start[kMaxK], fin_tok[kMaxK];
     int mode, cur, lo, cnt, depth, n_nodes, pool_n, thr_shared, long_runs_only, full_lo, full_cnt;
     int n_running, n_cap;
+    int memo_slot;                              // >= 0: the node being expanded goes into this memo entry when it is done
 };
 
 // Tokens from index `from` on of the suffix at s against the pattern; returns the sign and, in `matched`, how many
-// leading tokens agree.  Four corpus tokens are (then sixteen) corpus tokens are requested at a time so their latencies overlap (the corpus has
-// readable slack behind its last separator, and a separator always ends the walk).
+// leading tokens agree.  Eight corpus tokens, then sixteen at a time, are requested together so their latencies
+// overlap (the corpus has readable slack behind its last separator, and a separator always ends the walk).
 __device__ __forceinline__ int compare_suffix(const int32_t* __restrict__ corpus, int64_t s, const int* pat, int len, int from,
                                               int& matched) {
     int t = from;
     {
-        int c[4];
+        int c[8];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) c[i] = corpus[s + t + i];
+        for (int i = 0; i < 8; ++i) c[i] = corpus[s + t + i];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 8; ++i) {
             if (t + i < len) {
                 const int p = pat[t + i];
                 if (c[i] != p) { matched = t + i; return c[i] < p ? -1 : 1; }
             }
         }
-        t += 4;
+        t += 8;
     }
     // most comparisons end above; the ones that go on share a long prefix, so fetch far ahead
     for (; t < len; t += 16) {
@@ -258,7 +260,7 @@ __device__ __forceinline__ int compare_suffix(const int32_t* __restrict__ corpus
 
 __global__ void __launch_bounds__(kThreads, 2)
 war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, const uint8_t* __restrict__ lcp,
-                 const int32_t* __restrict__ bucket, int vocab, const int32_t* __restrict__ tail,
+                 const int32_t* __restrict__ bucket, int32_t* memo, int vocab, const int32_t* __restrict__ tail,
                  const int32_t* __restrict__ tail_len, int B, int P, int N, int K, int min_match, int spec_batch_limit,
                  int fac_num, int fac_den, int prob_num, int prob_den, int32_t* __restrict__ match_len, int32_t* __restrict__ num_nodes, int32_t* __restrict__ ids,
                  int32_t* __restrict__ parent, int32_t* __restrict__ count) {
@@ -304,11 +306,34 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
     auto publish = [&](int slot, int lo, int cnt, int depth) {          // warp 0, all lanes
         if (cnt <= 32) {                                                // handled in registers, one suffix per lane
             if (lane == 0) { sh.cur = slot; sh.lo = lo; sh.cnt = cnt; sh.depth = depth; sh.long_runs_only = 0; sh.mode = 3;
-                             sh.full_lo = lo; sh.full_cnt = cnt; }
+                             sh.full_lo = lo; sh.full_cnt = cnt; sh.memo_slot = -1; }
             return;
+        }
+        // Large nodes are looked up in the index's memo first (same node, same k => same answer for every request)
+        int memo_slot = -1;
+        if (cnt >= kMemoMinCount) {
+            const unsigned long long key = ((unsigned long long)(unsigned)(lo + 1) << 16) | ((unsigned long long)depth << 8) | (unsigned)K;
+            unsigned h = (unsigned)(key * 0x9E3779B97F4A7C15ull >> 40) & (kMemoEntries - 1);
+            volatile int32_t* en = memo + (size_t)h * kMemoInts;
+            const unsigned long long got = *(volatile unsigned long long*)en;
+            if (got == key) {
+                if (en[2] == 2) {                                        // ready: the payload was written before the state
+                    __threadfence();
+                    const int n_fin = en[3];
+                    if (lane < kMaxK) { sh.fin_cnt[lane] = en[4 + lane]; sh.fin_start[lane] = en[12 + lane]; sh.fin_tok[lane] = en[20 + lane]; }
+                    if (lane == 0) {
+                        sh.cur = slot; sh.lo = lo; sh.cnt = cnt; sh.depth = depth; sh.full_lo = lo; sh.full_cnt = cnt;
+                        sh.long_runs_only = 0; sh.thr_shared = 0; sh.memo_slot = -1 - n_fin; sh.mode = 4;
+                    }
+                    return;
+                }
+            } else if (got == 0ull) {
+                memo_slot = (int)h;                                      // free: this expansion will try to fill it
+            }
         }
         const int e = count_ending(corpus, sa, lo, lo + cnt, depth, lane);
         if (lane == 0) {
+            sh.memo_slot = memo_slot;
             sh.cur = slot; sh.lo = lo + e; sh.cnt = cnt - e; sh.depth = depth; sh.full_lo = lo; sh.full_cnt = cnt;
             // Large nodes are first scanned for runs of 16 positions or more only (bar preset to 16): that pass never
             // walks the boundaries inside a lane.  It is exact whenever it finds k such runs; otherwise the node is
@@ -342,8 +367,9 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                         if (compare_suffix(corpus, sa[mid], pat, len, min(ma, mz), m) < 0) { a = mid + 1; ma = m; } else { z = mid; mz = m; }
                     }
                     lo = a;
-                    // the pattern occurs iff the suffix there starts with it
-                    occurs = lo < bucket_hi && compare_suffix(corpus, sa[lo], pat, len, 1, m) == 0;
+                    // the pattern occurs iff the suffix there starts with it: that suffix was the last probe that was
+                    // not below the pattern, and mz tokens of it agreed
+                    occurs = lo < bucket_hi && mz == len;
                 }
             }
         }
@@ -358,6 +384,19 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         if (ml > 1) {
             const int* pat = sh.pat + (P - ml);
             int a = lo + 1, z = bucket_hi, m;                    // positions < a match, positions >= z do not
+            // A deep match has few occurrences, and they end where the LCP array first drops below the match length:
+            // look at the next 128 entries before probing the corpus.
+            {
+                int first = 1 << 30;
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int i = a + r * 32 + lane;
+                    const bool end = i >= z || (int)lcp[i] < ml;
+                    const unsigned e = __ballot_sync(0xffffffffu, end);
+                    if (e && first == (1 << 30)) first = a + r * 32 + __ffs(e) - 1;
+                }
+                if (first != (1 << 30)) { a = min(first, z); z = a; } else a += 128;      // uniform
+            }
             while (a < z) {
                 const int step = (z - a + 31) / 32;
                 const int pos = min(a + lane * step, z - 1);
@@ -413,7 +452,9 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         if (warp == 0) {
             const int cur = sh.cur;
             int n_fin = 0;
-            if (mode == 3) {
+            if (mode == 4) {
+                n_fin = -1 - sh.memo_slot;                               // everything is in sh.fin_* already
+            } else if (mode == 3) {
                 // at most 32 suffixes: lane i reads the continuation token of suffix lo+i; suffixes that end here hold a
                 // separator (negative) and sort first; equal tokens are adjacent, so a run is a head lane plus followers
                 const int tok = lane < cnt ? corpus[(int64_t)sa[lo + lane] + d] : -1;
@@ -501,6 +542,29 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 if (lane == 0) { sh.long_runs_only = 0; sh.thr_shared = 0; }
                 continue;
             }
+            // tokens of the winners, one lane each (the register path and the memo already have them)
+            if (mode != 3 && mode != 4 && lane < n_fin) sh.fin_tok[lane] = corpus[(int64_t)sa[sh.fin_start[lane]] + d];
+            __syncwarp();
+            if (mode != 4 && sh.memo_slot >= 0) {
+                // claim the free entry, write the payload, then mark it ready (another CTA may be doing the same for the
+                // same node: whoever loses the claim just goes on)
+                int32_t* en = memo + (size_t)sh.memo_slot * kMemoInts;
+                const unsigned long long key = ((unsigned long long)(unsigned)(sh.full_lo + 1) << 16) | ((unsigned long long)d << 8) | (unsigned)K;
+                int won = 0;
+                if (lane == 0) won = atomicCAS((unsigned long long*)en, 0ull, key) == 0ull;
+                won = __shfl_sync(0xffffffffu, won, 0);
+                if (won) {
+                    if (lane < kMaxK) {
+                        en[4 + lane] = lane < n_fin ? sh.fin_cnt[lane] : 0;
+                        en[12 + lane] = lane < n_fin ? sh.fin_start[lane] : 0;
+                        en[20 + lane] = lane < n_fin ? sh.fin_tok[lane] : 0;
+                    }
+                    if (lane == 0) en[3] = n_fin;
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) atomicExch(&en[2], 2);
+                }
+            }
             // ---- chain shortcut ----
             // If every occurrence of this node continues with the same token, that child has the node's own count; when
             // no pooled offer reaches that count it is the strict best and becomes the next slot, and the same holds for
@@ -532,9 +596,6 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                     }
                 }
             }
-            // tokens of the winners, one lane each (the register path above already has them)
-            if (mode != 3 && lane < n_fin) sh.fin_tok[lane] = corpus[(int64_t)sa[sh.fin_start[lane]] + d];
-            __syncwarp();
             if (lane == 0) {
                 int pn = sh.pool_n;
                 const long long need = (long long)prob_num * sh.full_cnt;      // count(child) * den >= num * count(parent)
@@ -604,7 +665,7 @@ extern "C" war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, 
     if (p->B == 0) return WAR_OK;
     if (!d_tail || !d_tail_len || !d_match_len || !d_num_nodes || !d_ids || !d_parent) return WAR_ERR_INVALID_ARG;
     const war_index_arrays arr = const_cast<war_index_t*>(ix)->published();       // a complete index, also during an update
-    war_draft_kernel<<<p->B, kThreads, 0, stream>>>(ix->corpus, arr.sa, arr.lcp, arr.bucket, ix->vocab, d_tail, d_tail_len,
+    war_draft_kernel<<<p->B, kThreads, 0, stream>>>(ix->corpus, arr.sa, arr.lcp, arr.bucket, arr.memo, ix->vocab, d_tail, d_tail_len,
                                                    p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, p->spec_factor_num,
                                                    p->spec_factor_num > 0 ? p->spec_factor_den : 1, p->min_prob_num,
                                                    p->min_prob_num > 0 ? p->min_prob_den : 1, d_match_len,

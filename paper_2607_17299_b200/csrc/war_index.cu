@@ -232,6 +232,7 @@ war_status_t finish_index(war_index* ix, cudaStream_t s) {
     lcp_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, a.sa, M, ix->max_depth, a.lcp);
     bucket_from_sa_kernel<<<grid_for(M + 1), kThreads, 0, s>>>(ix->corpus, a.sa, M, ix->vocab, a.bucket);
     WAR_LAUNCH_CHECK();
+    WAR_CUDA_TRY(cudaMemsetAsync(a.memo, 0, sizeof(int32_t) * kMemoEntries * kMemoInts, s));   // it described another suffix array
     WAR_CUDA_TRY(cudaStreamSynchronize(s));
     ix->publish();
     return WAR_OK;
@@ -464,6 +465,8 @@ extern "C" war_status_t war_index_build(const int32_t* d_tokens, const int64_t* 
         if (e == cudaSuccess) e = cudaMalloc((void**)&ix->set[k].sa, sizeof(int32_t) * cap);
         if (e == cudaSuccess) e = cudaMalloc((void**)&ix->set[k].lcp, cap + 64);
         if (e == cudaSuccess) e = cudaMalloc((void**)&ix->set[k].bucket, sizeof(int32_t) * (vocab + 1));
+        if (e == cudaSuccess) e = cudaMalloc((void**)&ix->set[k].memo, sizeof(int32_t) * kMemoEntries * kMemoInts);
+        if (e == cudaSuccess) e = cudaMemsetAsync(ix->set[k].memo, 0, sizeof(int32_t) * kMemoEntries * kMemoInts, stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(ix->set[k].lcp, 0, cap + 64, stream);
         if (e == cudaSuccess) e = cudaMemsetAsync(ix->set[k].bucket, 0, sizeof(int32_t) * (vocab + 1), stream);
     }
@@ -529,6 +532,7 @@ extern "C" war_status_t war_index_destroy(war_index_t* ix) {
         if (ix->set[k].sa) cudaFree(ix->set[k].sa);
         if (ix->set[k].lcp) cudaFree(ix->set[k].lcp);
         if (ix->set[k].bucket) cudaFree(ix->set[k].bucket);
+        if (ix->set[k].memo) cudaFree(ix->set[k].memo);
     }
     delete ix;
     return WAR_OK;

@@ -11,7 +11,15 @@ struct war_index_arrays {
     int32_t* sa = nullptr;       // [capacity]
     uint8_t* lcp = nullptr;      // [capacity + slack]
     int32_t* bucket = nullptr;   // [vocab + 1]
+    int32_t* memo = nullptr;     // [kMemoEntries * kMemoInts] expansions of large nodes, filled by the draft kernel
 };
+
+// Memo of node expansions (library-internal cache, part of a set: it describes that set's suffix array).  The draft
+// kernel spends most of a slow request in nodes with many occurrences (one- and two-token strings of frequent
+// tokens), and those nodes are the same for every request and step until the index changes.  An entry holds the
+// k best continuations of one node: key (lo + 1, depth, k), state, n, then count / start / token per continuation.
+constexpr int kMemoEntries = 1 << 16;
+constexpr int kMemoInts = 32;             // 128 bytes per entry
 
 struct war_index {
     int32_t* corpus = nullptr;   // [capacity + slack] trajectories joined by unique negative separators
