@@ -402,3 +402,38 @@ def test_drafts_keep_running_while_the_index_is_updated(war):
     assert state == 2                                                 # the last drafts saw everything
     assert war.war_device_status() == 0
     ix.destroy()
+
+
+def test_memo_of_node_expansions_never_changes_an_answer(war):
+    """The index caches the expansions of large nodes.  Same answers on an empty and on a filled memo, for different
+    k on the same nodes, and after an append (which must drop the entries of the old suffix array)."""
+    rng = np.random.default_rng(23)
+    vocab = 3                                                          # tiny alphabet: every node near the root is large
+    trajs = [rng.integers(0, vocab, size=int(rng.integers(500, 4000))).tolist() for _ in range(10)]
+    tok, off = _flat(trajs)
+    tails = rng.integers(0, vocab, size=(64, 8)).astype(np.int32)
+    tl = rng.integers(0, 9, size=64).astype(np.int32)
+    d_tok = torch.from_numpy(tok).to("cuda:0")
+    ix = U.build_index(war, tok[:off[7]], off[:8], vocab, max_depth=96, capacity=len(tok) + len(trajs))
+    corpus = D.Corpus(tok[:off[7]], off[:8])
+    first = {}
+    for rep in range(3):
+        for k in (1, 3, 2, 8):
+            got = U.run_draft(war, ix, tails, tl, 40, k)
+            if rep == 0:
+                want = D.draft_batch(corpus, tails, tl, 40, k)
+                for g, w in zip(got, want):
+                    assert np.array_equal(g, w)
+                first[k] = got
+                assert got[4][:, 0].max() > 1000                        # large nodes were expanded
+            else:
+                for g, w in zip(got, first[k]):
+                    assert np.array_equal(g, w)
+    war.war_index_append(ix, d_tok, off[7:])
+    want = D.draft_batch(D.Corpus(tok, off), tails, tl, 40, 3)
+    got = U.run_draft(war, ix, tails, tl, 40, 3)
+    for g, w in zip(got, want):
+        assert np.array_equal(g, w)
+    assert not all(np.array_equal(g, w) for g, w in zip(got, first[3]))   # the append did change the answers
+    assert war.war_device_status() == 0
+    ix.destroy()
