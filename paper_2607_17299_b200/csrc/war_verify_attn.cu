@@ -21,7 +21,7 @@ __device__ __forceinline__ uint64_t shfl64(uint64_t v, int src) {
 
 __global__ void __launch_bounds__(1024)
 attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ num_nodes,
-                 const int32_t* __restrict__ parent, int B, int N, int Hkv, int G, int page_size, int max_pages,
+                 const int32_t* __restrict__ parent, int B, int N, int Hkv, int G, int page_size, int max_pages, int n_ctas,
                  AttnWorkspace w, int* status_word) {
     constexpr int kPer = kMaxPlanB / 1024;    // requests per thread in the per-request phases
     __shared__ int s_tiles[kMaxPlanB];
@@ -30,7 +30,8 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     __shared__ uint8_t s_n[kMaxPlanB];        // validated slot count
     __shared__ int s_red[32];
     __shared__ long long s_sum[32];
-    __shared__ int s_chunk_tiles, s_total;
+    __shared__ int s_chunk_tiles, s_total, s_one_wave;
+    __shared__ long long s_tot;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     // ---- per request, one warp: validate, ancestor masks by pointer jumping, tile count ----
@@ -110,11 +111,42 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         long long ct = (tot + kTargetUnits - 1) / kTargetUnits;
         if (ct < kMinChunkTiles) ct = kMinChunkTiles;
         s_chunk_tiles = (int)ct;
+        s_tot = tot;
+        s_one_wave = 0;
         w.counters[0] = 0;
         w.counters[2] = (int)ct;
     }
     __syncthreads();
     const int chunk_tiles = s_chunk_tiles;
+    // Little work (few requests): one unit per CTA instead of many short ones.  Every (request, kv head, row block)
+    // gets a share of the CTAs in proportion to its tiles, rounded down; if that fits the grid it is used: one
+    // pipeline fill and one epilogue per CTA, and far fewer partials to merge.
+    const long long tot_all = s_tot;
+    auto chunks_one_wave = [&](int t) -> int {
+        if (t <= 0) return 0;
+        long long nc = tot_all > 0 ? (long long)t * n_ctas / tot_all : 1;        // tot_all: the tiles of all such triples
+        const int cap = max(1, t / 4);                                           // a chunk keeps at least four tiles
+        return (int)max(1ll, min(nc, (long long)cap));
+    };
+    {
+        long long mine = 0;
+#pragma unroll
+        for (int k = 0; k < kPer; ++k) mine += (long long)chunks_one_wave(r_tiles[k]) * Hkv * r_rbs[k];
+        for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+        if (lane == 0) s_sum[warp] = mine;
+        __syncthreads();
+        if (tid == 0) {
+            long long units = 0;
+            for (int i = 0; i < (int)(blockDim.x >> 5); ++i) units += s_sum[i];
+            s_one_wave = units <= n_ctas;
+        }
+        __syncthreads();
+    }
+    const bool one_wave = s_one_wave != 0;
+    auto chunks_of = [&](int t) -> int {
+        if (t <= 0) return 0;
+        return one_wave ? chunks_one_wave(t) : (t + chunk_tiles - 1) / chunk_tiles;
+    };
     // longest-first order: position = number of requests that rank before this one
 #pragma unroll
     for (int k = 0; k < kPer; ++k) {
@@ -127,7 +159,7 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
             pos += (tq > t) || (tq == t && q < i);
         }
         r_pos[k] = pos;
-        r_nc[k] = t > 0 ? (t + chunk_tiles - 1) / chunk_tiles : 0;
+        r_nc[k] = chunks_of(t);
         s_units[pos] = r_nc[k] * Hkv * r_rbs[k];
         s_order[pos] = (uint16_t)i;
     }
@@ -174,7 +206,7 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         const int i = s_order[lo];
         const int t = s_tiles[i], n = s_n[i];
         const int rbs = (G * n + kRowBlock - 1) / kRowBlock;
-        const int nc = (t + chunk_tiles - 1) / chunk_tiles;
+        const int nc = chunks_of(t);
         const int local = u - s_units[lo];
         const int c = local / (Hkv * rbs), rem = local % (Hkv * rbs);
         AttnUnit x;
@@ -408,8 +440,13 @@ extern "C" war_status_t war_verify_attn(const void* d_q, const void* d_kpool, co
     if (!status_word) return WAR_ERR_CUDA;
     const AttnWorkspace w = war_attn_workspace_layout(p, d_workspace);
     const int G = p->Hq / p->Hkv;
+    static int sm_count[64] = {0};
+    int dev = 0;
+    WAR_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return WAR_ERR_UNSUPPORTED;
+    if (!sm_count[dev]) WAR_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
     attn_plan_kernel<<<1, 1024, 0, stream>>>(d_prefix_len, d_num_nodes, d_parent, p->B, p->N, p->Hkv, G, p->page_size,
-                                            p->max_pages_per_req, w, status_word);
+                                            p->max_pages_per_req, sm_count[dev], w, status_word);
     WAR_LAUNCH_CHECK();
     if (p->kernel == 1)
         st = war_attn_launch_simple(d_q, d_kpool, d_vpool, d_page_table, d_prefix_len, p, w, d_out, d_lse, status_word, stream);
