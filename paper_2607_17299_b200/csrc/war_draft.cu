@@ -535,8 +535,8 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 }
             }
             __syncwarp();
-            int covered = 0;                                             // suffixes accounted for by the runs found
-            for (int e = 0; e < n_fin; ++e) covered += sh.fin_cnt[e];
+            // suffixes accounted for by the runs found
+            const int covered = __reduce_add_sync(0xffffffffu, lane < n_fin ? sh.fin_cnt[lane] : 0);
             if (sh.long_runs_only && n_fin < K && covered < cnt) {       // uniform: fewer than k long runs and more runs exist
                 __syncwarp();
                 if (lane == 0) { sh.long_runs_only = 0; sh.thr_shared = 0; }
@@ -596,15 +596,17 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                     }
                 }
             }
-            if (lane == 0) {
-                int pn = sh.pool_n;
-                const long long need = (long long)prob_num * sh.full_cnt;      // count(child) * den >= num * count(parent)
-                for (int e = 0; e < n_fin && pn < kPoolCap; ++e) {
-                    if (prob_num > 0 && (long long)sh.fin_cnt[e] * prob_den < need) continue;
-                    sh.pool_cnt[pn] = sh.fin_cnt[e]; sh.pool_par[pn] = cur; sh.pool_tok[pn] = sh.fin_tok[e]; sh.pool_lo[pn] = sh.fin_start[e];
-                    ++pn;
+            {   // the winners become offers, one lane each: count(child) * den >= num * count(parent) when a threshold is set
+                const int pn0 = sh.pool_n;
+                const int my_cnt = lane < n_fin ? sh.fin_cnt[lane] : 0;
+                const bool keep = lane < n_fin && (prob_num == 0 || (long long)my_cnt * prob_den >= (long long)prob_num * sh.full_cnt);
+                const unsigned km = __ballot_sync(0xffffffffu, keep);
+                const int at = pn0 + __popc(km & ((1u << lane) - 1u));
+                if (keep && at < kPoolCap) {
+                    sh.pool_cnt[at] = my_cnt; sh.pool_par[at] = cur; sh.pool_tok[at] = sh.fin_tok[lane]; sh.pool_lo[at] = sh.fin_start[lane];
                 }
-                sh.pool_n = pn;
+                __syncwarp();
+                if (lane == 0) sh.pool_n = min(kPoolCap, pn0 + __popc(km));
             }
             __syncwarp();
             // ---- take the best offer: count desc, parent slot asc, token asc ----
@@ -614,11 +616,16 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 const int c = sh.pool_cnt[i], p = sh.pool_par[i], t = sh.pool_tok[i];
                 if (bi < 0 || c > bc || (c == bc && (p < bp || (p == bp && t < bt)))) { bi = i; bc = c; bp = p; bt = t; }
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const int oi = __shfl_xor_sync(0xffffffffu, bi, o), oc = __shfl_xor_sync(0xffffffffu, bc, o);
-                const int op = __shfl_xor_sync(0xffffffffu, bp, o), ot = __shfl_xor_sync(0xffffffffu, bt, o);
-                if (oi >= 0 && (bi < 0 || oc > bc || (oc == bc && (op < bp || (op == bp && ot < bt))))) { bi = oi; bc = oc; bp = op; bt = ot; }
+            {   // best of the lanes' candidates: largest count, then smallest parent slot, then smallest token (unique)
+                const int c_best = __reduce_max_sync(0xffffffffu, bc);                       // -1 when the pool is empty
+                const bool in1 = bi >= 0 && bc == c_best;
+                const int p_best = __reduce_min_sync(0xffffffffu, in1 ? bp : 0x7fffffff);
+                const bool in2 = in1 && bp == p_best;
+                const int t_best = __reduce_min_sync(0xffffffffu, in2 ? bt : 0x7fffffff);
+                const unsigned wm = __ballot_sync(0xffffffffu, in2 && bt == t_best);
+                const int wl = wm ? __ffs(wm) - 1 : 0;
+                bi = wm ? __shfl_sync(0xffffffffu, bi, wl) : -1;
+                bc = c_best; bp = p_best; bt = t_best;
             }
             // every lane now holds the same winner
             if (bi < 0) {
