@@ -469,10 +469,10 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 for (int r = 0; r < K; ++r) {
                     const int key = __reduce_max_sync(0xffffffffu, c * 64 + (63 - lane));
                     if (key < 64) break;                                  // no run left
-                    const int wl = 63 - (key & 63);
-                    const int wt = __shfl_sync(0xffffffffu, tok, wl);
-                    if (lane == 0) { sh.fin_cnt[n_fin] = key >> 6; sh.fin_start[n_fin] = lo + wl; sh.fin_tok[n_fin] = wt; }
-                    if (lane == wl) c = 0;
+                    if (lane == 63 - (key & 63)) {                        // the winning head writes its own run
+                        sh.fin_cnt[n_fin] = c; sh.fin_start[n_fin] = lo + lane; sh.fin_tok[n_fin] = tok;
+                        c = 0;
+                    }
                     ++n_fin;
                 }
             } else if (cnt > 0 && mode == 1) {
