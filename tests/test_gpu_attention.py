@@ -248,3 +248,33 @@ def test_token_major_pools(war, kernel, pg):
     c = W.AttnInputs(q=a.q, k_pool=b.k_pool, v_pool=a.v_pool, page_table=a.page_table, prefix_len=a.prefix_len,
                      num_pages=a.num_pages, max_pages=a.max_pages)
     assert war.war_verify_attn_workspace_bytes(war.attn_params(c.q, c.k_pool, c.v_pool, c.page_table, 0.088, kernel)) == 0
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes_against_the_checker(war, seed):
+    """Shapes drawn at random: batch, slots, heads per group, page size, pool layout, contexts from 1 token to a few
+    thousand (so that single-tile requests, split requests, one-wave and many-unit plans, ragged last tiles and empty
+    requests all occur together), random trees.  Every request is compared; the call is repeated for determinism."""
+    rng = np.random.default_rng(900 + seed)
+    for _ in range(4):
+        G = int(rng.choice([1, 2, 4, 8]))
+        Hkv = int(rng.choice([1, 2, 8]))
+        N = int(rng.choice([1, 3, 8, 16, 33, 64]))
+        while G * N > 512:
+            N //= 2
+        pg = int(rng.choice([8, 16, 32, 64, 128]))
+        B = int(rng.integers(1, 12))
+        ctx = rng.integers(1, int(rng.choice([40, 300, 2500, 6000])), size=B)
+        cfg = W.scaled(W.CONFIGS["tiny"], B=B, N=N, Hq=G * Hkv, Hkv=Hkv, page_size=pg)
+        nn, parent = _random_trees(rng, B, N)
+        if B > 2:
+            nn[int(rng.integers(0, B))] = 0                                   # a request that is not running
+        a = W.make_attention_inputs(cfg, ctx, device="cuda:0")
+        if rng.random() < 0.5:                                                # token-major pools
+            tm = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+            a = W.AttnInputs(q=a.q, k_pool=tm(a.k_pool), v_pool=tm(a.v_pool), page_table=a.page_table, prefix_len=a.prefix_len,
+                             num_pages=a.num_pages, max_pages=a.max_pages)
+        scale = float(rng.choice([0.05, 0.088, 0.2]))
+        _, raw1 = _check(war, cfg, ctx, nn, parent, 0, scale=scale, a=a)
+        _, _, raw2 = U.run_attn(war, a, nn, parent, scale, 0)
+        assert torch.equal(raw1, raw2)
