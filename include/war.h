@@ -91,6 +91,17 @@ war_status_t war_index_append(war_index_t* ix, const int32_t* d_tokens, const in
  * corpus itself, so no war_draft call may be in flight on this index while it runs. */
 war_status_t war_index_evict(war_index_t* ix, int32_t n_oldest, war_stream_t stream);
 
+/* Export / import: the whole index as one host buffer (header, trajectory bounds, corpus, suffix array, LCP,
+ * buckets), so that a replica that starts later, or restarts, takes the arrays instead of sorting again.  The paper
+ * has no counterpart (its cache lives in the serving process).  war_index_export writes
+ * war_index_export_bytes(ix) bytes to h_dst; war_index_import checks the header and the sizes (not the arrays'
+ * contents: import only what an export wrote) and returns an index of the given capacity that answers exactly as the
+ * exported one.  Both synchronise `stream`. */
+size_t war_index_export_bytes(const war_index_t* ix);
+war_status_t war_index_export(const war_index_t* ix, void* h_dst, size_t bytes, war_stream_t stream);
+war_status_t war_index_import(const void* h_src, size_t bytes, int64_t capacity_tokens, war_stream_t stream,
+                              war_index_t** out);
+
 typedef struct {
     int64_t M;                  /* corpus entries in use: tokens + one separator per trajectory */
     int64_t capacity_tokens;

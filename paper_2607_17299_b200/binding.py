@@ -25,7 +25,8 @@ WAR_OK = 0
 STATUS_NAMES = {0: "WAR_OK", 1: "WAR_ERR_INVALID_ARG", 2: "WAR_ERR_OOM", 3: "WAR_ERR_CAPACITY", 4: "WAR_ERR_CUDA",
                 5: "WAR_ERR_TIMEOUT", 6: "WAR_ERR_UNSUPPORTED", 7: "WAR_ERR_BAD_TREE", 8: "WAR_ERR_BAD_PAGE"}
 
-EXPORTS = ["war_index_build", "war_index_append", "war_index_evict", "war_index_info", "war_index_destroy", "war_draft",
+EXPORTS = ["war_index_build", "war_index_append", "war_index_evict", "war_index_export_bytes", "war_index_export",
+           "war_index_import", "war_index_info", "war_index_destroy", "war_draft",
            "war_verify_attn_workspace_bytes", "war_verify_attn", "war_verify_attn_noalloc", "war_accept", "war_commit", "war_device_status",
            "war_status_string"]
 
@@ -64,6 +65,12 @@ _lib.war_index_append.restype = C.c_int
 _lib.war_index_append.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
 _lib.war_index_evict.restype = C.c_int
 _lib.war_index_evict.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+_lib.war_index_export_bytes.restype = C.c_size_t
+_lib.war_index_export_bytes.argtypes = [C.c_void_p]
+_lib.war_index_export.restype = C.c_int
+_lib.war_index_export.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.war_index_import.restype = C.c_int
+_lib.war_index_import.argtypes = [C.c_void_p, C.c_size_t, C.c_int64, C.c_void_p, C.POINTER(C.c_void_p)]
 _lib.war_index_info.restype = C.c_int
 _lib.war_index_info.argtypes = [C.c_void_p, C.POINTER(IndexInfo)]
 _lib.war_index_destroy.restype = C.c_int
@@ -153,6 +160,21 @@ def war_index_append(ix: Index, d_tokens: torch.Tensor, h_offsets) -> None:
 
 def war_index_evict(ix: Index, n_oldest: int) -> None:
     _check("war_index_evict", _lib.war_index_evict(ix.handle, int(n_oldest), _stream()))
+
+
+def war_index_export(ix: Index) -> np.ndarray:
+    """The whole index as one host byte array (see war_index_import)."""
+    n = int(_lib.war_index_export_bytes(ix.handle))
+    buf = np.empty(n, dtype=np.uint8)
+    _check("war_index_export", _lib.war_index_export(ix.handle, buf.ctypes.data, n, _stream()))
+    return buf
+
+
+def war_index_import(buf: np.ndarray, capacity_tokens: int) -> Index:
+    buf = np.ascontiguousarray(buf, dtype=np.uint8)
+    h = C.c_void_p()
+    _check("war_index_import", _lib.war_index_import(buf.ctypes.data, buf.nbytes, int(capacity_tokens), _stream(), C.byref(h)))
+    return Index(h.value)
 
 
 def war_index_info(ix: Index) -> IndexInfo:

@@ -7,6 +7,7 @@
 // Suffixes that still tie after the last round keep the order the stable sort left them in; no output of the
 // library depends on that order.
 #include <cub/cub.cuh>
+#include <cstring>
 #include <new>
 #include "war_common.cuh"
 #include "war_index.cuh"
@@ -507,6 +508,90 @@ extern "C" war_status_t war_index_evict(war_index_t* ix, int32_t n_oldest, war_s
     if (!ix || n_oldest < 0 || n_oldest > ix->T) return WAR_ERR_INVALID_ARG;
     if (n_oldest == 0) return WAR_OK;
     return evict_oldest(ix, n_oldest, stream);
+}
+
+// ---- export / import ------------------------------------------------------------------------------
+// Layout of an exported index (host memory, little endian): header, int64 bounds[T+1], int32 corpus[M], int32 sa[M],
+// uint8 lcp[M] padded to 8 bytes, int32 bucket[vocab+1].
+struct ExportHeader {
+    uint64_t magic;              // "WARINDX1"
+    int64_t M;
+    int32_t T, vocab, max_depth, reserved;
+};
+constexpr uint64_t kExportMagic = 0x3158444e49524157ull;
+static size_t pad8(size_t x) { return (x + 7) & ~(size_t)7; }
+static size_t export_bytes(int64_t M, int32_t T, int32_t vocab) {
+    return sizeof(ExportHeader) + sizeof(int64_t) * ((size_t)T + 1) + 2 * pad8(sizeof(int32_t) * (size_t)M) + pad8((size_t)M) +
+           pad8(sizeof(int32_t) * ((size_t)vocab + 1));
+}
+
+extern "C" size_t war_index_export_bytes(const war_index_t* ix) {
+    return ix ? export_bytes(ix->M, ix->T, ix->vocab) : 0;
+}
+
+extern "C" war_status_t war_index_export(const war_index_t* cix, void* h_dst, size_t bytes, war_stream_t stream) {
+    war_index* ix = const_cast<war_index*>(cix);
+    if (!ix || !h_dst || bytes < export_bytes(ix->M, ix->T, ix->vocab)) return WAR_ERR_INVALID_ARG;
+    const war_index_arrays a = ix->published();
+    const size_t M = (size_t)ix->M;
+    char* at = (char*)h_dst;
+    ExportHeader h = {kExportMagic, ix->M, ix->T, ix->vocab, ix->max_depth, 0};
+    memcpy(at, &h, sizeof(h)); at += sizeof(h);
+    memcpy(at, ix->bounds.data(), sizeof(int64_t) * ((size_t)ix->T + 1)); at += sizeof(int64_t) * ((size_t)ix->T + 1);
+    WAR_CUDA_TRY(cudaMemcpyAsync(at, ix->corpus, sizeof(int32_t) * M, cudaMemcpyDeviceToHost, stream)); at += pad8(sizeof(int32_t) * M);
+    WAR_CUDA_TRY(cudaMemcpyAsync(at, a.sa, sizeof(int32_t) * M, cudaMemcpyDeviceToHost, stream)); at += pad8(sizeof(int32_t) * M);
+    WAR_CUDA_TRY(cudaMemcpyAsync(at, a.lcp, M, cudaMemcpyDeviceToHost, stream)); at += pad8(M);
+    WAR_CUDA_TRY(cudaMemcpyAsync(at, a.bucket, sizeof(int32_t) * ((size_t)ix->vocab + 1), cudaMemcpyDeviceToHost, stream));
+    WAR_CUDA_TRY(cudaStreamSynchronize(stream));
+    // the few bytes that pad a section to 8 are defined too (an export is a function of the index alone)
+    char* sec = (char*)h_dst + sizeof(ExportHeader) + sizeof(int64_t) * ((size_t)ix->T + 1);
+    const size_t lens[4] = {sizeof(int32_t) * M, sizeof(int32_t) * M, M, sizeof(int32_t) * ((size_t)ix->vocab + 1)};
+    for (int k = 0; k < 4; ++k) {
+        memset(sec + lens[k], 0, pad8(lens[k]) - lens[k]);
+        sec += pad8(lens[k]);
+    }
+    return WAR_OK;
+}
+
+extern "C" war_status_t war_index_import(const void* h_src, size_t bytes, int64_t capacity_tokens, war_stream_t stream,
+                                         war_index_t** out) {
+    if (!out) return WAR_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!h_src || bytes < sizeof(ExportHeader)) return WAR_ERR_INVALID_ARG;
+    ExportHeader h;
+    memcpy(&h, h_src, sizeof(h));
+    if (h.magic != kExportMagic || h.M < 0 || h.T < 0 || h.vocab < 1 || h.max_depth < 1 || h.max_depth > 128 || h.M < h.T)
+        return WAR_ERR_INVALID_ARG;
+    if (bytes < export_bytes(h.M, h.T, h.vocab)) return WAR_ERR_INVALID_ARG;
+    if (capacity_tokens < h.M) return WAR_ERR_CAPACITY;
+    const char* at = (const char*)h_src + sizeof(h);
+    const int64_t* bounds = (const int64_t*)at;
+    if (bounds[0] != 0 || bounds[h.T] != h.M) return WAR_ERR_INVALID_ARG;
+    for (int t = 0; t < h.T; ++t)
+        if (bounds[t + 1] <= bounds[t]) return WAR_ERR_INVALID_ARG;     // every trajectory holds at least its separator
+    // an empty index of that capacity, then the arrays
+    const int64_t zero = 0;
+    war_index_t* ix = nullptr;
+    war_status_t st = war_index_build(nullptr, &zero, 0, h.vocab, h.max_depth, capacity_tokens, stream, &ix);
+    if (st != WAR_OK) return st;
+    const size_t M = (size_t)h.M;
+    at += sizeof(int64_t) * ((size_t)h.T + 1);
+    war_index_arrays& a = ix->shadow();
+    cudaError_t e = cudaMemcpyAsync(ix->corpus, at, sizeof(int32_t) * M, cudaMemcpyHostToDevice, stream); at += pad8(sizeof(int32_t) * M);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(a.sa, at, sizeof(int32_t) * M, cudaMemcpyHostToDevice, stream);
+    at += pad8(sizeof(int32_t) * M);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(a.lcp, at, M, cudaMemcpyHostToDevice, stream);
+    at += pad8(M);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(a.bucket, at, sizeof(int32_t) * ((size_t)h.vocab + 1), cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(a.memo, 0, sizeof(int32_t) * kMemoEntries * kMemoInts, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); war_index_destroy(ix); return WAR_ERR_CUDA; }
+    try { ix->bounds.assign(bounds, bounds + h.T + 1); } catch (...) { war_index_destroy(ix); return WAR_ERR_OOM; }
+    ix->M = h.M;
+    ix->T = h.T;
+    ix->publish();
+    *out = ix;
+    return WAR_OK;
 }
 
 extern "C" war_status_t war_index_info(const war_index_t* ix, war_index_info_t* out) {

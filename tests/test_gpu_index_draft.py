@@ -437,3 +437,37 @@ def test_memo_of_node_expansions_never_changes_an_answer(war):
     assert not all(np.array_equal(g, w) for g, w in zip(got, first[3]))   # the append did change the answers
     assert war.war_device_status() == 0
     ix.destroy()
+
+
+def test_export_and_import(war):
+    """An imported index answers exactly as the exported one, can be appended to, and bad buffers are refused."""
+    cfg = W.CONFIGS["tiny"]
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(W.scaled(cfg, B=24))
+    cut = cfg.n_traj - 9
+    ix = U.build_index(war, tok[:off[cut]], off[:cut + 1], cfg.vocab, max_depth=cfg.P + cfg.N)
+    buf = war.war_index_export(ix)
+    want = U.run_draft(war, ix, tails, tl, cfg.N, cfg.topk)
+    ix.destroy()
+    ix2 = war.war_index_import(buf, len(tok) + cfg.n_traj)
+    info = war.war_index_info(ix2)
+    assert info.T == cut and info.M == off[cut] + cut and info.capacity_tokens == len(tok) + cfg.n_traj
+    got = U.run_draft(war, ix2, tails, tl, cfg.N, cfg.topk)
+    for g, w in zip(got, want):
+        assert np.array_equal(g, w)
+    assert np.array_equal(war.war_index_export(ix2), buf)                  # a fixed point
+    war.war_index_append(ix2, torch.from_numpy(tok).to("cuda:0"), off[cut:])
+    _compare_with_oracle(war, tok, off, cfg.vocab, tails, tl, cfg.N, cfg.topk, ix=ix2)
+    ix2.destroy()
+    bad = buf.copy(); bad[0] ^= 0xFF                                       # magic
+    with pytest.raises(war.WarError):
+        war.war_index_import(bad, len(tok) + cfg.n_traj)
+    with pytest.raises(war.WarError):
+        war.war_index_import(buf[:len(buf) // 2], len(tok) + cfg.n_traj)   # truncated
+    with pytest.raises(war.WarError) as e:
+        war.war_index_import(buf, 10)                                      # does not fit
+    assert e.value.code == 3
+    empty = U.build_index(war, np.zeros(0, np.int32), np.zeros(1, np.int64), vocab=10, capacity=64)
+    ix3 = war.war_index_import(war.war_index_export(empty), 64)
+    assert war.war_index_info(ix3).M == 0
+    empty.destroy(); ix3.destroy()
