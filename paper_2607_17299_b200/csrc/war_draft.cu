@@ -220,6 +220,8 @@ struct Shared {
     int mode, cur, lo, cnt, depth, n_nodes, pool_n, thr_shared, long_runs_only, full_lo, full_cnt;
     int n_running, n_cap;
     int memo_slot;                              // >= 0: the node being expanded goes into this memo entry when it is done
+    // a batch of small nodes created in one round (equal counts), expanded by one warp each
+    int it_slot[kWarps], it_lo[kWarps], it_cnt[kWarps], it_depth[kWarps], n_items;
 };
 
 // Tokens from index `from` on of the suffix at s against the pattern; returns the sign and, in `matched`, how many
@@ -227,32 +229,38 @@ struct Shared {
 // overlap (the corpus has readable slack behind its last separator, and a separator always ends the walk).
 __device__ __forceinline__ int compare_suffix(const int32_t* __restrict__ corpus, int64_t s, const int* pat, int len, int from,
                                               int& matched) {
+    // Branch-free inside a batch: one bit per position for "differs" and one for "corpus token is smaller"; the first
+    // set bit decides.  (A chain of early exits costs a divergent branch per token on a path that is pure latency.)
     int t = from;
     {
+        unsigned ne = 0, lt = 0;
         int c[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) c[i] = corpus[s + t + i];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            if (t + i < len) {
-                const int p = pat[t + i];
-                if (c[i] != p) { matched = t + i; return c[i] < p ? -1 : 1; }
-            }
+            const int p = pat[min(t + i, len - 1)];
+            const bool in = t + i < len;
+            ne |= (unsigned)(in && c[i] != p) << i;
+            lt |= (unsigned)(c[i] < p) << i;
         }
+        if (ne) { const int f = __ffs(ne) - 1; matched = t + f; return (lt >> f) & 1u ? -1 : 1; }
         t += 8;
     }
     // most comparisons end above; the ones that go on share a long prefix, so fetch far ahead
     for (; t < len; t += 16) {
+        unsigned ne = 0, lt = 0;
         int c[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) c[i] = (t + i < len) ? corpus[s + t + i] : 0;
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-            if (t + i < len) {
-                const int p = pat[t + i];
-                if (c[i] != p) { matched = t + i; return c[i] < p ? -1 : 1; }
-            }
+            const int p = pat[min(t + i, len - 1)];
+            const bool in = t + i < len;
+            ne |= (unsigned)(in && c[i] != p) << i;
+            lt |= (unsigned)(c[i] < p) << i;
         }
+        if (ne) { const int f = __ffs(ne) - 1; matched = t + f; return (lt >> f) & 1u ? -1 : 1; }
     }
     matched = len;
     return 0;
@@ -433,6 +441,38 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         const int mode = sh.mode;
         if (mode == 0) break;
         const int lo = sh.lo, cnt = sh.cnt, d = sh.depth, hi = lo + cnt;
+        if (mode == 6) {
+            // A batch of small nodes: warp w expands item w in registers (one suffix per lane) and adds its k best
+            // continuations to the offer pool.
+            if (warp < sh.n_items) {
+                const int j = sh.it_slot[warp], ilo = sh.it_lo[warp], icnt = sh.it_cnt[warp], idp = sh.it_depth[warp];
+                const int tok = lane < icnt ? corpus[(int64_t)sa[ilo + lane] + idp] : -1;
+                const int prev_tok = __shfl_up_sync(0xffffffffu, tok, 1);
+                const bool real = lane < icnt && tok >= 0;
+                const bool head = real && (lane == 0 || tok != prev_tok);
+                const unsigned hm = __ballot_sync(0xffffffffu, head);
+                const unsigned vm = __ballot_sync(0xffffffffu, real);
+                const int end = vm ? 32 - __clz(vm) : 0;
+                const unsigned after = (hm >> 1) >> lane;
+                int c = head ? (after ? lane + __ffs(after) : end) - lane : 0;
+                int my_c = 0;
+                for (int r = 0; r < K; ++r) {
+                    const int key = __reduce_max_sync(0xffffffffu, c * 64 + (63 - lane));
+                    if (key < 64) break;
+                    if (lane == 63 - (key & 63)) { my_c = c; c = 0; }
+                }
+                const bool keep = my_c > 0 && (prob_num == 0 || (long long)my_c * prob_den >= (long long)prob_num * icnt);
+                const unsigned km = __ballot_sync(0xffffffffu, keep);
+                int base = 0;
+                if (lane == 0 && km) base = atomicAdd(&sh.pool_n, __popc(km));
+                base = __shfl_sync(0xffffffffu, base, 0);
+                if (keep) {
+                    const int at = base + __popc(km & ((1u << lane) - 1u));
+                    if (at < kPoolCap) { sh.pool_cnt[at] = my_c; sh.pool_par[at] = j; sh.pool_tok[at] = tok; sh.pool_lo[at] = ilo + lane; }
+                }
+            }
+            __syncthreads();
+        }
         if (mode == 2) {
             const int a0 = lo & ~15;
             int span = (hi - a0 + kWarps - 1) / kWarps;
@@ -452,6 +492,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         if (warp == 0) {
             const int cur = sh.cur;
             int n_fin = 0;
+            if (mode != 6) {
             if (mode == 4) {
                 n_fin = -1 - sh.memo_slot;                               // everything is in sh.fin_* already
             } else if (mode == 3) {
@@ -608,8 +649,14 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 __syncwarp();
                 if (lane == 0) sh.pool_n = min(kPoolCap, pn0 + __popc(km));
             }
+            }   // mode != 6
             __syncwarp();
             // ---- take the best offer: count desc, parent slot asc, token asc ----
+            // Offers that tie with the best one on the count follow it in exactly this order whatever their own
+            // continuations are (a continuation's count is not larger and its parent slot is newer), so all of them, up to
+            // one per warp, become slots now; if they are small nodes they are expanded together in the next round.
+            int n_items = 0, batch_c = 0;
+            while (true) {
             const int pn = sh.pool_n;
             int bi = -1, bc = -1, bp = 0, bt = 0;
             for (int i = lane; i < pn; i += 32) {
@@ -628,25 +675,37 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 bc = c_best; bp = p_best; bt = t_best;
             }
             // every lane now holds the same winner
-            if (bi < 0) {
+            if (bi < 0 || (n_items > 0 && bc != batch_c)) break;
+            const int j = sh.n_nodes;
+            const int slo = sh.pool_lo[bi];
+            const int depth = sh.slot_depth[bp] + 1;
+            __syncwarp();
+            if (lane == 0) {
+                const int last = pn - 1;
+                sh.pool_cnt[bi] = sh.pool_cnt[last]; sh.pool_par[bi] = sh.pool_par[last];
+                sh.pool_tok[bi] = sh.pool_tok[last]; sh.pool_lo[bi] = sh.pool_lo[last];
+                sh.pool_n = last;
+                o_ids[j] = bt; o_par[j] = bp;
+                if (o_cnt) o_cnt[j] = bc;
+                sh.slot_depth[j] = depth;
+                sh.n_nodes = j + 1;
+                sh.it_slot[n_items] = j; sh.it_lo[n_items] = slo; sh.it_cnt[n_items] = bc; sh.it_depth[n_items] = depth;
+            }
+            __syncwarp();
+            batch_c = bc;
+            ++n_items;
+            if (j + 1 >= sh.n_cap) { n_items = -1; break; }        // the budget is used up: nothing is expanded any more
+            if (bc > 32 || n_items == kWarps) break;              // large nodes go one at a time
+            }
+            // what the next round does
+            if (n_items <= 0) {
                 if (lane == 0) sh.mode = 0;
-            } else {
-                const int j = sh.n_nodes;
-                const int slo = sh.pool_lo[bi];
-                const int depth = sh.slot_depth[bp] + 1;
+            } else if (n_items == 1) {
+                if (lane == 0) sh.mode = 0;
                 __syncwarp();
-                if (lane == 0) {
-                    const int last = pn - 1;
-                    sh.pool_cnt[bi] = sh.pool_cnt[last]; sh.pool_par[bi] = sh.pool_par[last];
-                    sh.pool_tok[bi] = sh.pool_tok[last]; sh.pool_lo[bi] = sh.pool_lo[last];
-                    sh.pool_n = last;
-                    o_ids[j] = bt; o_par[j] = bp;
-                    if (o_cnt) o_cnt[j] = bc;
-                    sh.slot_depth[j] = depth;
-                    sh.n_nodes = j + 1;
-                    sh.mode = 0;
-                }
-                if (j + 1 < sh.n_cap) publish(j, slo, bc, depth);
+                publish(sh.it_slot[0], sh.it_lo[0], sh.it_cnt[0], sh.it_depth[0]);
+            } else {
+                if (lane == 0) { sh.n_items = n_items; sh.mode = 6; }
             }
         }
     }
