@@ -181,6 +181,80 @@ def build_draft_tree(corpus: Corpus, tail: np.ndarray, match_len: int, ends: np.
     return np.array(ids, np.int32), np.array(parent, np.int32), np.array(count, np.int32)
 
 
+def suffix_occurrences(corpus: Corpus, tail: np.ndarray, l: int) -> np.ndarray:
+    """Flat positions of the LAST token of every occurrence of the last l tokens of the tail (one plain scan per
+    token of the suffix, written on its own rather than through `longest_suffix_match`)."""
+    P = len(tail)
+    tok = corpus.tokens
+    ends = np.arange(len(tok), dtype=np.int64)
+    for i in range(l):                                    # token i counted from the end of the suffix
+        at = ends - i
+        ok = at >= corpus.start_of[ends]
+        ok[ok] = tok[at[ok]] == tail[P - 1 - i]
+        ends = ends[ok]
+    return ends
+
+
+def tree_score(count: np.ndarray) -> Tuple[int, int]:
+    """Score of a draft tree as an exact fraction (numerator, denominator) = (sum of the counts of slots 1.., count
+    of the root).  count(slot) / count(root) is the empirical probability that the text continues with the slot's
+    whole root path, so the fraction is the number of draft tokens one expects to be accepted if the continuation is
+    drawn from the occurrences of the matched string.  The SuffixDecoding method scores candidate trees by the sum
+    of such path probabilities (the product of the per-node probabilities along a path telescopes to this ratio)."""
+    return int(np.sum(count[1:], dtype=np.int64)), int(count[0])
+
+
+def draft_scored(corpus: Corpus, tail: np.ndarray, tail_len: int, N: int, k: int, n_lengths: int, min_match: int = 1,
+                 spec_factor=(0, 1), min_prob=(0, 1)):
+    """Draft from the best-scoring of several suffix lengths instead of from the longest match alone (a variant of
+    the SuffixDecoding method the paper adopts in Section 3.2; the paper itself does not spell it out).
+
+    Candidates are the lengths match_len, match_len - 1, ..., down n_lengths of them, never below max(1, min_match)
+    (every shorter suffix of an occurring string occurs too).  Each candidate gets its own tree by the rules of
+    `build_draft_tree` (its own root interval, its own node budget under spec_factor).  The tree with the largest
+    `tree_score` wins; fractions are compared exactly (cross-multiplied integers); equal scores go to the longer
+    suffix.  Returns (match_len, used_len, ids, parent, count): match_len is the longest match, used_len the
+    length the returned tree was built from."""
+    ml, _ = longest_suffix_match(corpus, tail, tail_len)
+    best = None
+    for c in range(max(1, n_lengths)):
+        l = ml - c
+        if c > 0 and l < max(1, min_match):
+            break
+        ends = suffix_occurrences(corpus, tail, l) if l > 0 else np.zeros(0, np.int64)
+        tree = build_draft_tree(corpus, tail, l, ends, N, k, min_match, spec_factor, min_prob)
+        num, den = tree_score(tree[2])
+        if best is None or num * best[1] > best[0] * den:          # strictly better only: ties keep the longer suffix
+            best = (num, den, l, tree)
+    _, _, used, (ids, parent, count) = best
+    return ml, used, ids, parent, count
+
+
+def draft_scored_batch(corpus: Corpus, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, n_lengths: int,
+                       min_match: int = 1, spec_batch_limit: int = 0, spec_factor=(0, 1), min_prob=(0, 1)):
+    """Batched `draft_scored` with the library's output convention and the same switch as `draft_batch`
+    (used_len is 0 wherever no tree is built)."""
+    B = tails.shape[0]
+    match_len = np.zeros(B, np.int32)
+    used_len = np.zeros(B, np.int32)
+    num_nodes = np.zeros(B, np.int32)
+    ids = np.full((B, N), -1, np.int32)
+    parent = np.full((B, N), -1, np.int32)
+    count = np.zeros((B, N), np.int32)
+    running = [i for i in range(B) if int(tail_len[i]) >= 0]
+    plain = spec_batch_limit > 0 and len(running) > spec_batch_limit
+    for i in running:
+        if plain:
+            num_nodes[i] = 1
+            ids[i, 0] = tails[i, -1]
+            continue
+        ml, used, a, b, c = draft_scored(corpus, tails[i], int(tail_len[i]), N, k, n_lengths, min_match, spec_factor, min_prob)
+        n = len(a)
+        match_len[i], used_len[i], num_nodes[i] = ml, used, n
+        ids[i, :n], parent[i, :n], count[i, :n] = a, b, c
+    return match_len, used_len, num_nodes, ids, parent, count
+
+
 def draft_batch(corpus: Corpus, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, min_match: int = 1,
                 spec_batch_limit: int = 0, spec_factor=(0, 1), min_prob=(0, 1)):
     """Batched form with the library's output convention: unused slots hold ids = -1, parent = -1, count = 0.

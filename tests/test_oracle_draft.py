@@ -283,3 +283,92 @@ def test_node_budget_and_probability_threshold():
         x = D.build_draft_tree(corpus, tail, ml, ends, 20, 3, spec_factor=(0, 1), min_prob=(0, 1))
         y = D.build_draft_tree(corpus, tail, ml, ends, 20, 3)
         assert all(np.array_equal(p, q) for p, q in zip(x, y))
+
+
+# ----------------------------------------------------------------------------------------------
+# drafting from the best-scoring of several suffix lengths
+# ----------------------------------------------------------------------------------------------
+
+def _mean_accepted_by_enumeration(tokens, offsets, s, ids, parent):
+    """Total number of draft tokens accepted when each occurrence of s in turn is taken as the true continuation
+    (walks the tree along the text; shares nothing with the checker's score)."""
+    children = {}
+    for j in range(1, len(ids)):
+        children.setdefault(int(parent[j]), {})[int(ids[j])] = j
+    total, occ = 0, _window_occurrences(tokens, offsets, s)
+    for t, p in occ:
+        tr = tokens[offsets[t]:offsets[t + 1]]
+        at, node = p + len(s), 0
+        while at < len(tr) and int(tr[at]) in children.get(node, {}):
+            node = children[node][int(tr[at])]
+            at += 1
+            total += 1
+    return total, len(occ)
+
+
+def test_scored_lengths_hand_worked_case():
+    g = _load("draft_scored_case1.json")
+    corpus = D.Corpus.from_lists(g["trajectories"])
+    tail = np.array(g["tail"], np.int32)
+    for l, want in g["candidates"].items():
+        ends = D.suffix_occurrences(corpus, tail, int(l))
+        ids, par, cnt = D.build_draft_tree(corpus, tail, int(l), ends, g["N"], g["k"])
+        assert (ids.tolist(), par.tolist(), cnt.tolist()) == (want["ids"], want["parent"], want["count"])
+        assert list(D.tree_score(cnt)) == want["score"]
+    for nl, used in g["used_len"].items():
+        ml, u, ids, par, cnt = D.draft_scored(corpus, tail, g["tail_len"], g["N"], g["k"], int(nl))
+        assert (ml, u) == (g["match_len"], used)
+        want = g["candidates"][str(used)]
+        assert (ids.tolist(), par.tolist(), cnt.tolist()) == (want["ids"], want["parent"], want["count"])
+    corpus2 = D.Corpus.from_lists(g["trajectories"][:-1])
+    assert D.draft_scored(corpus2, tail, 3, g["N"], g["k"], 3)[1] == g["without_last_trajectory"]["used_len"]["3"]
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_score_is_the_mean_accepted_length_and_the_best_one_wins(seed):
+    from fractions import Fraction
+    rng = np.random.default_rng(100 + seed)
+    V = int(rng.integers(2, 5))
+    trajs = [rng.integers(0, V, int(rng.integers(1, 40))).astype(np.int32) for _ in range(int(rng.integers(1, 7)))]
+    corpus = D.Corpus.from_lists(trajs)
+    P = 6
+    for _ in range(25):
+        tail = rng.integers(0, V, P).astype(np.int32)
+        tl = int(rng.integers(0, P + 1))
+        N, k, nl, mm = int(rng.integers(1, 12)), int(rng.integers(1, 4)), int(rng.integers(1, 7)), int(rng.integers(0, 3))
+        fac = (int(rng.integers(0, 3)), int(rng.integers(1, 3)))
+        ml, used, ids, par, cnt = D.draft_scored(corpus, tail, tl, N, k, nl, mm, spec_factor=fac)
+        assert ml == D.match_definitional(trajs, tail.tolist(), tl)
+        lens = [l for c, l in enumerate(range(ml, ml - nl, -1)) if c == 0 or l >= max(1, mm)]
+        assert used in lens
+        scores = {}
+        for l in lens:
+            s = tail[P - l:] if l > 0 else tail[:0]
+            ends = D.suffix_occurrences(corpus, tail, l) if l > 0 else np.zeros(0, np.int64)
+            assert len(ends) == (len(_window_occurrences(corpus.tokens, corpus.offsets, s)) if l > 0 else 0)
+            t_ids, t_par, t_cnt = D.build_draft_tree(corpus, tail, l, ends, N, k, mm, spec_factor=fac)
+            num, den = D.tree_score(t_cnt)
+            if l > 0:
+                assert (num, den) == _mean_accepted_by_enumeration(corpus.tokens, corpus.offsets, s, t_ids, t_par)
+            scores[l] = Fraction(num, den) if den else Fraction(0)
+            if l == used:
+                assert np.array_equal(t_ids, ids) and np.array_equal(t_par, par) and np.array_equal(t_cnt, cnt)
+        top = max(scores.values())
+        assert used == max(l for l in lens if scores[l] == top)
+
+
+def test_one_scored_length_is_the_plain_draft(tiny):
+    cfg, tok, off, tails, tl, _ = tiny
+    corpus = D.Corpus(tok, off)
+    a = D.draft_batch(corpus, tails, tl, cfg.N, cfg.topk)
+    b = D.draft_scored_batch(corpus, tails, tl, cfg.N, cfg.topk, 1)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(b[1], np.where(b[2] > 0, b[0], 0))
+    for x, y in zip(a[1:], b[2:]):
+        assert np.array_equal(x, y)
+    # more lengths never lower the score of the chosen tree
+    c = D.draft_scored_batch(corpus, tails, tl, cfg.N, cfg.topk, 4)
+    for i in range(len(tl)):
+        n1, d1 = D.tree_score(b[5][i, :b[2][i]])
+        n4, d4 = D.tree_score(c[5][i, :c[2][i]])
+        assert n4 * max(d1, 1) >= n1 * max(d4, 1)
+        assert c[0][i] == b[0][i] and c[1][i] <= c[0][i]
