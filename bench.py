@@ -138,6 +138,9 @@ def main():
     ap.add_argument("--spec-batch-limit", type=int, default=0,
                     help="workload-aware switch of war_draft: above this many running requests the step is a plain decode "
                          "step (root-only trees); 0 = always speculate")
+    ap.add_argument("--score-lengths", type=int, default=1,
+                    help="draft from the best-scoring of this many suffix lengths (war_draft_scored) instead of from the "
+                         "longest match (war_draft); 1 = war_draft, the configuration the metric is quoted on")
     ap.add_argument("--requests", type=int, default=0,
                     help="run the workload's recipe with this many requests instead of its own count (profiling-size cases)")
     args = ap.parse_args()
@@ -262,11 +265,23 @@ def main():
 
     # targets depend on the trees; the trees are a deterministic function of the inputs, so draft once to make them
     # (this is also the first draft call on the freshly published index: its memo of large-node expansions is empty)
+    if args.score_lengths > 1:
+        d_used = torch.zeros(cfg.B, dtype=torch.int32, device=dev)
+        draft_ws = torch.empty(war.war_draft_scored_workspace_bytes(cfg.B, cfg.P, N, cfg.topk, args.score_lengths),
+                               dtype=torch.uint8, device=dev)
+
+    def draft():
+        if args.score_lengths > 1:
+            war.war_draft_scored(ix, d_tails, d_tl, N, cfg.topk, 1, args.score_lengths, draft_ws, d_ml, d_used, d_nn, d_ids,
+                                 d_par, d_cnt, args.spec_batch_limit)
+        else:
+            war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt, args.spec_batch_limit)
+
     ev = lambda: torch.cuda.Event(enable_timing=True)
     cold0, cold1 = ev(), ev()
     torch.cuda.synchronize()
     cold0.record()
-    war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt, args.spec_batch_limit)
+    draft()
     cold1.record()
     torch.cuda.synchronize()
     draft_cold_ms = cold0.elapsed_time(cold1)
@@ -275,7 +290,7 @@ def main():
     d_target = torch.from_numpy(targets).to(dev)
 
     def step(attn_events=None):
-        war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt, args.spec_batch_limit)
+        draft()
         if attn_events is not None:
             attn_events[0].record()
         war.war_verify_attn(attn.q, attn.k_pool, attn.v_pool, attn.page_table, attn.prefix_len, d_nn, d_par, params, ws,
@@ -345,7 +360,7 @@ def main():
         else:
             attn.q.copy_(h_q, non_blocking=True)
         d_target.copy_(h_target, non_blocking=True)
-        war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, d_ml, d_nn, d_ids, d_par, d_cnt, args.spec_batch_limit)
+        draft()
         if overlap_q:
             main_stream.wait_event(q_ready)
         war.war_verify_attn(attn.q, attn.k_pool, attn.v_pool, attn.page_table, attn.prefix_len, d_nn, d_par, params, ws,
@@ -422,11 +437,12 @@ def main():
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": dict(base_config, kernel="tcgen05" if args.kernel == 0 else "cuda-core",
-                           **({"spec_batch_limit": args.spec_batch_limit} if args.spec_batch_limit else {})),
+                           **({"spec_batch_limit": args.spec_batch_limit} if args.spec_batch_limit else {}),
+                           **({"score_lengths": args.score_lengths} if args.score_lengths > 1 else {})),
             "clocks": clocks.summary(),
             "e2e": {"value": verified_all / (e2e_ms / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
-            "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+            "gpu_launches": (LAUNCHES_PER_STEP + (args.score_lengths > 1)) * args.steps,
             "roofline": ({"bound": "tensor", "achieved": flops / (attn_ms * 1e-3) / 1e12, "peak": peak_tf, "unit": "TFLOP/s",
                           "frac": t_tensor / (attn_ms * 1e-3), "traffic": traffic, "flops_per_launch": flops,
                           "peak_source": "measured (MEASURED_PEAKS.json bf16_tflops_sustained)" if os.path.exists(peaks_path) else "fallback",

@@ -10,6 +10,7 @@
  *
  *   war_index_build / war_index_append   the trajectory cache: suffix array + capped LCP over the corpus
  *   war_draft                            longest-suffix match + frequency-ranked draft token tree
+ *   war_draft_scored                     the same from the best-scoring of several suffix lengths
  *   war_verify_attn                      tree-masked GQA decode attention over a paged bf16 KV cache
  *   war_accept                           longest root path of the tree that equals the target's tokens
  *   war_commit                           the accepted tokens become context: KV rows, prefix length, tail window
@@ -158,6 +159,28 @@ war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, const int32
                        const war_draft_params_t* params,
                        int32_t* d_match_len, int32_t* d_num_nodes,
                        int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream);
+
+/* Drafting from the best-scoring of several suffix lengths (a variant of the SuffixDecoding method that Section 3.2
+ * adopts; the paper does not spell it out).  Candidates are the suffix lengths match_len, match_len - 1, ...,
+ * n_lengths of them (1 <= n_lengths <= 32), never below max(1, min_match); every shorter suffix of an occurring
+ * string occurs too, usually more often.  Each candidate gets its own tree by the rules of war_draft (its own root
+ * interval, its own slot budget under spec_factor).  A tree's score is
+ *     (sum of count[j], j = 1 .. num_nodes-1) / count[0]
+ * = the sum over its slots of the empirical probability that the text continues with the slot's whole root path
+ * = the number of draft tokens one expects to be accepted when the continuation is drawn from the occurrences of
+ * the suffix.  The tree with the largest score is returned; scores are compared exactly (cross-multiplied 64-bit
+ * integers); equal scores go to the longer suffix.  d_match_len [B] receives the longest match as in war_draft,
+ * d_used_len [B] the length the returned tree was built from (0 where no tree was built).  With n_lengths = 1 the
+ * outputs equal war_draft's.  The switch and the thresholds act as in war_draft.
+ * Candidates run as separate thread blocks (B * n_lengths of them), so scoring costs no latency while the GPU
+ * has idle SMs, which is when speculation is on.  d_workspace: device memory of
+ * war_draft_scored_workspace_bytes(params, n_lengths) bytes (0 for invalid arguments), 4-byte aligned, owned by the
+ * caller, overwritten by every call.  Nothing is allocated; the call can be captured in a CUDA graph. */
+size_t war_draft_scored_workspace_bytes(const war_draft_params_t* params, int32_t n_lengths);
+war_status_t war_draft_scored(const war_index_t* ix, const int32_t* d_tail, const int32_t* d_tail_len,
+                              const war_draft_params_t* params, int32_t n_lengths, void* d_workspace,
+                              int32_t* d_match_len, int32_t* d_used_len, int32_t* d_num_nodes,
+                              int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Verification attention (paper Section 3.2: the predicted tokens "are then verified by the target model"

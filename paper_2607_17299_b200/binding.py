@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "WAR_OK", 1: "WAR_ERR_INVALID_ARG", 2: "WAR_ERR_OOM", 3: "WAR
                 5: "WAR_ERR_TIMEOUT", 6: "WAR_ERR_UNSUPPORTED", 7: "WAR_ERR_BAD_TREE", 8: "WAR_ERR_BAD_PAGE"}
 
 EXPORTS = ["war_index_build", "war_index_append", "war_index_evict", "war_index_export_bytes", "war_index_export",
-           "war_index_import", "war_index_info", "war_index_destroy", "war_draft",
+           "war_index_import", "war_index_info", "war_index_destroy", "war_draft", "war_draft_scored_workspace_bytes", "war_draft_scored",
            "war_verify_attn_workspace_bytes", "war_verify_attn", "war_verify_attn_noalloc", "war_accept", "war_commit", "war_device_status",
            "war_status_string"]
 
@@ -78,6 +78,10 @@ _lib.war_index_destroy.argtypes = [C.c_void_p]
 _lib.war_draft.restype = C.c_int
 _lib.war_draft.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(DraftParams)] + [C.c_void_p] * 6
 _lib.war_verify_attn_workspace_bytes.restype = C.c_size_t
+_lib.war_draft_scored_workspace_bytes.restype = C.c_size_t
+_lib.war_draft_scored_workspace_bytes.argtypes = [C.POINTER(DraftParams), C.c_int32]
+_lib.war_draft_scored.restype = C.c_int
+_lib.war_draft_scored.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(DraftParams), C.c_int32] + [C.c_void_p] * 8
 _lib.war_verify_attn_workspace_bytes.argtypes = [C.POINTER(AttnParams)]
 _lib.war_verify_attn.restype = C.c_int
 _lib.war_verify_attn.argtypes = [C.c_void_p] * 7 + [C.POINTER(AttnParams)] + [C.c_void_p] * 4
@@ -197,6 +201,29 @@ def war_draft(ix: Index, d_tail: torch.Tensor, d_tail_len: torch.Tensor, N: int,
                           _ptr(d_match_len, torch.int32), _ptr(d_num_nodes, torch.int32), _ptr(d_ids, torch.int32),
                           _ptr(d_parent, torch.int32), _ptr(d_count, torch.int32), _stream())
     _check("war_draft", code)
+
+
+def war_draft_scored_workspace_bytes(B: int, P: int, N: int, topk: int, n_lengths: int) -> int:
+    p = DraftParams(B, P, N, topk, 1, 0, 0, 1, 0, 1)
+    return int(_lib.war_draft_scored_workspace_bytes(C.byref(p), n_lengths))
+
+
+def war_draft_scored(ix: Index, d_tail: torch.Tensor, d_tail_len: torch.Tensor, N: int, topk: int, min_match: int,
+                     n_lengths: int, d_workspace: torch.Tensor, d_match_len: torch.Tensor, d_used_len: torch.Tensor,
+                     d_num_nodes: torch.Tensor, d_ids: torch.Tensor, d_parent: torch.Tensor, d_count: Optional[torch.Tensor],
+                     spec_batch_limit: int = 0, spec_factor=(0, 1), min_prob=(0, 1)) -> None:
+    """war_draft from the best-scoring of n_lengths suffix lengths; d_workspace is a uint8 CUDA tensor of at least
+    war_draft_scored_workspace_bytes(...) bytes."""
+    B, P = d_tail.shape
+    p = DraftParams(B, P, N, topk, min_match, spec_batch_limit, spec_factor[0], spec_factor[1], min_prob[0], min_prob[1])
+    need = int(_lib.war_draft_scored_workspace_bytes(C.byref(p), n_lengths))
+    if need == 0 or d_workspace.dtype != torch.uint8 or not d_workspace.is_cuda or d_workspace.numel() < need:
+        raise ValueError("workspace must be a uint8 CUDA tensor of war_draft_scored_workspace_bytes bytes")
+    code = _lib.war_draft_scored(ix.handle, _ptr(d_tail, torch.int32), _ptr(d_tail_len, torch.int32), C.byref(p), n_lengths,
+                                 d_workspace.data_ptr(), _ptr(d_match_len, torch.int32), _ptr(d_used_len, torch.int32),
+                                 _ptr(d_num_nodes, torch.int32), _ptr(d_ids, torch.int32), _ptr(d_parent, torch.int32),
+                                 _ptr(d_count, torch.int32), _stream())
+    _check("war_draft_scored", code)
 
 
 def attn_params(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, page_table: torch.Tensor, scale: float,

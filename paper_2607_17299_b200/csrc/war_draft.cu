@@ -271,13 +271,18 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                  const int32_t* __restrict__ bucket, int32_t* memo, int vocab, const int32_t* __restrict__ tail,
                  const int32_t* __restrict__ tail_len, int B, int P, int N, int K, int min_match, int spec_batch_limit,
                  int fac_num, int fac_den, int prob_num, int prob_den, int32_t* __restrict__ match_len, int32_t* __restrict__ num_nodes, int32_t* __restrict__ ids,
-                 int32_t* __restrict__ parent, int32_t* __restrict__ count) {
+                 int32_t* __restrict__ parent, int32_t* __restrict__ count, int32_t* __restrict__ cand_len) {
     __shared__ Shared sh;
     const int b = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    int32_t* o_ids = ids + (size_t)b * N;
-    int32_t* o_par = parent + (size_t)b * N;
-    int32_t* o_cnt = count ? count + (size_t)b * N : nullptr;
+    // Scoring several suffix lengths: CTA (b, c) drafts request b from the suffix that is c tokens shorter than the
+    // longest match and leaves its tree in row b * gridDim.y + c of the candidate arrays (all output pointers then
+    // address those); a second kernel picks the winner.  With one candidate per request the row is the request.
+    const int cand = blockIdx.y;
+    const size_t row = (size_t)b * gridDim.y + cand;
+    int32_t* o_ids = ids + row * N;
+    int32_t* o_par = parent + row * N;
+    int32_t* o_cnt = count ? count + row * N : nullptr;
 
     if (tid < P) sh.pat[tid] = tail[(size_t)b * P + tid];
     // Workload-aware switch: a request with tail_len < 0 is not running; when more requests run than the limit,
@@ -300,7 +305,8 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
     if (my_tl < 0 || plain) {
         const int n = my_tl < 0 ? 0 : 1;
         if (tid == 0) {
-            match_len[b] = 0; num_nodes[b] = n;
+            match_len[row] = 0; num_nodes[row] = n;
+            if (cand_len) cand_len[row] = cand == 0 ? 0 : -1;            // one candidate: the root alone (or nothing)
             if (n) { o_ids[0] = sh.pat[P - 1]; o_par[0] = -1; if (o_cnt) o_cnt[0] = 0; }
         }
         for (int j = n + tid; j < N; j += kThreads) {
@@ -382,7 +388,13 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             }
         }
         const unsigned found = __ballot_sync(0xffffffffu, occurs);
-        const int ml = found ? 32 - __clz(found) : 0;
+        const int ml_longest = found ? 32 - __clz(found) : 0;
+        // candidate c drafts from the suffix of ml_longest - c tokens (every shorter suffix of an occurring string
+        // occurs, and its lane holds that suffix's lower bound); lengths below max(1, min_match) are no candidates
+        const int ml = ml_longest - cand;
+        if (cand > 0 && ml < max(1, min_match)) {
+            if (lane == 0) { match_len[row] = ml_longest; cand_len[row] = -1; sh.n_nodes = 0; sh.mode = 0; }
+        } else {
         const int src = ml > 0 ? ml - 1 : 0;
         lo = __shfl_sync(0xffffffffu, lo, src);
         bucket_hi = __shfl_sync(0xffffffffu, bucket_hi, src);
@@ -423,7 +435,8 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         const bool expand = ml >= max(1, min_match) && n_cap > 1;
         if (lane == 0) {
             sh.n_cap = n_cap;
-            match_len[b] = ml;
+            match_len[row] = ml_longest;
+            if (cand_len) cand_len[row] = ml;
             o_ids[0] = sh.pat[P - 1];
             o_par[0] = -1;
             if (o_cnt) o_cnt[0] = c0;
@@ -433,6 +446,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             sh.mode = 0;
         }
         if (expand) publish(0, lo, c0, ml);
+        }
     }
 
     // ---- best-first expansion ----
@@ -710,24 +724,117 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         }
     }
     const int n = sh.n_nodes;
-    if (tid == 0) num_nodes[b] = n;
+    if (tid == 0) num_nodes[row] = n;
     for (int j = n + tid; j < N; j += kThreads) {
         o_ids[j] = -1; o_par[j] = -1;
         if (o_cnt) o_cnt[j] = 0;
     }
 }
 
+// Candidate arrays of the scored draft, all int32, in the caller's workspace.
+struct CandArrays {
+    int32_t *len, *match_len, *num_nodes, *ids, *parent, *count;
+};
+__host__ __device__ inline CandArrays cand_layout(void* base, size_t rows, int N) {
+    CandArrays c;
+    int32_t* p = (int32_t*)base;
+    c.len = p; p += rows;
+    c.match_len = p; p += rows;
+    c.num_nodes = p; p += rows;
+    c.ids = p; p += rows * N;
+    c.parent = p; p += rows * N;
+    c.count = p;
+    return c;
+}
+
+// Picks, per request, the candidate tree with the largest score = (sum of the counts of slots 1..) / (count of the
+// root), compared exactly by cross-multiplication; equal scores go to the longer suffix (the smaller candidate index).
+// One warp per request, one lane per candidate.
+__global__ void __launch_bounds__(256)
+war_draft_select_kernel(CandArrays ca, int B, int C, int N, int32_t* __restrict__ match_len, int32_t* __restrict__ used_len,
+                        int32_t* __restrict__ num_nodes, int32_t* __restrict__ ids, int32_t* __restrict__ parent,
+                        int32_t* __restrict__ count) {
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (b >= B) return;
+    const size_t row = (size_t)b * C + lane;
+    int len = -1, n = 0, den = 0, best = lane;
+    long long num = 0;
+    if (lane < C) {
+        len = ca.len[row];
+        if (len >= 0) {
+            n = ca.num_nodes[row];
+            den = n > 0 ? ca.count[row * N] : 0;
+            for (int j = 1; j < n; ++j) num += ca.count[row * N + j];
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const int o_len = __shfl_xor_sync(0xffffffffu, len, o), o_den = __shfl_xor_sync(0xffffffffu, den, o);
+        const int o_best = __shfl_xor_sync(0xffffffffu, best, o);
+        const long long o_num = __shfl_xor_sync(0xffffffffu, num, o);
+        bool take;
+        if (o_len < 0) take = false;
+        else if (len < 0) take = true;
+        else {
+            const long long l = o_num * den, r = num * o_den;            // o_num / o_den against num / den
+            take = l > r || (l == r && o_best < best);
+        }
+        if (take) { len = o_len; den = o_den; num = o_num; best = o_best; }
+    }
+    // every lane holds the winner (candidate 0 is always valid)
+    const size_t win = (size_t)b * C + best;
+    const int wn = ca.num_nodes[win];
+    if (lane == 0) { match_len[b] = ca.match_len[(size_t)b * C]; used_len[b] = max(len, 0); num_nodes[b] = wn; }
+    for (int j = lane; j < N; j += 32) {
+        ids[(size_t)b * N + j] = ca.ids[win * N + j];
+        parent[(size_t)b * N + j] = ca.parent[win * N + j];
+        if (count) count[(size_t)b * N + j] = ca.count[win * N + j];
+    }
+}
+
+bool draft_params_ok(const war_index_t* ix, const war_draft_params_t* p) {
+    if (p->B < 0 || p->P < 1 || p->P > kMaxP || p->N < 1 || p->N > kMaxN || p->topk < 1 || p->topk > kMaxK || p->min_match < 0 ||
+        p->spec_batch_limit < 0 || p->spec_factor_num < 0 || (p->spec_factor_num > 0 && p->spec_factor_den < 1) ||
+        p->min_prob_num < 0 || (p->min_prob_num > 0 && (p->min_prob_den < 1 || p->min_prob_num > p->min_prob_den)))
+        return false;
+    return p->P + p->N <= ix->max_depth;                            // else the index is not ordered deep enough
+}
+
 }  // namespace
+
+extern "C" size_t war_draft_scored_workspace_bytes(const war_draft_params_t* p, int32_t n_lengths) {
+    if (!p || p->B < 0 || p->N < 1 || p->N > kMaxN || n_lengths < 1 || n_lengths > kMaxP) return 0;
+    const size_t rows = (size_t)p->B * n_lengths;
+    return sizeof(int32_t) * (3 * rows + 3 * rows * p->N) + 256;
+}
+
+extern "C" war_status_t war_draft_scored(const war_index_t* ix, const int32_t* d_tail, const int32_t* d_tail_len,
+                                         const war_draft_params_t* p, int32_t n_lengths, void* d_workspace,
+                                         int32_t* d_match_len, int32_t* d_used_len, int32_t* d_num_nodes, int32_t* d_ids,
+                                         int32_t* d_parent, int32_t* d_count, war_stream_t stream) {
+    if (!ix || !p) return WAR_ERR_INVALID_ARG;
+    if (!draft_params_ok(ix, p) || n_lengths < 1 || n_lengths > kMaxP) return WAR_ERR_INVALID_ARG;
+    if (p->B == 0) return WAR_OK;
+    if (!d_tail || !d_tail_len || !d_workspace || !d_match_len || !d_used_len || !d_num_nodes || !d_ids || !d_parent)
+        return WAR_ERR_INVALID_ARG;
+    const war_index_arrays arr = const_cast<war_index_t*>(ix)->published();
+    const CandArrays ca = cand_layout(d_workspace, (size_t)p->B * n_lengths, p->N);
+    war_draft_kernel<<<dim3(p->B, n_lengths), kThreads, 0, stream>>>(
+        ix->corpus, arr.sa, arr.lcp, arr.bucket, arr.memo, ix->vocab, d_tail, d_tail_len, p->B, p->P, p->N, p->topk, p->min_match,
+        p->spec_batch_limit, p->spec_factor_num, p->spec_factor_num > 0 ? p->spec_factor_den : 1, p->min_prob_num,
+        p->min_prob_num > 0 ? p->min_prob_den : 1, ca.match_len, ca.num_nodes, ca.ids, ca.parent, ca.count, ca.len);
+    WAR_LAUNCH_CHECK();
+    war_draft_select_kernel<<<(p->B + 7) / 8, 256, 0, stream>>>(ca, p->B, n_lengths, p->N, d_match_len, d_used_len, d_num_nodes,
+                                                              d_ids, d_parent, d_count);
+    WAR_LAUNCH_CHECK();
+    return WAR_OK;
+}
 
 extern "C" war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, const int32_t* d_tail_len,
                                   const war_draft_params_t* p, int32_t* d_match_len, int32_t* d_num_nodes,
                                   int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream) {
     if (!ix || !p) return WAR_ERR_INVALID_ARG;
-    if (p->B < 0 || p->P < 1 || p->P > kMaxP || p->N < 1 || p->N > kMaxN || p->topk < 1 || p->topk > kMaxK || p->min_match < 0 ||
-        p->spec_batch_limit < 0 || p->spec_factor_num < 0 || (p->spec_factor_num > 0 && p->spec_factor_den < 1) ||
-        p->min_prob_num < 0 || (p->min_prob_num > 0 && (p->min_prob_den < 1 || p->min_prob_num > p->min_prob_den)))
-        return WAR_ERR_INVALID_ARG;
-    if (p->P + p->N > ix->max_depth) return WAR_ERR_INVALID_ARG;     // the index is not ordered deep enough
+    if (!draft_params_ok(ix, p)) return WAR_ERR_INVALID_ARG;
     if (p->B == 0) return WAR_OK;
     if (!d_tail || !d_tail_len || !d_match_len || !d_num_nodes || !d_ids || !d_parent) return WAR_ERR_INVALID_ARG;
     const war_index_arrays arr = const_cast<war_index_t*>(ix)->published();       // a complete index, also during an update
@@ -735,7 +842,7 @@ extern "C" war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, 
                                                    p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, p->spec_factor_num,
                                                    p->spec_factor_num > 0 ? p->spec_factor_den : 1, p->min_prob_num,
                                                    p->min_prob_num > 0 ? p->min_prob_den : 1, d_match_len,
-                                                   d_num_nodes, d_ids, d_parent, d_count);
+                                                   d_num_nodes, d_ids, d_parent, d_count, nullptr);
     WAR_LAUNCH_CHECK();
     return WAR_OK;
 }

@@ -31,6 +31,26 @@ def run_draft(war, ix, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, 
     return out
 
 
+def run_draft_scored(war, ix, tails: np.ndarray, tail_len: np.ndarray, N: int, k: int, n_lengths: int, min_match: int = 1,
+                     with_count=True, spec_batch_limit: int = 0, spec_factor=(0, 1), min_prob=(0, 1)):
+    """Returns [match_len, used_len, num_nodes, ids, parent, count] as numpy arrays."""
+    B, P = tails.shape
+    d = dev()
+    t = torch.from_numpy(np.ascontiguousarray(tails, dtype=np.int32)).to(d)
+    tl = torch.from_numpy(np.ascontiguousarray(tail_len, dtype=np.int32)).to(d)
+    ws = torch.full((max(1, war.war_draft_scored_workspace_bytes(B, P, N, k, n_lengths)),), 0x5a, dtype=torch.uint8, device=d)
+    ml, ul, nn = (torch.full((B,), -7, dtype=torch.int32, device=d) for _ in range(3))
+    ids = torch.full((B, N), -7, dtype=torch.int32, device=d)
+    par = torch.full((B, N), -7, dtype=torch.int32, device=d)
+    cnt = torch.full((B, N), -7, dtype=torch.int32, device=d) if with_count else None
+    war.war_draft_scored(ix, t, tl, N, k, min_match, n_lengths, ws, ml, ul, nn, ids, par, cnt, spec_batch_limit, spec_factor,
+                         min_prob)
+    torch.cuda.synchronize()
+    out = [x.cpu().numpy() for x in (ml, ul, nn, ids, par)]
+    out.append(cnt.cpu().numpy() if with_count else None)
+    return out
+
+
 def run_attn(war, a, num_nodes: np.ndarray, parent: np.ndarray, scale: float, kernel: int = 0, fill: float = 7.0):
     """`a` is workloads.AttnInputs already on the device.  Returns (out fp32 numpy [B,N,Hq,D], lse numpy [B,N,Hq])."""
     d = dev()

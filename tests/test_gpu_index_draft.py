@@ -471,3 +471,94 @@ def test_export_and_import(war):
     ix3 = war.war_index_import(war.war_index_export(empty), 64)
     assert war.war_index_info(ix3).M == 0
     empty.destroy(); ix3.destroy()
+
+
+# ----------------------------------------------------------------------------------------------
+# drafting from the best-scoring of several suffix lengths
+# ----------------------------------------------------------------------------------------------
+
+def _compare_scored(war, ix, corpus, tails, tl, N, k, n_lengths, **kw):
+    got = U.run_draft_scored(war, ix, tails, tl, N, k, n_lengths, **kw)
+    want = D.draft_scored_batch(corpus, tails, tl, N, k, n_lengths, **kw)
+    for name, g, w in zip(["match_len", "used_len", "num_nodes", "ids", "parent", "count"], got, want):
+        assert np.array_equal(g, w), f"{name} differs at request(s) {np.flatnonzero((g != w).reshape(len(g), -1).any(axis=1))[:8]}"
+    assert war.war_device_status() == 0
+    return got
+
+
+def test_scored_lengths_hand_worked_case(war):
+    with open(os.path.join(GOLD, "draft_scored_case1.json")) as f:
+        g = json.load(f)
+    tok, off = _flat(g["trajectories"])
+    ix = U.build_index(war, tok, off, vocab=10)
+    tails = np.array([g["tail"]], np.int32)
+    tl = np.array([g["tail_len"]], np.int32)
+    for nl, used in g["used_len"].items():
+        ml, ul, nn, ids, par, cnt = U.run_draft_scored(war, ix, tails, tl, g["N"], g["k"], int(nl))
+        want = g["candidates"][str(used)]
+        n = len(want["ids"])
+        assert (ml[0], ul[0], nn[0]) == (g["match_len"], used, n)
+        assert (ids[0, :n].tolist(), par[0, :n].tolist(), cnt[0, :n].tolist()) == (want["ids"], want["parent"], want["count"])
+        assert (ids[0, n:] == -1).all() and (par[0, n:] == -1).all() and (cnt[0, n:] == 0).all()
+    ix.destroy()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_scored_lengths_on_tiny_alphabets(war, seed):
+    """Few symbols: every suffix length has many occurrences, scores tie often, every rule of the choice is exercised."""
+    rng = np.random.default_rng(300 + seed)
+    vocab = int(rng.integers(2, 6))
+    trajs = [rng.integers(0, vocab, size=int(rng.integers(0, 200))).tolist() for _ in range(int(rng.integers(1, 9)))]
+    tok, off = _flat(trajs)
+    P = int(rng.integers(1, 33))
+    N = int(rng.integers(1, 65))
+    k = int(rng.integers(1, 9))
+    B = 24
+    tails = rng.integers(0, vocab + 1, size=(B, P)).astype(np.int32)
+    tails[0, :] = -1
+    tl = rng.integers(-1, P + 1, size=B).astype(np.int32)              # -1: not running
+    ix = U.build_index(war, tok, off, vocab + 1)
+    corpus = D.Corpus(tok, off)
+    for nl in (1, 2, 5, 32):
+        _compare_scored(war, ix, corpus, tails, tl, N, k, nl, min_match=int(rng.integers(0, 4)),
+                        spec_factor=(int(rng.integers(0, 3)), int(rng.integers(1, 4))),
+                        min_prob=(int(rng.integers(0, 2)), int(rng.integers(2, 6))))
+    ix.destroy()
+
+
+def test_scored_lengths_on_the_tiny_workload(war):
+    cfg = W.CONFIGS["tiny"]
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(W.scaled(cfg, B=40))
+    ix = U.build_index(war, tok, off, cfg.vocab, max_depth=cfg.P + 64)
+    corpus = D.Corpus(tok, off)
+    one = U.run_draft_scored(war, ix, tails, tl, cfg.N, cfg.topk, 1)
+    plain = U.run_draft(war, ix, tails, tl, cfg.N, cfg.topk)
+    assert np.array_equal(one[0], plain[0]) and all(np.array_equal(a, b) for a, b in zip(one[2:], plain[1:]))
+    picked_shorter = 0
+    for nl, N, k in ((4, cfg.N, cfg.topk), (8, 64, 8), (3, 2, 1)):
+        got = _compare_scored(war, ix, corpus, tails, tl, N, k, nl)
+        picked_shorter += int((got[1] < got[0]).sum())
+    assert picked_shorter > 0                                           # the choice is not always the longest match
+    # the switch: over the limit nothing is looked up
+    got = _compare_scored(war, ix, corpus, tails, tl, cfg.N, cfg.topk, 4, spec_batch_limit=8)
+    assert (got[2] == 1).all() and (got[1] == 0).all()
+    # no count output
+    nc = U.run_draft_scored(war, ix, tails, tl, cfg.N, cfg.topk, 4, with_count=False)
+    ref = U.run_draft_scored(war, ix, tails, tl, cfg.N, cfg.topk, 4)
+    assert all(np.array_equal(a, b) for a, b in zip(nc[:5], ref[:5]))
+    ix.destroy()
+
+
+def test_scored_lengths_argument_checks(war):
+    tok, off = _flat([[1, 2, 3, 1, 2, 3]])
+    ix = U.build_index(war, tok, off, vocab=4)
+    assert war.war_draft_scored_workspace_bytes(4, 8, 8, 2, 0) == 0
+    assert war.war_draft_scored_workspace_bytes(4, 8, 8, 2, 33) == 0
+    assert war.war_draft_scored_workspace_bytes(4, 8, 8, 2, 3) >= 4 * (3 * 12 + 3 * 12 * 8)
+    tails = np.array([[1, 2, 3]], np.int32)
+    with pytest.raises(ValueError):
+        U.run_draft_scored(war, ix, tails, np.array([3], np.int32), 8, 2, 0)
+    got = U.run_draft_scored(war, ix, np.zeros((0, 3), np.int32), np.zeros(0, np.int32), 8, 2, 2)      # B = 0
+    assert got[0].shape == (0,)
+    ix.destroy()
