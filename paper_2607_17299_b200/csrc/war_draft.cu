@@ -328,13 +328,22 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         if (cnt >= kMemoMinCount) {
             const unsigned long long key = ((unsigned long long)(unsigned)(lo + 1) << 16) | ((unsigned long long)depth << 8) | (unsigned)K;
             unsigned h = (unsigned)(key * 0x9E3779B97F4A7C15ull >> 40) & (kMemoEntries - 1);
+            // One coalesced read of the whole 128-byte entry (plus the key as one 64-bit word on lane 0).  Payload
+            // words are stored with 1 added and the table starts zeroed, so every word says by itself whether it has
+            // been written: a hit needs the key and all words it uses to be there, in whatever order they arrived.
             volatile int32_t* en = memo + (size_t)h * kMemoInts;
-            const unsigned long long got = *(volatile unsigned long long*)en;
+            unsigned long long got = 0ull;
+            if (lane == 0) got = *(volatile unsigned long long*)en;
+            const int word = en[lane];
+            got = __shfl_sync(0xffffffffu, got, 0);
             if (got == key) {
-                if (en[2] == 2) {                                        // ready: the payload was written before the state
-                    __threadfence();
-                    const int n_fin = en[3];
-                    if (lane < kMaxK) { sh.fin_cnt[lane] = en[4 + lane]; sh.fin_start[lane] = en[12 + lane]; sh.fin_tok[lane] = en[20 + lane]; }
+                const int n_fin = __shfl_sync(0xffffffffu, word, 3) - 1;
+                const bool mine = lane >= 4 && lane < 28 && ((lane - 4) & 7) < n_fin;      // a word this node's answer uses
+                if (n_fin >= 0 && __ballot_sync(0xffffffffu, mine && word == 0) == 0u) {
+                    if (mine) {
+                        int* dst = lane < 12 ? sh.fin_cnt : lane < 20 ? sh.fin_start : sh.fin_tok;
+                        dst[(lane - 4) & 7] = word - (lane < 12 ? 0 : 1);
+                    }
                     if (lane == 0) {
                         sh.cur = slot; sh.lo = lo; sh.cnt = cnt; sh.depth = depth; sh.full_lo = lo; sh.full_cnt = cnt;
                         sh.long_runs_only = 0; sh.thr_shared = 0; sh.memo_slot = -1 - n_fin; sh.mode = 4;
@@ -376,9 +385,15 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                     // lower bound by binary search; it remembers how many tokens the pattern shares with the suffixes
                     // at its current ends, so comparisons restart there (all bucket members share token 0)
                     int a = lo, z = bucket_hi, ma = 1, mz = 1, m;
+                    // The suffix-array entries of both possible next probes are requested together with this probe's
+                    // corpus tokens, so a step costs one memory latency, not two.
+                    int mid = a + ((z - a) >> 1);
+                    int s_mid = sa[mid];                         // the bucket is not empty
                     while (a < z) {                              // first suffix >= pattern
-                        const int mid = a + ((z - a) >> 1);
-                        if (compare_suffix(corpus, sa[mid], pat, len, min(ma, mz), m) < 0) { a = mid + 1; ma = m; } else { z = mid; mz = m; }
+                        const int mid_l = a + ((mid - a) >> 1), mid_r = mid + 1 + ((z - mid - 1) >> 1);
+                        const int s_l = a < mid ? sa[mid_l] : 0, s_r = mid + 1 < z ? sa[mid_r] : 0;
+                        if (compare_suffix(corpus, s_mid, pat, len, min(ma, mz), m) < 0) { a = mid + 1; ma = m; mid = mid_r; s_mid = s_r; }
+                        else { z = mid; mz = m; mid = mid_l; s_mid = s_l; }
                     }
                     lo = a;
                     // the pattern occurs iff the suffix there starts with it: that suffix was the last probe that was
@@ -601,23 +616,20 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             if (mode != 3 && mode != 4 && lane < n_fin) sh.fin_tok[lane] = corpus[(int64_t)sa[sh.fin_start[lane]] + d];
             __syncwarp();
             if (mode != 4 && sh.memo_slot >= 0) {
-                // claim the free entry, write the payload, then mark it ready (another CTA may be doing the same for the
-                // same node: whoever loses the claim just goes on)
+                // claim the free entry and write the payload (another CTA may be doing the same for the same node:
+                // whoever loses the claim just goes on)
                 int32_t* en = memo + (size_t)sh.memo_slot * kMemoInts;
                 const unsigned long long key = ((unsigned long long)(unsigned)(sh.full_lo + 1) << 16) | ((unsigned long long)d << 8) | (unsigned)K;
                 int won = 0;
                 if (lane == 0) won = atomicCAS((unsigned long long*)en, 0ull, key) == 0ull;
                 won = __shfl_sync(0xffffffffu, won, 0);
                 if (won) {
-                    if (lane < kMaxK) {
-                        en[4 + lane] = lane < n_fin ? sh.fin_cnt[lane] : 0;
-                        en[12 + lane] = lane < n_fin ? sh.fin_start[lane] : 0;
-                        en[20 + lane] = lane < n_fin ? sh.fin_tok[lane] : 0;
+                    if (lane < n_fin) {                                  // counts are positive; starts and tokens get 1 added
+                        en[4 + lane] = sh.fin_cnt[lane];
+                        en[12 + lane] = sh.fin_start[lane] + 1;
+                        en[20 + lane] = sh.fin_tok[lane] + 1;
                     }
-                    if (lane == 0) en[3] = n_fin;
-                    __threadfence();
-                    __syncwarp();
-                    if (lane == 0) atomicExch(&en[2], 2);
+                    if (lane == 0) en[3] = n_fin + 1;
                 }
             }
             // ---- chain shortcut ----
