@@ -211,14 +211,17 @@ __device__ int count_ending(const int32_t* __restrict__ corpus, const int32_t* _
 
 struct Shared {
     int pat[kMaxP];
-    int pool_cnt[kPoolCap], pool_par[kPoolCap], pool_tok[kPoolCap], pool_lo[kPoolCap];
+    // offers: the rank-r continuation of slot j sits at j * kMaxK + r, a slot's offers in the order (count desc, token asc);
+    // count 0 ends a slot's list
+    int pool_cnt[kPoolCap], pool_tok[kPoolCap], pool_lo[kPoolCap];
     int slot_depth[kMaxN];
     int w_first[kWarps], w_last[kWarps], w_n[kWarps];
     int w_cnt[kWarps][kMaxK], w_start[kWarps][kMaxK];
     int st_cnt[32], st_start[32];               // runs that cross span edges (one per span) and the closing run
     int fin_cnt[kMaxK], fin_start[kMaxK], fin_tok[kMaxK];
-    int mode, cur, lo, cnt, depth, n_nodes, pool_n, thr_shared, long_runs_only, full_lo, full_cnt;
+    int mode, cur, lo, cnt, depth, n_nodes, thr_shared, long_runs_only, full_lo, full_cnt;
     int n_running, n_cap;
+    int m_lo[32], m_hi[32], m_occ[32];          // per candidate length: lower bound, bucket end, occurs
     int memo_slot;                              // >= 0: the node being expanded goes into this memo entry when it is done
     // a batch of small nodes created in one round (equal counts), expanded by one warp each
     int it_slot[kWarps], it_lo[kWarps], it_cnt[kWarps], it_depth[kWarps], n_items;
@@ -266,7 +269,10 @@ __device__ __forceinline__ int compare_suffix(const int32_t* __restrict__ corpus
     return 0;
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+// kCtasPerSm = 2: 64 registers per thread, 296 requests in one wave; 1: 128 registers (nothing spills), used when the
+// grid fits the SMs anyway, which is the low-load case where this kernel's latency matters most.
+template <int kCtasPerSm>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, const uint8_t* __restrict__ lcp,
                  const int32_t* __restrict__ bucket, int32_t* memo, int vocab, const int32_t* __restrict__ tail,
                  const int32_t* __restrict__ tail_len, int B, int P, int N, int K, int min_match, int spec_batch_limit,
@@ -367,47 +373,117 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         }
     };
 
-    if (warp == 0) {
-        // ---- longest-suffix match ----
-        const int tl = min(max(tail_len[b], 0), P);
-        const int len = lane + 1;
+    // Warp 0's running state of the expansion lives in registers (uniform across its lanes unless noted), so that taking
+    // the next offer waits for no shared-memory round trip: slots made so far, slot budget, and per lane the offer lists
+    // of slots lane and lane + 32: how many of a list's offers were taken (cur) and the count of its next one (head, 0 =
+    // none left).  A list is sorted, so the best offer of all is the best head: count desc, then the smaller slot.
+    int n_nodes = 1, n_cap = N, head0 = 0, head1 = 0, cur0 = 0, cur1 = 0;
+    // Rank of a run among the runs of a small node under (length desc, lane asc): c = run length on head lanes (<= 32),
+    // 0 elsewhere.  Six ballots, one per bit of the length, instead of one warp arg-max per winner.
+    auto run_rank = [&](int c) -> int {
+        unsigned gt = 0, eq = 0xffffffffu;
+#pragma unroll
+        for (int bit = 5; bit >= 0; --bit) {
+            const unsigned m = __ballot_sync(0xffffffffu, (c >> bit) & 1);
+            if ((c >> bit) & 1) eq &= m; else { gt |= eq & m; eq &= ~m; }
+        }
+        return __popc(gt) + __popc(eq & ((1u << lane) - 1u));
+    };
+
+    // ---- longest-suffix match ----
+    // Warps 0-3: four lanes per candidate length (thread t: length t / 4 + 1, every fourth token from t % 4 on behind the
+    // known common prefix), so one probe of the binary search compares up to 32 tokens in a single memory latency whatever
+    // the depth of the match.  The four lanes of a group hold the same search state.
+    const int tl = min(max(my_tl, 0), P);
+    if (warp < 4) {
+        const int len = (tid >> 2) + 1, part = tid & 3;
+        const int* pat = sh.pat + (P - len);
         int lo = 0, bucket_hi = 0;
-        bool occurs = false;
+        bool occurs = false, searching = false;
         if (len <= tl) {
-            const int* pat = sh.pat + (P - len);
             bool valid = true;
             for (int t = 0; t < len; ++t) valid = valid && pat[t] >= 0 && pat[t] < vocab;
             if (valid) {
                 lo = bucket[pat[0]];
                 bucket_hi = bucket[pat[0] + 1];
                 occurs = bucket_hi > lo;
-                if (len > 1 && occurs) {
-                    // lower bound by binary search; it remembers how many tokens the pattern shares with the suffixes
-                    // at its current ends, so comparisons restart there (all bucket members share token 0)
-                    int a = lo, z = bucket_hi, ma = 1, mz = 1, m;
-                    // The suffix-array entries of both possible next probes are requested together with this probe's
-                    // corpus tokens, so a step costs one memory latency, not two.
-                    int mid = a + ((z - a) >> 1);
-                    int s_mid = sa[mid];                         // the bucket is not empty
-                    while (a < z) {                              // first suffix >= pattern
-                        const int mid_l = a + ((mid - a) >> 1), mid_r = mid + 1 + ((z - mid - 1) >> 1);
-                        const int s_l = a < mid ? sa[mid_l] : 0, s_r = mid + 1 < z ? sa[mid_r] : 0;
-                        if (compare_suffix(corpus, s_mid, pat, len, min(ma, mz), m) < 0) { a = mid + 1; ma = m; mid = mid_r; s_mid = s_r; }
-                        else { z = mid; mz = m; mid = mid_l; s_mid = s_l; }
-                    }
-                    lo = a;
-                    // the pattern occurs iff the suffix there starts with it: that suffix was the last probe that was
-                    // not below the pattern, and mz tokens of it agreed
-                    occurs = lo < bucket_hi && mz == len;
-                }
+                searching = len > 1 && occurs;
             }
         }
+        // lower bound by binary search; it remembers how many tokens the pattern shares with the suffixes at its
+        // current ends, so comparisons restart there (all bucket members share token 0).  The suffix-array entries
+        // of both possible next probes are requested together with this probe's corpus tokens, so a step costs one
+        // memory latency, not two.  The loop runs while any group of the warp still searches (full-warp shuffles).
+        int a = searching ? lo : 0, z = searching ? bucket_hi : 0, ma = 1, mz = 1;
+        int mid = a + ((z - a) >> 1);
+        int s_mid = searching ? sa[mid] : 0;                      // the bucket is not empty
+        while (__any_sync(0xffffffffu, a < z)) {                  // first suffix >= pattern
+            const bool active = a < z;
+            const int mid_l = a + ((mid - a) >> 1), mid_r = mid + 1 + ((z - mid - 1) >> 1);
+            const int s_l = active && a < mid ? sa[mid_l] : 0, s_r = active && mid + 1 < z ? sa[mid_r] : 0;
+            const int from = min(ma, mz), t0 = from + part;       // lane's tokens: t0, t0 + 4, ... (a group reads 4 adjacent ints per load)
+            // first differing position of the group (position * 2 + "corpus token smaller"); 2 * len = none differs.
+            // Eight tokens first: most probes differ there; the rest (up to 24 more) only for the groups that need them.
+            int key;
+            {
+                unsigned ne = 0, lt = 0;
+                int c[2];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) c[i] = (active && t0 + 4 * i < len) ? corpus[(int64_t)s_mid + t0 + 4 * i] : 0;
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int q = pat[min(t0 + 4 * i, len - 1)];
+                    ne |= (unsigned)(t0 + 4 * i < len && c[i] != q) << i;
+                    lt |= (unsigned)(c[i] < q) << i;
+                }
+                const int f = __ffs(ne) - 1;
+                key = ne ? ((t0 + 4 * f) << 1) | (int)((lt >> f) & 1u) : (len << 1);
+                key = min(key, __shfl_xor_sync(0xffffffffu, key, 1));
+                key = min(key, __shfl_xor_sync(0xffffffffu, key, 2));
+            }
+            const bool more = active && key == (len << 1) && from + 8 < len;      // the same for the lanes of a group
+            if (__any_sync(0xffffffffu, more)) {
+                unsigned ne = 0, lt = 0;
+                int c[6];
+#pragma unroll
+                for (int i = 0; i < 6; ++i) c[i] = (more && t0 + 8 + 4 * i < len) ? corpus[(int64_t)s_mid + t0 + 8 + 4 * i] : 0;
+#pragma unroll
+                for (int i = 0; i < 6; ++i) {
+                    const int q = pat[min(t0 + 8 + 4 * i, len - 1)];
+                    ne |= (unsigned)(t0 + 8 + 4 * i < len && c[i] != q) << i;
+                    lt |= (unsigned)(c[i] < q) << i;
+                }
+                const int f = __ffs(ne) - 1;
+                int key2 = ne ? ((t0 + 8 + 4 * f) << 1) | (int)((lt >> f) & 1u) : (len << 1);
+                key2 = min(key2, __shfl_xor_sync(0xffffffffu, key2, 1));
+                key2 = min(key2, __shfl_xor_sync(0xffffffffu, key2, 2));
+                if (more) key = key2;
+            }
+            if (active) {
+                const int m = key >> 1;                             // leading tokens that agree
+                if (m < len && (key & 1)) { a = mid + 1; ma = m; mid = mid_r; s_mid = s_r; }
+                else { z = mid; mz = m; mid = mid_l; s_mid = s_l; }
+            }
+        }
+        if (searching) {
+            lo = a;
+            // the pattern occurs iff the suffix there starts with it: that suffix was the last probe that was not
+            // below the pattern, and mz tokens of it agreed
+            occurs = lo < bucket_hi && mz == len;
+        }
+        if (part == 0) { sh.m_lo[len - 1] = lo; sh.m_hi[len - 1] = bucket_hi; sh.m_occ[len - 1] = occurs; }
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int lo = sh.m_lo[lane], bucket_hi = sh.m_hi[lane];
+        const bool occurs = sh.m_occ[lane] != 0;
         const unsigned found = __ballot_sync(0xffffffffu, occurs);
         const int ml_longest = found ? 32 - __clz(found) : 0;
         // candidate c drafts from the suffix of ml_longest - c tokens (every shorter suffix of an occurring string
         // occurs, and its lane holds that suffix's lower bound); lengths below max(1, min_match) are no candidates
         const int ml = ml_longest - cand;
         if (cand > 0 && ml < max(1, min_match)) {
+            n_nodes = 0;
             if (lane == 0) { match_len[row] = ml_longest; cand_len[row] = -1; sh.n_nodes = 0; sh.mode = 0; }
         } else {
         const int src = ml > 0 ? ml - 1 : 0;
@@ -420,8 +496,8 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             const int* pat = sh.pat + (P - ml);
             int a = lo + 1, z = bucket_hi, m;                    // positions < a match, positions >= z do not
             // A deep match has few occurrences, and they end where the LCP array first drops below the match length:
-            // look at the next 128 entries before probing the corpus.
-            {
+            // look at the next 128 entries (512 for a match of 8 tokens or more, 128 at a time) before probing the corpus.
+            for (int pass = 0; pass < (ml >= 8 ? 4 : 1) && a < z; ++pass) {
                 int first = 1 << 30;
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
@@ -446,7 +522,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         }
         const int c0 = ml > 0 ? hi - lo : 0;
         // node budget: a longer match earns a larger tree (at most 1 + floor(match_len * fac_num / fac_den) slots)
-        const int n_cap = fac_num > 0 ? min(N, 1 + (int)(((long long)ml * fac_num) / fac_den)) : N;
+        n_cap = fac_num > 0 ? min(N, 1 + (int)(((long long)ml * fac_num) / fac_den)) : N;
         const bool expand = ml >= max(1, min_match) && n_cap > 1;
         if (lane == 0) {
             sh.n_cap = n_cap;
@@ -457,7 +533,6 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             if (o_cnt) o_cnt[0] = c0;
             sh.slot_depth[0] = ml;
             sh.n_nodes = 1;
-            sh.pool_n = 0;
             sh.mode = 0;
         }
         if (expand) publish(0, lo, c0, ml);
@@ -484,21 +559,14 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 const int end = vm ? 32 - __clz(vm) : 0;
                 const unsigned after = (hm >> 1) >> lane;
                 int c = head ? (after ? lane + __ffs(after) : end) - lane : 0;
-                int my_c = 0;
-                for (int r = 0; r < K; ++r) {
-                    const int key = __reduce_max_sync(0xffffffffu, c * 64 + (63 - lane));
-                    if (key < 64) break;
-                    if (lane == 63 - (key & 63)) { my_c = c; c = 0; }
+                const int rank = run_rank(c);
+                if (head && rank < K) {
+                    const bool keep = prob_num == 0 || (long long)c * prob_den >= (long long)prob_num * icnt;
+                    const int at = j * kMaxK + rank;
+                    sh.pool_cnt[at] = keep ? c : 0; sh.pool_tok[at] = tok; sh.pool_lo[at] = ilo + lane;
                 }
-                const bool keep = my_c > 0 && (prob_num == 0 || (long long)my_c * prob_den >= (long long)prob_num * icnt);
-                const unsigned km = __ballot_sync(0xffffffffu, keep);
-                int base = 0;
-                if (lane == 0 && km) base = atomicAdd(&sh.pool_n, __popc(km));
-                base = __shfl_sync(0xffffffffu, base, 0);
-                if (keep) {
-                    const int at = base + __popc(km & ((1u << lane) - 1u));
-                    if (at < kPoolCap) { sh.pool_cnt[at] = my_c; sh.pool_par[at] = j; sh.pool_tok[at] = tok; sh.pool_lo[at] = ilo + lane; }
-                }
+                const int n_runs = min(K, __popc(hm));
+                if (lane >= n_runs && lane < kMaxK) sh.pool_cnt[j * kMaxK + lane] = 0;
             }
             __syncthreads();
         }
@@ -520,11 +588,17 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         }
         if (warp == 0) {
             const int cur = sh.cur;
-            int n_fin = 0;
-            if (mode != 6) {
-            if (mode == 4) {
-                n_fin = -1 - sh.memo_slot;                               // everything is in sh.fin_* already
-            } else if (mode == 3) {
+            if (mode == 6) {
+                // the batch's warps wrote the lists of slots it_slot[0 .. n_items): their owners pick up the heads
+                const int j_first = sh.it_slot[0];
+                const int jj = j_first + ((lane - j_first) & 31);
+                if (jj < j_first + sh.n_items) {
+                    const int h = sh.pool_cnt[jj * kMaxK];
+                    if (jj < 32) { head0 = h; cur0 = 0; } else { head1 = h; cur1 = 0; }
+                }
+            } else {
+            int n_fin = 0, covered = 0;
+            if (mode == 3) {
                 // at most 32 suffixes: lane i reads the continuation token of suffix lo+i; suffixes that end here hold a
                 // separator (negative) and sort first; equal tokens are adjacent, so a run is a head lane plus followers
                 const int tok = lane < cnt ? corpus[(int64_t)sa[lo + lane] + d] : -1;
@@ -536,15 +610,19 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 const int end = vm ? 32 - __clz(vm) : 0;
                 const unsigned after = (hm >> 1) >> lane;                  // heads strictly after this lane
                 int c = head ? (after ? lane + __ffs(after) : end) - lane : 0;
-                for (int r = 0; r < K; ++r) {
-                    const int key = __reduce_max_sync(0xffffffffu, c * 64 + (63 - lane));
-                    if (key < 64) break;                                  // no run left
-                    if (lane == 63 - (key & 63)) {                        // the winning head writes its own run
-                        sh.fin_cnt[n_fin] = c; sh.fin_start[n_fin] = lo + lane; sh.fin_tok[n_fin] = tok;
-                        c = 0;
-                    }
-                    ++n_fin;
+                const int rank = run_rank(c);
+                const bool win = head && rank < K;                        // the k longest runs, each written by its head lane
+                if (win) {
+                    const bool keep = prob_num == 0 || (long long)c * prob_den >= (long long)prob_num * cnt;
+                    const int at = cur * kMaxK + rank;
+                    sh.pool_cnt[at] = keep ? c : 0; sh.pool_tok[at] = tok; sh.pool_lo[at] = lo + lane;
                 }
+                n_fin = min(K, __popc(hm));
+                covered = __reduce_add_sync(0xffffffffu, win ? c : 0);
+                if (lane >= n_fin && lane < kMaxK) sh.pool_cnt[cur * kMaxK + lane] = 0;
+            } else {
+            if (mode == 4) {
+                n_fin = -1 - sh.memo_slot;                               // everything is in sh.fin_* already
             } else if (cnt > 0 && mode == 1) {
                 // one warp saw the whole node: its list plus the closing run (last boundary to the end) is the answer
                 TopK tk;
@@ -580,25 +658,25 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 int* wc = &sh.w_cnt[0][0];
                 int* ws = &sh.w_start[0][0];
                 for (int r = 0; r < K; ++r) {
-                    int bc = 0, bs = 0, bsrc = -1;
+                    int xc = 0, xs = 0, xsrc = -1;
                     for (int i = lane; i < nw * kMaxK; i += 32) {
                         const int c = wc[i], st = ws[i];
-                        if (c > bc || (c == bc && c > 0 && st < bs)) { bc = c; bs = st; bsrc = i; }
+                        if (c > xc || (c == xc && c > 0 && st < xs)) { xc = c; xs = st; xsrc = i; }
                     }
                     {
                         const int c = sh.st_cnt[lane], st = sh.st_start[lane];
-                        if (c > bc || (c == bc && c > 0 && st < bs)) { bc = c; bs = st; bsrc = 0x1000 + lane; }
+                        if (c > xc || (c == xc && c > 0 && st < xs)) { xc = c; xs = st; xsrc = 0x1000 + lane; }
                     }
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) {
-                        const int oc = __shfl_xor_sync(0xffffffffu, bc, o), os = __shfl_xor_sync(0xffffffffu, bs, o);
-                        const int osrc = __shfl_xor_sync(0xffffffffu, bsrc, o);
-                        if (oc > bc || (oc == bc && oc > 0 && os < bs)) { bc = oc; bs = os; bsrc = osrc; }
+                        const int oc = __shfl_xor_sync(0xffffffffu, xc, o), os = __shfl_xor_sync(0xffffffffu, xs, o);
+                        const int osrc = __shfl_xor_sync(0xffffffffu, xsrc, o);
+                        if (oc > xc || (oc == xc && oc > 0 && os < xs)) { xc = oc; xs = os; xsrc = osrc; }
                     }
-                    if (bc <= 0) break;                                  // uniform: no candidate left
+                    if (xc <= 0) break;                                  // uniform: no candidate left
                     if (lane == 0) {
-                        sh.fin_cnt[n_fin] = bc; sh.fin_start[n_fin] = bs;
-                        if (bsrc >= 0x1000) sh.st_cnt[bsrc - 0x1000] = 0; else wc[bsrc] = 0;
+                        sh.fin_cnt[n_fin] = xc; sh.fin_start[n_fin] = xs;
+                        if (xsrc >= 0x1000) sh.st_cnt[xsrc - 0x1000] = 0; else wc[xsrc] = 0;
                     }
                     ++n_fin;
                     __syncwarp();
@@ -606,14 +684,14 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             }
             __syncwarp();
             // suffixes accounted for by the runs found
-            const int covered = __reduce_add_sync(0xffffffffu, lane < n_fin ? sh.fin_cnt[lane] : 0);
+            covered = __reduce_add_sync(0xffffffffu, lane < n_fin ? sh.fin_cnt[lane] : 0);
             if (sh.long_runs_only && n_fin < K && covered < cnt) {       // uniform: fewer than k long runs and more runs exist
                 __syncwarp();
                 if (lane == 0) { sh.long_runs_only = 0; sh.thr_shared = 0; }
                 continue;
             }
-            // tokens of the winners, one lane each (the register path and the memo already have them)
-            if (mode != 3 && mode != 4 && lane < n_fin) sh.fin_tok[lane] = corpus[(int64_t)sa[sh.fin_start[lane]] + d];
+            // tokens of the winners, one lane each (the memo already has them)
+            if (mode != 4 && lane < n_fin) sh.fin_tok[lane] = corpus[(int64_t)sa[sh.fin_start[lane]] + d];
             __syncwarp();
             if (mode != 4 && sh.memo_slot >= 0) {
                 // claim the free entry and write the payload (another CTA may be doing the same for the same node:
@@ -632,17 +710,25 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                     if (lane == 0) en[3] = n_fin + 1;
                 }
             }
+            // the winners become offers, one lane each, rank = lane: count(child) * den >= num * count(parent) when a
+            // threshold is set (an offer that fails it is written as retired)
+            if (lane < kMaxK) {
+                const int my_cnt = lane < n_fin ? sh.fin_cnt[lane] : 0;
+                const bool keep = prob_num == 0 || (long long)my_cnt * prob_den >= (long long)prob_num * sh.full_cnt;
+                const int at = cur * kMaxK + lane;
+                sh.pool_cnt[at] = keep ? my_cnt : 0;
+                if (lane < n_fin) { sh.pool_tok[at] = sh.fin_tok[lane]; sh.pool_lo[at] = sh.fin_start[lane]; }
+            }
+            }   // mode != 3
             // ---- chain shortcut ----
             // If every occurrence of this node continues with the same token, that child has the node's own count; when
             // no pooled offer reaches that count it is the strict best and becomes the next slot, and the same holds for
             // its own single child, and so on for as long as the first and the last suffix of the interval agree (their
-            // common prefix is the common prefix of the whole interval).  All those slots are emitted at once.
+            // common prefix is the common prefix of the whole interval).  All those slots are emitted at once; the offer
+            // written above is simply not counted in.
             if (n_fin == 1 && covered == sh.full_cnt) {
-                int pmax = 0;
-                for (int i = lane; i < sh.pool_n; i += 32) pmax = max(pmax, sh.pool_cnt[i]);
-                pmax = __reduce_max_sync(0xffffffffu, pmax);
-                const int c = sh.full_cnt, flo = sh.full_lo, j0 = sh.n_nodes, room = sh.n_cap - j0;
-                __syncwarp();
+                const int pmax = __reduce_max_sync(0xffffffffu, max(head0, head1));
+                const int c = sh.full_cnt, flo = sh.full_lo, j0 = n_nodes, room = n_cap - j0;
                 if (pmax < c && room > 0) {
                     const int64_t s_first = sa[flo], s_last = sa[flo + c - 1];
                     const int tf = lane < room ? corpus[s_first + d + lane] : -1;
@@ -656,80 +742,59 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                             if (o_cnt) o_cnt[j0 + lane] = c;
                             sh.slot_depth[j0 + lane] = d + 1 + lane;
                         }
+                        n_nodes = j0 + len;
+                        if (lane == 0) { sh.n_nodes = n_nodes; sh.mode = 0; }
                         __syncwarp();
-                        if (lane == 0) { sh.n_nodes = j0 + len; sh.mode = 0; }
-                        if (j0 + len < sh.n_cap) publish(j0 + len - 1, flo, c, d + len);
+                        if (n_nodes < n_cap) publish(n_nodes - 1, flo, c, d + len);
                         continue;
                     }
                 }
             }
-            {   // the winners become offers, one lane each: count(child) * den >= num * count(parent) when a threshold is set
-                const int pn0 = sh.pool_n;
-                const int my_cnt = lane < n_fin ? sh.fin_cnt[lane] : 0;
-                const bool keep = lane < n_fin && (prob_num == 0 || (long long)my_cnt * prob_den >= (long long)prob_num * sh.full_cnt);
-                const unsigned km = __ballot_sync(0xffffffffu, keep);
-                const int at = pn0 + __popc(km & ((1u << lane) - 1u));
-                if (keep && at < kPoolCap) {
-                    sh.pool_cnt[at] = my_cnt; sh.pool_par[at] = cur; sh.pool_tok[at] = sh.fin_tok[lane]; sh.pool_lo[at] = sh.fin_start[lane];
-                }
-                __syncwarp();
-                if (lane == 0) sh.pool_n = min(kPoolCap, pn0 + __popc(km));
+            // the list of this slot is in place: its owner picks up the head
+            __syncwarp();
+            if (lane == (cur & 31)) {
+                const int h = sh.pool_cnt[cur * kMaxK];
+                if (cur < 32) { head0 = h; cur0 = 0; } else { head1 = h; cur1 = 0; }
             }
             }   // mode != 6
-            __syncwarp();
             // ---- take the best offer: count desc, parent slot asc, token asc ----
             // Offers that tie with the best one on the count follow it in exactly this order whatever their own
             // continuations are (a continuation's count is not larger and its parent slot is newer), so all of them, up to
             // one per warp, become slots now; if they are small nodes they are expanded together in the next round.
-            int n_items = 0, batch_c = 0;
+            int n_items = 0, batch_c = 0, j = 0, slo = 0, depth = 0;
             while (true) {
-            const int pn = sh.pool_n;
-            int bi = -1, bc = -1, bp = 0, bt = 0;
-            for (int i = lane; i < pn; i += 32) {
-                const int c = sh.pool_cnt[i], p = sh.pool_par[i], t = sh.pool_tok[i];
-                if (bi < 0 || c > bc || (c == bc && (p < bp || (p == bp && t < bt)))) { bi = i; bc = c; bp = p; bt = t; }
+                const int c_best = __reduce_max_sync(0xffffffffu, max(head0, head1));
+                if (c_best <= 0 || (n_items > 0 && c_best != batch_c)) break;
+                // among the lists whose head has that count the smallest slot wins; its cursor rides along
+                const int mine = head0 == c_best ? (lane * kMaxK + cur0) : head1 == c_best ? ((lane + 32) * kMaxK + cur1) : 0x7fffffff;
+                const int bi = __reduce_min_sync(0xffffffffu, mine);     // parent slot * kMaxK + rank = where the offer sits
+                const int bp = bi / kMaxK;
+                j = n_nodes;
+                slo = sh.pool_lo[bi];
+                depth = sh.slot_depth[bp] + 1;                           // parents were made in earlier rounds
+                if (lane == (bp & 31)) {                                 // the list's owner emits the slot and moves to the next offer
+                    o_ids[j] = sh.pool_tok[bi]; o_par[j] = bp;
+                    if (o_cnt) o_cnt[j] = c_best;
+                    sh.slot_depth[j] = depth;
+                    sh.it_slot[n_items] = j; sh.it_lo[n_items] = slo; sh.it_cnt[n_items] = c_best; sh.it_depth[n_items] = depth;
+                    const int nr = (bi & (kMaxK - 1)) + 1;
+                    const int nh = nr < kMaxK ? sh.pool_cnt[bi + 1] : 0;
+                    if (bp < 32) { cur0 = nr; head0 = nh; } else { cur1 = nr; head1 = nh; }
+                }
+                ++n_nodes;
+                batch_c = c_best;
+                ++n_items;
+                if (n_nodes >= n_cap) { n_items = -1; break; }         // the budget is used up: nothing is expanded any more
+                if (c_best > 32 || n_items == kWarps) break;            // large nodes go one at a time
             }
-            {   // best of the lanes' candidates: largest count, then smallest parent slot, then smallest token (unique)
-                const int c_best = __reduce_max_sync(0xffffffffu, bc);                       // -1 when the pool is empty
-                const bool in1 = bi >= 0 && bc == c_best;
-                const int p_best = __reduce_min_sync(0xffffffffu, in1 ? bp : 0x7fffffff);
-                const bool in2 = in1 && bp == p_best;
-                const int t_best = __reduce_min_sync(0xffffffffu, in2 ? bt : 0x7fffffff);
-                const unsigned wm = __ballot_sync(0xffffffffu, in2 && bt == t_best);
-                const int wl = wm ? __ffs(wm) - 1 : 0;
-                bi = wm ? __shfl_sync(0xffffffffu, bi, wl) : -1;
-                bc = c_best; bp = p_best; bt = t_best;
-            }
-            // every lane now holds the same winner
-            if (bi < 0 || (n_items > 0 && bc != batch_c)) break;
-            const int j = sh.n_nodes;
-            const int slo = sh.pool_lo[bi];
-            const int depth = sh.slot_depth[bp] + 1;
-            __syncwarp();
-            if (lane == 0) {
-                const int last = pn - 1;
-                sh.pool_cnt[bi] = sh.pool_cnt[last]; sh.pool_par[bi] = sh.pool_par[last];
-                sh.pool_tok[bi] = sh.pool_tok[last]; sh.pool_lo[bi] = sh.pool_lo[last];
-                sh.pool_n = last;
-                o_ids[j] = bt; o_par[j] = bp;
-                if (o_cnt) o_cnt[j] = bc;
-                sh.slot_depth[j] = depth;
-                sh.n_nodes = j + 1;
-                sh.it_slot[n_items] = j; sh.it_lo[n_items] = slo; sh.it_cnt[n_items] = bc; sh.it_depth[n_items] = depth;
-            }
-            __syncwarp();
-            batch_c = bc;
-            ++n_items;
-            if (j + 1 >= sh.n_cap) { n_items = -1; break; }        // the budget is used up: nothing is expanded any more
-            if (bc > 32 || n_items == kWarps) break;              // large nodes go one at a time
-            }
+            if (lane == 0) sh.n_nodes = n_nodes;
             // what the next round does
             if (n_items <= 0) {
                 if (lane == 0) sh.mode = 0;
             } else if (n_items == 1) {
                 if (lane == 0) sh.mode = 0;
                 __syncwarp();
-                publish(sh.it_slot[0], sh.it_lo[0], sh.it_cnt[0], sh.it_depth[0]);
+                publish(j, slo, batch_c, depth);
             } else {
                 if (lane == 0) { sh.n_items = n_items; sh.mode = 6; }
             }
@@ -804,6 +869,28 @@ war_draft_select_kernel(CandArrays ca, int B, int C, int N, int32_t* __restrict_
     }
 }
 
+war_status_t launch_draft(const war_index_t* ix, const int32_t* d_tail, const int32_t* d_tail_len, const war_draft_params_t* p,
+                          int n_cand, int32_t* match_len, int32_t* num_nodes, int32_t* ids, int32_t* parent, int32_t* count,
+                          int32_t* cand_len, cudaStream_t stream) {
+    static int sm_count[64] = {0};
+    const int dev = ix->device;
+    if (dev < 0 || dev >= 64) return WAR_ERR_INVALID_ARG;
+    if (!sm_count[dev]) WAR_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+    const war_index_arrays arr = const_cast<war_index_t*>(ix)->published();       // a complete index, also during an update
+    const dim3 grid(p->B, n_cand);
+    const int fac_den = p->spec_factor_num > 0 ? p->spec_factor_den : 1, prob_den = p->min_prob_num > 0 ? p->min_prob_den : 1;
+    if ((long long)p->B * n_cand <= sm_count[dev])
+        war_draft_kernel<1><<<grid, kThreads, 0, stream>>>(ix->corpus, arr.sa, arr.lcp, arr.bucket, arr.memo, ix->vocab, d_tail, d_tail_len,
+                                                          p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, p->spec_factor_num,
+                                                          fac_den, p->min_prob_num, prob_den, match_len, num_nodes, ids, parent, count, cand_len);
+    else
+        war_draft_kernel<2><<<grid, kThreads, 0, stream>>>(ix->corpus, arr.sa, arr.lcp, arr.bucket, arr.memo, ix->vocab, d_tail, d_tail_len,
+                                                          p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, p->spec_factor_num,
+                                                          fac_den, p->min_prob_num, prob_den, match_len, num_nodes, ids, parent, count, cand_len);
+    WAR_LAUNCH_CHECK();
+    return WAR_OK;
+}
+
 bool draft_params_ok(const war_index_t* ix, const war_draft_params_t* p) {
     if (p->B < 0 || p->P < 1 || p->P > kMaxP || p->N < 1 || p->N > kMaxN || p->topk < 1 || p->topk > kMaxK || p->min_match < 0 ||
         p->spec_batch_limit < 0 || p->spec_factor_num < 0 || (p->spec_factor_num > 0 && p->spec_factor_den < 1) ||
@@ -829,13 +916,10 @@ extern "C" war_status_t war_draft_scored(const war_index_t* ix, const int32_t* d
     if (p->B == 0) return WAR_OK;
     if (!d_tail || !d_tail_len || !d_workspace || !d_match_len || !d_used_len || !d_num_nodes || !d_ids || !d_parent)
         return WAR_ERR_INVALID_ARG;
-    const war_index_arrays arr = const_cast<war_index_t*>(ix)->published();
     const CandArrays ca = cand_layout(d_workspace, (size_t)p->B * n_lengths, p->N);
-    war_draft_kernel<<<dim3(p->B, n_lengths), kThreads, 0, stream>>>(
-        ix->corpus, arr.sa, arr.lcp, arr.bucket, arr.memo, ix->vocab, d_tail, d_tail_len, p->B, p->P, p->N, p->topk, p->min_match,
-        p->spec_batch_limit, p->spec_factor_num, p->spec_factor_num > 0 ? p->spec_factor_den : 1, p->min_prob_num,
-        p->min_prob_num > 0 ? p->min_prob_den : 1, ca.match_len, ca.num_nodes, ca.ids, ca.parent, ca.count, ca.len);
-    WAR_LAUNCH_CHECK();
+    const war_status_t st = launch_draft(ix, d_tail, d_tail_len, p, n_lengths, ca.match_len, ca.num_nodes, ca.ids, ca.parent, ca.count,
+                                         ca.len, stream);
+    if (st != WAR_OK) return st;
     war_draft_select_kernel<<<(p->B + 7) / 8, 256, 0, stream>>>(ca, p->B, n_lengths, p->N, d_match_len, d_used_len, d_num_nodes,
                                                               d_ids, d_parent, d_count);
     WAR_LAUNCH_CHECK();
@@ -849,12 +933,5 @@ extern "C" war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, 
     if (!draft_params_ok(ix, p)) return WAR_ERR_INVALID_ARG;
     if (p->B == 0) return WAR_OK;
     if (!d_tail || !d_tail_len || !d_match_len || !d_num_nodes || !d_ids || !d_parent) return WAR_ERR_INVALID_ARG;
-    const war_index_arrays arr = const_cast<war_index_t*>(ix)->published();       // a complete index, also during an update
-    war_draft_kernel<<<p->B, kThreads, 0, stream>>>(ix->corpus, arr.sa, arr.lcp, arr.bucket, arr.memo, ix->vocab, d_tail, d_tail_len,
-                                                   p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, p->spec_factor_num,
-                                                   p->spec_factor_num > 0 ? p->spec_factor_den : 1, p->min_prob_num,
-                                                   p->min_prob_num > 0 ? p->min_prob_den : 1, d_match_len,
-                                                   d_num_nodes, d_ids, d_parent, d_count, nullptr);
-    WAR_LAUNCH_CHECK();
-    return WAR_OK;
+    return launch_draft(ix, d_tail, d_tail_len, p, 1, d_match_len, d_num_nodes, d_ids, d_parent, d_count, nullptr, stream);
 }
