@@ -540,11 +540,13 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
     }
 
     // ---- best-first expansion ----
+    // Modes: 1 a node scanned by warp 0 alone, 2 a node scanned by all warps, 3 a node of at most 32 suffixes (in
+    // registers), 4 a node answered by the memo, 6 a batch of small nodes (one per warp).  Only 2 and 6 need the other
+    // warps: they wait at the barrier below while warp 0 works through nodes of the other kinds on its own.
     while (true) {
         __syncthreads();
-        const int mode = sh.mode;
+        int mode = sh.mode;
         if (mode == 0) break;
-        const int lo = sh.lo, cnt = sh.cnt, d = sh.depth, hi = lo + cnt;
         if (mode == 6) {
             // A batch of small nodes: warp w expands item w in registers (one suffix per lane) and adds its k best
             // continuations to the offer pool.
@@ -571,6 +573,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             __syncthreads();
         }
         if (mode == 2) {
+            const int lo = sh.lo, d = sh.depth, hi = lo + sh.cnt;
             const int a0 = lo & ~15;
             int span = (hi - a0 + kWarps - 1) / kWarps;
             span = (span + 511) & ~511;
@@ -587,6 +590,8 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             __syncthreads();
         }
         if (warp == 0) {
+            while (true) {                                               // one node (or batch) per turn
+            const int lo = sh.lo, cnt = sh.cnt, d = sh.depth, hi = lo + cnt;
             const int cur = sh.cur;
             if (mode == 6) {
                 // the batch's warps wrote the lists of slots it_slot[0 .. n_items): their owners pick up the heads
@@ -688,7 +693,8 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             if (sh.long_runs_only && n_fin < K && covered < cnt) {       // uniform: fewer than k long runs and more runs exist
                 __syncwarp();
                 if (lane == 0) { sh.long_runs_only = 0; sh.thr_shared = 0; }
-                continue;
+                if (mode == 1) { __syncwarp(); continue; }               // warp 0 scans it again itself
+                break;
             }
             // tokens of the winners, one lane each (the memo already has them)
             if (mode != 4 && lane < n_fin) sh.fin_tok[lane] = corpus[(int64_t)sa[sh.fin_start[lane]] + d];
@@ -746,7 +752,10 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                         if (lane == 0) { sh.n_nodes = n_nodes; sh.mode = 0; }
                         __syncwarp();
                         if (n_nodes < n_cap) publish(n_nodes - 1, flo, c, d + len);
-                        continue;
+                        __syncwarp();
+                        mode = sh.mode;
+                        if (mode == 1 || mode == 3 || mode == 4) continue;
+                        break;
                     }
                 }
             }
@@ -797,6 +806,10 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 publish(j, slo, batch_c, depth);
             } else {
                 if (lane == 0) { sh.n_items = n_items; sh.mode = 6; }
+            }
+            __syncwarp();
+            mode = sh.mode;
+            if (mode != 1 && mode != 3 && mode != 4) break;               // done, or the next turn needs the other warps
             }
         }
     }
