@@ -77,7 +77,9 @@ __device__ __forceinline__ unsigned le_mask16(uint4 v, unsigned drep) {
 // that long exist somewhere in the node, so a run shorter than that cannot be among the node's k best (an equally
 // long one still can, by its earlier start).  Once the bar is at 16 or more, no run that lies inside one lane's 16
 // positions can pass it, and only the run ending at a lane's first boundary needs a look.
-__device__ void warp_scan_span(const uint8_t* __restrict__ lcp, int d, int sb, int se, int k, int lane,
+// (kept out of line, like the other rarely taken paths below: the kernel's hot path is one warp walking a long chain of
+// dependent steps, and it runs at the speed of the instruction cache unless the code it crosses stays small)
+__device__ __noinline__ void warp_scan_span(const uint8_t* __restrict__ lcp, int d, int sb, int se, int k, int lane,
                                TopK& tk, int& first_b, int& last_b, int* thr_shared) {
     topk_clear(tk);
     int thr_local = 0;                                     // a run must beat this count to enter this warp's top-k
@@ -190,7 +192,7 @@ __device__ void warp_scan_span(const uint8_t* __restrict__ lcp, int d, int sb, i
 // Number of suffixes of the interval [lo, hi) whose entry at depth d is a separator (the occurrence ends its
 // trajectory there).  They sort before every real token, so this is the first position holding a token >= 0,
 // found by a 32-way search of one warp; almost always the very first probe answers.
-__device__ int count_ending(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, int lo, int hi, int d, int lane) {
+__device__ __noinline__ int count_ending(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, int lo, int hi, int d, int lane) {
     int first = corpus[(int64_t)sa[lo] + d];
     if (first >= 0) return 0;
     int a = lo + 1, z = hi;                                 // answer in [a, z]: positions < a hold separators
@@ -230,7 +232,7 @@ struct Shared {
 // Tokens from index `from` on of the suffix at s against the pattern; returns the sign and, in `matched`, how many
 // leading tokens agree.  Eight corpus tokens, then sixteen at a time, are requested together so their latencies
 // overlap (the corpus has readable slack behind its last separator, and a separator always ends the walk).
-__device__ __forceinline__ int compare_suffix(const int32_t* __restrict__ corpus, int64_t s, const int* pat, int len, int from,
+__device__ __noinline__ int compare_suffix(const int32_t* __restrict__ corpus, int64_t s, const int* pat, int len, int from,
                                               int& matched) {
     // Branch-free inside a batch: one bit per position for "differs" and one for "corpus token is smaller"; the first
     // set bit decides.  (A chain of early exits costs a divergent branch per token on a path that is pure latency.)
@@ -322,15 +324,18 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         return;
     }
 
-    // Publishes the next node to expand: its token range (the interval minus the suffixes that end at this depth).
+    // The node warp 0 works on next, in its registers (uniform across the lanes): slot, token range (the interval minus
+    // the suffixes that end at this depth), depth, whole interval, memo entry to fill (-1 none), kind of turn, and for
+    // a memo hit the number of offers and the occurrences they cover.  What other warps read is mirrored in shared memory.
+    int t_cur = 0, t_lo = 0, t_cnt = 0, t_depth = 0, t_full_lo = 0, t_full_cnt = 0, t_memo_slot = -1, t_mode = 0, t_nfin = 0, t_cov = 0;
     auto publish = [&](int slot, int lo, int cnt, int depth) {          // warp 0, all lanes
+        t_cur = slot; t_lo = lo; t_cnt = cnt; t_depth = depth; t_full_lo = lo; t_full_cnt = cnt; t_memo_slot = -1;
         if (cnt <= 32) {                                                // handled in registers, one suffix per lane
-            if (lane == 0) { sh.cur = slot; sh.lo = lo; sh.cnt = cnt; sh.depth = depth; sh.long_runs_only = 0; sh.mode = 3;
-                             sh.full_lo = lo; sh.full_cnt = cnt; sh.memo_slot = -1; }
+            t_mode = 3;
+            if (lane == 0) sh.mode = 3;
             return;
         }
         // Large nodes are looked up in the index's memo first (same node, same k => same answer for every request)
-        int memo_slot = -1;
         if (cnt >= kMemoMinCount) {
             const unsigned long long key = ((unsigned long long)(unsigned)(lo + 1) << 16) | ((unsigned long long)depth << 8) | (unsigned)K;
             unsigned h = (unsigned)(key * 0x9E3779B97F4A7C15ull >> 40) & (kMemoEntries - 1);
@@ -344,32 +349,40 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             got = __shfl_sync(0xffffffffu, got, 0);
             if (got == key) {
                 const int n_fin = __shfl_sync(0xffffffffu, word, 3) - 1;
-                const bool mine = lane >= 4 && lane < 28 && ((lane - 4) & 7) < n_fin;      // a word this node's answer uses
+                const int r = (lane - 4) & 7;                            // lanes 4..11 counts, 12..19 starts, 20..27 tokens
+                const bool mine = lane >= 4 && lane < 28 && r < n_fin;  // a word this node's answer uses
                 if (n_fin >= 0 && __ballot_sync(0xffffffffu, mine && word == 0) == 0u) {
-                    if (mine) {
-                        int* dst = lane < 12 ? sh.fin_cnt : lane < 20 ? sh.fin_start : sh.fin_tok;
-                        dst[(lane - 4) & 7] = word - (lane < 12 ? 0 : 1);
+                    // the answer goes straight into this slot's offer list
+                    const int at = slot * kMaxK + r;
+                    if (lane >= 4 && lane < 12) {
+                        const bool keep = mine && (prob_num == 0 || (long long)word * prob_den >= (long long)prob_num * cnt);
+                        sh.pool_cnt[at] = keep ? word : 0;
+                    } else if (mine) {
+                        if (lane < 20) sh.pool_lo[at] = word - 1; else sh.pool_tok[at] = word - 1;
                     }
-                    if (lane == 0) {
-                        sh.cur = slot; sh.lo = lo; sh.cnt = cnt; sh.depth = depth; sh.full_lo = lo; sh.full_cnt = cnt;
-                        sh.long_runs_only = 0; sh.thr_shared = 0; sh.memo_slot = -1 - n_fin; sh.mode = 4;
-                    }
+                    __syncwarp();
+                    t_nfin = n_fin;
+                    t_cov = __reduce_add_sync(0xffffffffu, mine && lane < 12 ? word : 0);
+                    t_mode = 4;
+                    if (lane == 0) sh.mode = 4;
                     return;
                 }
             } else if (got == 0ull) {
-                memo_slot = (int)h;                                      // free: this expansion will try to fill it
+                t_memo_slot = (int)h;                                    // free: this expansion will try to fill it
             }
         }
         const int e = count_ending(corpus, sa, lo, lo + cnt, depth, lane);
+        t_lo = lo + e; t_cnt = cnt - e;
+        // Large nodes are first scanned for runs of 16 positions or more only (bar preset to 16): that pass never
+        // walks the boundaries inside a lane.  It is exact whenever it finds k such runs; otherwise the node is
+        // scanned again without the preset.
+        const int long_first = (cnt - e) >= kLongRunFirstMin;
+        t_mode = (cnt - e) >= kBlockScanMin ? 2 : 1;
         if (lane == 0) {
-            sh.memo_slot = memo_slot;
-            sh.cur = slot; sh.lo = lo + e; sh.cnt = cnt - e; sh.depth = depth; sh.full_lo = lo; sh.full_cnt = cnt;
-            // Large nodes are first scanned for runs of 16 positions or more only (bar preset to 16): that pass never
-            // walks the boundaries inside a lane.  It is exact whenever it finds k such runs; otherwise the node is
-            // scanned again without the preset.
-            sh.long_runs_only = (cnt - e) >= kLongRunFirstMin;
-            sh.thr_shared = sh.long_runs_only ? 16 : 0;
-            sh.mode = (cnt - e) >= kBlockScanMin ? 2 : 1;
+            sh.lo = lo + e; sh.cnt = cnt - e; sh.depth = depth;
+            sh.long_runs_only = long_first;
+            sh.thr_shared = long_first ? 16 : 0;
+            sh.mode = t_mode;
         }
     };
 
@@ -591,8 +604,8 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         }
         if (warp == 0) {
             while (true) {                                               // one node (or batch) per turn
-            const int lo = sh.lo, cnt = sh.cnt, d = sh.depth, hi = lo + cnt;
-            const int cur = sh.cur;
+            __syncwarp();                                                // single-lane stores end here: the lanes go on together
+            const int lo = t_lo, cnt = t_cnt, d = t_depth, hi = lo + cnt, cur = t_cur;
             if (mode == 6) {
                 // the batch's warps wrote the lists of slots it_slot[0 .. n_items): their owners pick up the heads
                 const int j_first = sh.it_slot[0];
@@ -625,10 +638,11 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 n_fin = min(K, __popc(hm));
                 covered = __reduce_add_sync(0xffffffffu, win ? c : 0);
                 if (lane >= n_fin && lane < kMaxK) sh.pool_cnt[cur * kMaxK + lane] = 0;
+                __syncwarp();
+            } else if (mode == 4) {
+                n_fin = t_nfin; covered = t_cov;                          // the memo's answer is in the slot's offer list already
             } else {
-            if (mode == 4) {
-                n_fin = -1 - sh.memo_slot;                               // everything is in sh.fin_* already
-            } else if (cnt > 0 && mode == 1) {
+            if (cnt > 0 && mode == 1) {
                 // one warp saw the whole node: its list plus the closing run (last boundary to the end) is the answer
                 TopK tk;
                 int fb, lb;
@@ -696,14 +710,14 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 if (mode == 1) { __syncwarp(); continue; }               // warp 0 scans it again itself
                 break;
             }
-            // tokens of the winners, one lane each (the memo already has them)
-            if (mode != 4 && lane < n_fin) sh.fin_tok[lane] = corpus[(int64_t)sa[sh.fin_start[lane]] + d];
+            // tokens of the winners, one lane each
+            if (lane < n_fin) sh.fin_tok[lane] = corpus[(int64_t)sa[sh.fin_start[lane]] + d];
             __syncwarp();
-            if (mode != 4 && sh.memo_slot >= 0) {
+            if (t_memo_slot >= 0) {
                 // claim the free entry and write the payload (another CTA may be doing the same for the same node:
                 // whoever loses the claim just goes on)
-                int32_t* en = memo + (size_t)sh.memo_slot * kMemoInts;
-                const unsigned long long key = ((unsigned long long)(unsigned)(sh.full_lo + 1) << 16) | ((unsigned long long)d << 8) | (unsigned)K;
+                int32_t* en = memo + (size_t)t_memo_slot * kMemoInts;
+                const unsigned long long key = ((unsigned long long)(unsigned)(t_full_lo + 1) << 16) | ((unsigned long long)d << 8) | (unsigned)K;
                 int won = 0;
                 if (lane == 0) won = atomicCAS((unsigned long long*)en, 0ull, key) == 0ull;
                 won = __shfl_sync(0xffffffffu, won, 0);
@@ -720,21 +734,21 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             // threshold is set (an offer that fails it is written as retired)
             if (lane < kMaxK) {
                 const int my_cnt = lane < n_fin ? sh.fin_cnt[lane] : 0;
-                const bool keep = prob_num == 0 || (long long)my_cnt * prob_den >= (long long)prob_num * sh.full_cnt;
+                const bool keep = prob_num == 0 || (long long)my_cnt * prob_den >= (long long)prob_num * t_full_cnt;
                 const int at = cur * kMaxK + lane;
                 sh.pool_cnt[at] = keep ? my_cnt : 0;
                 if (lane < n_fin) { sh.pool_tok[at] = sh.fin_tok[lane]; sh.pool_lo[at] = sh.fin_start[lane]; }
             }
-            }   // mode != 3
+            }   // a scanned node
             // ---- chain shortcut ----
             // If every occurrence of this node continues with the same token, that child has the node's own count; when
             // no pooled offer reaches that count it is the strict best and becomes the next slot, and the same holds for
             // its own single child, and so on for as long as the first and the last suffix of the interval agree (their
             // common prefix is the common prefix of the whole interval).  All those slots are emitted at once; the offer
             // written above is simply not counted in.
-            if (n_fin == 1 && covered == sh.full_cnt) {
+            if (n_fin == 1 && covered == t_full_cnt) {
                 const int pmax = __reduce_max_sync(0xffffffffu, max(head0, head1));
-                const int c = sh.full_cnt, flo = sh.full_lo, j0 = n_nodes, room = n_cap - j0;
+                const int c = t_full_cnt, flo = t_full_lo, j0 = n_nodes, room = n_cap - j0;
                 if (pmax < c && room > 0) {
                     const int64_t s_first = sa[flo], s_last = sa[flo + c - 1];
                     const int tf = lane < room ? corpus[s_first + d + lane] : -1;
@@ -749,11 +763,10 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                             sh.slot_depth[j0 + lane] = d + 1 + lane;
                         }
                         n_nodes = j0 + len;
+                        t_mode = 0;
                         if (lane == 0) { sh.n_nodes = n_nodes; sh.mode = 0; }
-                        __syncwarp();
                         if (n_nodes < n_cap) publish(n_nodes - 1, flo, c, d + len);
-                        __syncwarp();
-                        mode = sh.mode;
+                        mode = t_mode;
                         if (mode == 1 || mode == 3 || mode == 4) continue;
                         break;
                     }
@@ -765,6 +778,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 const int h = sh.pool_cnt[cur * kMaxK];
                 if (cur < 32) { head0 = h; cur0 = 0; } else { head1 = h; cur1 = 0; }
             }
+            __syncwarp();
             }   // mode != 6
             // ---- take the best offer: count desc, parent slot asc, token asc ----
             // Offers that tie with the best one on the count follow it in exactly this order whatever their own
@@ -790,6 +804,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                     const int nh = nr < kMaxK ? sh.pool_cnt[bi + 1] : 0;
                     if (bp < 32) { cur0 = nr; head0 = nh; } else { cur1 = nr; head1 = nh; }
                 }
+                __syncwarp();
                 ++n_nodes;
                 batch_c = c_best;
                 ++n_items;
@@ -797,18 +812,18 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 if (c_best > 32 || n_items == kWarps) break;            // large nodes go one at a time
             }
             if (lane == 0) sh.n_nodes = n_nodes;
+            __syncwarp();
             // what the next round does
             if (n_items <= 0) {
+                t_mode = 0;
                 if (lane == 0) sh.mode = 0;
             } else if (n_items == 1) {
-                if (lane == 0) sh.mode = 0;
-                __syncwarp();
                 publish(j, slo, batch_c, depth);
             } else {
+                t_mode = 6;
                 if (lane == 0) { sh.n_items = n_items; sh.mode = 6; }
             }
-            __syncwarp();
-            mode = sh.mode;
+            mode = t_mode;
             if (mode != 1 && mode != 3 && mode != 4) break;               // done, or the next turn needs the other warps
             }
         }
