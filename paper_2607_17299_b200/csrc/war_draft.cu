@@ -424,58 +424,69 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             }
         }
         // lower bound by binary search; it remembers how many tokens the pattern shares with the suffixes at its
-        // current ends, so comparisons restart there (all bucket members share token 0).  The suffix-array entries
-        // of both possible next probes are requested together with this probe's corpus tokens, so a step costs one
-        // memory latency, not two.  The loop runs while any group of the warp still searches (full-warp shuffles).
+        // current ends, so comparisons restart there (all bucket members share token 0).  The search is pipelined two
+        // probes deep so that a step costs one memory latency instead of two or three: while the current probe is
+        // compared, the first tokens of BOTH possible next probes are on their way (their suffix-array entries came
+        // in during the previous step), and so are the suffix-array entries of the four probes after those.  The loop
+        // runs while any group of the warp still searches (full-warp shuffles).
         int a = searching ? lo : 0, z = searching ? bucket_hi : 0, ma = 1, mz = 1;
         int mid = a + ((z - a) >> 1);
-        int s_mid = searching ? sa[mid] : 0;                      // the bucket is not empty
+        int s_mid = 0, s_l = 0, s_r = 0, c0 = 0, c1 = 0, at = 1 + part;   // at: pattern position of c0 (c1 is 4 further)
+        if (searching) {
+            const int mid_l = a + ((mid - a) >> 1), mid_r = mid + 1 + ((z - mid - 1) >> 1);
+            s_mid = sa[mid];                                      // the bucket is not empty
+            s_l = a < mid ? sa[mid_l] : 0;
+            s_r = mid + 1 < z ? sa[mid_r] : 0;
+            c0 = at < len ? corpus[(int64_t)s_mid + at] : 0;
+            c1 = at + 4 < len ? corpus[(int64_t)s_mid + at + 4] : 0;
+        }
         while (__any_sync(0xffffffffu, a < z)) {                  // first suffix >= pattern
             const bool active = a < z;
             const int mid_l = a + ((mid - a) >> 1), mid_r = mid + 1 + ((z - mid - 1) >> 1);
-            const int s_l = active && a < mid ? sa[mid_l] : 0, s_r = active && mid + 1 < z ? sa[mid_r] : 0;
-            const int from = min(ma, mz), t0 = from + part;       // lane's tokens: t0, t0 + 4, ... (a group reads 4 adjacent ints per load)
+            const bool has_l = active && a < mid, has_r = active && mid + 1 < z;
+            // suffix-array entries two steps ahead
+            const int mid_ll = a + ((mid_l - a) >> 1), mid_lr = mid_l + 1 + ((mid - mid_l - 1) >> 1);
+            const int mid_rl = mid + 1 + ((mid_r - mid - 1) >> 1), mid_rr = mid_r + 1 + ((z - mid_r - 1) >> 1);
+            const int s_ll = has_l && a < mid_l ? sa[mid_ll] : 0, s_lr = has_l && mid_l + 1 < mid ? sa[mid_lr] : 0;
+            const int s_rl = has_r && mid + 1 < mid_r ? sa[mid_rl] : 0, s_rr = has_r && mid_r + 1 < z ? sa[mid_rr] : 0;
+            // first tokens of both possible next probes, from the prefix known now (it can only grow)
+            const int from = min(ma, mz), nt = from + part;
+            const int l0 = has_l && nt < len ? corpus[(int64_t)s_l + nt] : 0, l1 = has_l && nt + 4 < len ? corpus[(int64_t)s_l + nt + 4] : 0;
+            const int r0 = has_r && nt < len ? corpus[(int64_t)s_r + nt] : 0, r1 = has_r && nt + 4 < len ? corpus[(int64_t)s_r + nt + 4] : 0;
             // first differing position of the group (position * 2 + "corpus token smaller"); 2 * len = none differs.
             // Eight tokens first: most probes differ there; the rest (up to 24 more) only for the groups that need them.
             int key;
             {
+                const int q0 = pat[min(at, len - 1)], q1 = pat[min(at + 4, len - 1)];
+                const bool d0 = at < len && c0 != q0, d1 = at + 4 < len && c1 != q1;
+                key = d0 ? (at << 1) | (int)(c0 < q0) : d1 ? ((at + 4) << 1) | (int)(c1 < q1) : (len << 1);
+                key = min(key, __shfl_xor_sync(0xffffffffu, key, 1));
+                key = min(key, __shfl_xor_sync(0xffffffffu, key, 2));
+            }
+            const int t0 = at + 8;                                                // the group's tokens so far: [at - part, + 8)
+            const bool more = active && key == (len << 1) && t0 - part < len;    // the same for the lanes of a group
+            if (__any_sync(0xffffffffu, more)) {
                 unsigned ne = 0, lt = 0;
-                int c[2];
+                int c[6];
 #pragma unroll
-                for (int i = 0; i < 2; ++i) c[i] = (active && t0 + 4 * i < len) ? corpus[(int64_t)s_mid + t0 + 4 * i] : 0;
+                for (int i = 0; i < 6; ++i) c[i] = (more && t0 + 4 * i < len) ? corpus[(int64_t)s_mid + t0 + 4 * i] : 0;
 #pragma unroll
-                for (int i = 0; i < 2; ++i) {
+                for (int i = 0; i < 6; ++i) {
                     const int q = pat[min(t0 + 4 * i, len - 1)];
                     ne |= (unsigned)(t0 + 4 * i < len && c[i] != q) << i;
                     lt |= (unsigned)(c[i] < q) << i;
                 }
                 const int f = __ffs(ne) - 1;
-                key = ne ? ((t0 + 4 * f) << 1) | (int)((lt >> f) & 1u) : (len << 1);
-                key = min(key, __shfl_xor_sync(0xffffffffu, key, 1));
-                key = min(key, __shfl_xor_sync(0xffffffffu, key, 2));
-            }
-            const bool more = active && key == (len << 1) && from + 8 < len;      // the same for the lanes of a group
-            if (__any_sync(0xffffffffu, more)) {
-                unsigned ne = 0, lt = 0;
-                int c[6];
-#pragma unroll
-                for (int i = 0; i < 6; ++i) c[i] = (more && t0 + 8 + 4 * i < len) ? corpus[(int64_t)s_mid + t0 + 8 + 4 * i] : 0;
-#pragma unroll
-                for (int i = 0; i < 6; ++i) {
-                    const int q = pat[min(t0 + 8 + 4 * i, len - 1)];
-                    ne |= (unsigned)(t0 + 8 + 4 * i < len && c[i] != q) << i;
-                    lt |= (unsigned)(c[i] < q) << i;
-                }
-                const int f = __ffs(ne) - 1;
-                int key2 = ne ? ((t0 + 8 + 4 * f) << 1) | (int)((lt >> f) & 1u) : (len << 1);
+                int key2 = ne ? ((t0 + 4 * f) << 1) | (int)((lt >> f) & 1u) : (len << 1);
                 key2 = min(key2, __shfl_xor_sync(0xffffffffu, key2, 1));
                 key2 = min(key2, __shfl_xor_sync(0xffffffffu, key2, 2));
                 if (more) key = key2;
             }
             if (active) {
                 const int m = key >> 1;                             // leading tokens that agree
-                if (m < len && (key & 1)) { a = mid + 1; ma = m; mid = mid_r; s_mid = s_r; }
-                else { z = mid; mz = m; mid = mid_l; s_mid = s_l; }
+                if (m < len && (key & 1)) { a = mid + 1; ma = m; mid = mid_r; s_mid = s_r; c0 = r0; c1 = r1; s_l = s_rl; s_r = s_rr; }
+                else { z = mid; mz = m; mid = mid_l; s_mid = s_l; c0 = l0; c1 = l1; s_l = s_ll; s_r = s_lr; }
+                at = nt;
             }
         }
         if (searching) {
