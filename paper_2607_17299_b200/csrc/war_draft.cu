@@ -223,53 +223,11 @@ struct Shared {
     int fin_cnt[kMaxK], fin_start[kMaxK], fin_tok[kMaxK];
     int mode, cur, lo, cnt, depth, n_nodes, thr_shared, long_runs_only, full_lo, full_cnt;
     int n_running, n_cap;
-    int m_lo[32], m_hi[32], m_occ[32];          // per candidate length: lower bound, bucket end, occurs
+    int m_lo[32], m_hi[32], m_occ[32];          // per candidate length: interval [lo, hi) of its pattern, occurs
     int memo_slot;                              // >= 0: the node being expanded goes into this memo entry when it is done
     // a batch of small nodes created in one round (equal counts), expanded by one warp each
     int it_slot[kWarps], it_lo[kWarps], it_cnt[kWarps], it_depth[kWarps], n_items;
 };
-
-// Tokens from index `from` on of the suffix at s against the pattern; returns the sign and, in `matched`, how many
-// leading tokens agree.  Eight corpus tokens, then sixteen at a time, are requested together so their latencies
-// overlap (the corpus has readable slack behind its last separator, and a separator always ends the walk).
-__device__ __noinline__ int compare_suffix(const int32_t* __restrict__ corpus, int64_t s, const int* pat, int len, int from,
-                                              int& matched) {
-    // Branch-free inside a batch: one bit per position for "differs" and one for "corpus token is smaller"; the first
-    // set bit decides.  (A chain of early exits costs a divergent branch per token on a path that is pure latency.)
-    int t = from;
-    {
-        unsigned ne = 0, lt = 0;
-        int c[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) c[i] = corpus[s + t + i];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int p = pat[min(t + i, len - 1)];
-            const bool in = t + i < len;
-            ne |= (unsigned)(in && c[i] != p) << i;
-            lt |= (unsigned)(c[i] < p) << i;
-        }
-        if (ne) { const int f = __ffs(ne) - 1; matched = t + f; return (lt >> f) & 1u ? -1 : 1; }
-        t += 8;
-    }
-    // most comparisons end above; the ones that go on share a long prefix, so fetch far ahead
-    for (; t < len; t += 16) {
-        unsigned ne = 0, lt = 0;
-        int c[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) c[i] = (t + i < len) ? corpus[s + t + i] : 0;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int p = pat[min(t + i, len - 1)];
-            const bool in = t + i < len;
-            ne |= (unsigned)(in && c[i] != p) << i;
-            lt |= (unsigned)(c[i] < p) << i;
-        }
-        if (ne) { const int f = __ffs(ne) - 1; matched = t + f; return (lt >> f) & 1u ? -1 : 1; }
-    }
-    matched = len;
-    return 0;
-}
 
 // kCtasPerSm = 2: 64 registers per thread, 296 requests in one wave; 1: 128 registers (nothing spills), used when the
 // grid fits the SMs anyway, which is the low-load case where this kernel's latency matters most.
@@ -404,12 +362,14 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
     };
 
     // ---- longest-suffix match ----
-    // Warps 0-3: four lanes per candidate length (thread t: length t / 4 + 1, every fourth token from t % 4 on behind the
-    // known common prefix), so one probe of the binary search compares up to 32 tokens in a single memory latency whatever
-    // the depth of the match.  The four lanes of a group hold the same search state.
+    // Warps 0-3 find the lower end of every candidate length's interval, warps 4-7 at the same time the upper end: four
+    // lanes per length (thread t: length (t % 128) / 4 + 1, every fourth token from t % 4 on behind the known common
+    // prefix), so one probe of a binary search compares up to 32 tokens in a single memory latency whatever the depth of
+    // the match.  The four lanes of a group hold the same search state.
     const int tl = min(max(my_tl, 0), P);
-    if (warp < 4) {
-        const int len = (tid >> 2) + 1, part = tid & 3;
+    if (warp < 8) {
+        const bool upper = warp >= 4;                             // first suffix above every suffix that starts with the pattern
+        const int len = ((tid & 127) >> 2) + 1, part = tid & 3;
         const int* pat = sh.pat + (P - len);
         int lo = 0, bucket_hi = 0;
         bool occurs = false, searching = false;
@@ -423,7 +383,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
                 searching = len > 1 && occurs;
             }
         }
-        // lower bound by binary search; it remembers how many tokens the pattern shares with the suffixes at its
+        // bound by binary search; it remembers how many tokens the pattern shares with the suffixes at its
         // current ends, so comparisons restart there (all bucket members share token 0).  The search is pipelined two
         // probes deep so that a step costs one memory latency instead of two or three: while the current probe is
         // compared, the first tokens of BOTH possible next probes are on their way (their suffix-array entries came
@@ -440,7 +400,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             c0 = at < len ? corpus[(int64_t)s_mid + at] : 0;
             c1 = at + 4 < len ? corpus[(int64_t)s_mid + at + 4] : 0;
         }
-        while (__any_sync(0xffffffffu, a < z)) {                  // first suffix >= pattern
+        while (__any_sync(0xffffffffu, a < z)) {                  // first suffix >= pattern (upper: > every match)
             const bool active = a < z;
             const int mid_l = a + ((mid - a) >> 1), mid_r = mid + 1 + ((z - mid - 1) >> 1);
             const bool has_l = active && a < mid, has_r = active && mid + 1 < z;
@@ -484,27 +444,31 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
             }
             if (active) {
                 const int m = key >> 1;                             // leading tokens that agree
-                if (m < len && (key & 1)) { a = mid + 1; ma = m; mid = mid_r; s_mid = s_r; c0 = r0; c1 = r1; s_l = s_rl; s_r = s_rr; }
+                if (m < len ? (key & 1) != 0 : upper) { a = mid + 1; ma = m; mid = mid_r; s_mid = s_r; c0 = r0; c1 = r1; s_l = s_rl; s_r = s_rr; }
                 else { z = mid; mz = m; mid = mid_l; s_mid = s_l; c0 = l0; c1 = l1; s_l = s_ll; s_r = s_lr; }
                 at = nt;
             }
         }
-        if (searching) {
-            lo = a;
-            // the pattern occurs iff the suffix there starts with it: that suffix was the last probe that was not
-            // below the pattern, and mz tokens of it agreed
-            occurs = lo < bucket_hi && mz == len;
+        if (!upper) {
+            if (searching) {
+                lo = a;
+                // the pattern occurs iff the suffix there starts with it: that suffix was the last probe that was not
+                // below the pattern, and mz tokens of it agreed
+                occurs = lo < bucket_hi && mz == len;
+            }
+            if (part == 0) { sh.m_lo[len - 1] = lo; sh.m_occ[len - 1] = occurs; }
+        } else if (part == 0) {
+            sh.m_hi[len - 1] = searching ? a : bucket_hi;         // a one-token pattern's interval is its bucket
         }
-        if (part == 0) { sh.m_lo[len - 1] = lo; sh.m_hi[len - 1] = bucket_hi; sh.m_occ[len - 1] = occurs; }
     }
     __syncthreads();
     if (warp == 0) {
-        int lo = sh.m_lo[lane], bucket_hi = sh.m_hi[lane];
+        int lo = sh.m_lo[lane], hi = sh.m_hi[lane];
         const bool occurs = sh.m_occ[lane] != 0;
         const unsigned found = __ballot_sync(0xffffffffu, occurs);
         const int ml_longest = found ? 32 - __clz(found) : 0;
         // candidate c drafts from the suffix of ml_longest - c tokens (every shorter suffix of an occurring string
-        // occurs, and its lane holds that suffix's lower bound); lengths below max(1, min_match) are no candidates
+        // occurs, and its lane holds that suffix's interval); lengths below max(1, min_match) are no candidates
         const int ml = ml_longest - cand;
         if (cand > 0 && ml < max(1, min_match)) {
             n_nodes = 0;
@@ -512,38 +476,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__
         } else {
         const int src = ml > 0 ? ml - 1 : 0;
         lo = __shfl_sync(0xffffffffu, lo, src);
-        bucket_hi = __shfl_sync(0xffffffffu, bucket_hi, src);
-        // Only the longest match needs its upper end: 32-way search by the whole warp over (lo, bucket end) for the
-        // first suffix that no longer starts with the pattern (one probe per lane and round).
-        int hi = bucket_hi;
-        if (ml > 1) {
-            const int* pat = sh.pat + (P - ml);
-            int a = lo + 1, z = bucket_hi, m;                    // positions < a match, positions >= z do not
-            // A deep match has few occurrences, and they end where the LCP array first drops below the match length:
-            // look at the next 128 entries (512 for a match of 8 tokens or more, 128 at a time) before probing the corpus.
-            for (int pass = 0; pass < (ml >= 8 ? 4 : 1) && a < z; ++pass) {
-                int first = 1 << 30;
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const int i = a + r * 32 + lane;
-                    const bool end = i >= z || (int)lcp[i] < ml;
-                    const unsigned e = __ballot_sync(0xffffffffu, end);
-                    if (e && first == (1 << 30)) first = a + r * 32 + __ffs(e) - 1;
-                }
-                if (first != (1 << 30)) { a = min(first, z); z = a; } else a += 128;      // uniform
-            }
-            while (a < z) {
-                const int step = (z - a + 31) / 32;
-                const int pos = min(a + lane * step, z - 1);
-                const bool hit = compare_suffix(corpus, sa[pos], pat, ml, 1, m) == 0;
-                const int nm = __popc(__ballot_sync(0xffffffffu, hit));          // hits are a prefix of the lanes
-                if (nm == 32) { a = min(a + 31 * step, z - 1) + 1; continue; }
-                const int z_old = z;
-                z = min(a + nm * step, z_old - 1);
-                if (nm > 0) a = min(a + (nm - 1) * step, z_old - 1) + 1;
-            }
-            hi = a;
-        }
+        hi = __shfl_sync(0xffffffffu, hi, src);
         const int c0 = ml > 0 ? hi - lo : 0;
         // node budget: a longer match earns a larger tree (at most 1 + floor(match_len * fac_num / fac_den) slots)
         n_cap = fac_num > 0 ? min(N, 1 + (int)(((long long)ml * fac_num) / fac_den)) : N;
