@@ -11,6 +11,8 @@
  *   war_index_build / war_index_append   the trajectory cache: suffix array + capped LCP over the corpus
  *   war_draft                            longest-suffix match + frequency-ranked draft token tree
  *   war_draft_scored                     the same from the best-scoring of several suffix lengths
+ *   war_draft_local                      draft trees from each request's own context
+ *   war_draft_pick                       choice between two draft trees by score
  *   war_verify_attn                      tree-masked GQA decode attention over a paged bf16 KV cache
  *   war_accept                           longest root path of the tree that equals the target's tokens
  *   war_commit                           the accepted tokens become context: KV rows, prefix length, tail window
@@ -181,6 +183,41 @@ war_status_t war_draft_scored(const war_index_t* ix, const int32_t* d_tail, cons
                               const war_draft_params_t* params, int32_t n_lengths, void* d_workspace,
                               int32_t* d_match_len, int32_t* d_used_len, int32_t* d_num_nodes,
                               int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream);
+
+/* Drafting from each request's own context (a part of the SuffixDecoding method that Section 3.2 adopts; the paper
+ * does not spell it out): text a rollout has produced or read once tends to come back inside the same trajectory.
+ * d_ctx holds the contexts of all requests back to back (int32 token ids), d_ctx_off [B+1] (int64, DEVICE memory)
+ * their bounds: request b owns c = d_ctx[d_ctx_off[b] .. d_ctx_off[b+1]), L tokens, the last one being the root of
+ * its tree.  No index is kept (a context changes every step): the call scans the contexts.
+ *   match   the largest l <= min(P, tail_len[b], L - 1) such that the last l tokens of c also occur ending at an
+ *           earlier position e <= L - 2 (so that at least one token follows the occurrence inside the context);
+ *           occurrences may overlap each other and the tail.  A token < 0 matches nothing and nothing continues
+ *           into it.
+ *   window  of all occurrences of that suffix only the 32 most recent ones (largest e) are used.
+ *   tree    the rules of war_draft with the window as the occurrence list: count = number of window occurrences
+ *           followed by the slot's root path inside the context (count[0] = size of the window, at most 32); topk,
+ *           min_match, spec_factor, min_prob and the switch (tail_len < 0, spec_batch_limit) act as in war_draft.
+ * Outputs as in war_draft (d_count may be NULL).  A request without tokens gets the root alone with id -1.
+ * Contexts of 2^31 tokens or more set WAR_ERR_INVALID_ARG in the device status and give num_nodes = 0. */
+war_status_t war_draft_local(const int32_t* d_ctx, const int64_t* d_ctx_off, const int32_t* d_tail_len,
+                             const war_draft_params_t* params,
+                             int32_t* d_match_len, int32_t* d_num_nodes,
+                             int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream);
+
+/* Choice between two draft trees per request, e.g. the one from the stored trajectories (war_draft) and the one
+ * from the request's own context (war_draft_local).  A tree's score is (sum of count[j], j = 1 .. num_nodes-1) /
+ * count[0], the number of draft tokens one expects to be accepted under the tree's own statistics (0 when count[0]
+ * is 0); scores are compared exactly (128-bit products).  Tree b is taken only if its score is strictly larger.
+ * All arrays are device memory, [B] or [B, N] as in war_draft; the count arrays of both inputs are required.
+ * d_source [B] receives 0 or 1; the chosen tree is copied to d_match_len, d_num_nodes, d_ids, d_parent and, if not
+ * NULL, d_count.  The outputs must not alias the inputs. */
+war_status_t war_draft_pick(int32_t B, int32_t N,
+                            const int32_t* a_match_len, const int32_t* a_num_nodes, const int32_t* a_ids,
+                            const int32_t* a_parent, const int32_t* a_count,
+                            const int32_t* b_match_len, const int32_t* b_num_nodes, const int32_t* b_ids,
+                            const int32_t* b_parent, const int32_t* b_count,
+                            int32_t* d_source, int32_t* d_match_len, int32_t* d_num_nodes,
+                            int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Verification attention (paper Section 3.2: the predicted tokens "are then verified by the target model"

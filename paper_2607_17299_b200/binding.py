@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "WAR_OK", 1: "WAR_ERR_INVALID_ARG", 2: "WAR_ERR_OOM", 3: "WAR
                 5: "WAR_ERR_TIMEOUT", 6: "WAR_ERR_UNSUPPORTED", 7: "WAR_ERR_BAD_TREE", 8: "WAR_ERR_BAD_PAGE"}
 
 EXPORTS = ["war_index_build", "war_index_append", "war_index_evict", "war_index_export_bytes", "war_index_export",
-           "war_index_import", "war_index_info", "war_index_destroy", "war_draft", "war_draft_scored_workspace_bytes", "war_draft_scored",
+           "war_index_import", "war_index_info", "war_index_destroy", "war_draft", "war_draft_scored_workspace_bytes", "war_draft_scored", "war_draft_local", "war_draft_pick",
            "war_verify_attn_workspace_bytes", "war_verify_attn", "war_verify_attn_noalloc", "war_accept", "war_commit", "war_device_status",
            "war_status_string"]
 
@@ -82,6 +82,10 @@ _lib.war_draft_scored_workspace_bytes.restype = C.c_size_t
 _lib.war_draft_scored_workspace_bytes.argtypes = [C.POINTER(DraftParams), C.c_int32]
 _lib.war_draft_scored.restype = C.c_int
 _lib.war_draft_scored.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(DraftParams), C.c_int32] + [C.c_void_p] * 8
+_lib.war_draft_local.restype = C.c_int
+_lib.war_draft_local.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(DraftParams)] + [C.c_void_p] * 6
+_lib.war_draft_pick.restype = C.c_int
+_lib.war_draft_pick.argtypes = [C.c_int32, C.c_int32] + [C.c_void_p] * 17
 _lib.war_verify_attn_workspace_bytes.argtypes = [C.POINTER(AttnParams)]
 _lib.war_verify_attn.restype = C.c_int
 _lib.war_verify_attn.argtypes = [C.c_void_p] * 7 + [C.POINTER(AttnParams)] + [C.c_void_p] * 4
@@ -224,6 +228,30 @@ def war_draft_scored(ix: Index, d_tail: torch.Tensor, d_tail_len: torch.Tensor, 
                                  _ptr(d_num_nodes, torch.int32), _ptr(d_ids, torch.int32), _ptr(d_parent, torch.int32),
                                  _ptr(d_count, torch.int32), _stream())
     _check("war_draft_scored", code)
+
+
+def war_draft_local(d_ctx: torch.Tensor, d_ctx_off: torch.Tensor, d_tail_len: torch.Tensor, P: int, N: int, topk: int,
+                    min_match: int, d_match_len: torch.Tensor, d_num_nodes: torch.Tensor, d_ids: torch.Tensor,
+                    d_parent: torch.Tensor, d_count: Optional[torch.Tensor], spec_batch_limit: int = 0, spec_factor=(0, 1),
+                    min_prob=(0, 1)) -> None:
+    """d_ctx: int32 tokens of all contexts back to back; d_ctx_off: int64 [B+1] bounds, both on the device."""
+    B = d_ctx_off.numel() - 1
+    p = DraftParams(B, P, N, topk, min_match, spec_batch_limit, spec_factor[0], spec_factor[1], min_prob[0], min_prob[1])
+    code = _lib.war_draft_local(_ptr(d_ctx, torch.int32), _ptr(d_ctx_off, torch.int64), _ptr(d_tail_len, torch.int32),
+                                C.byref(p), _ptr(d_match_len, torch.int32), _ptr(d_num_nodes, torch.int32),
+                                _ptr(d_ids, torch.int32), _ptr(d_parent, torch.int32), _ptr(d_count, torch.int32), _stream())
+    _check("war_draft_local", code)
+
+
+def war_draft_pick(a, b, d_source: torch.Tensor, d_match_len: torch.Tensor, d_num_nodes: torch.Tensor, d_ids: torch.Tensor,
+                   d_parent: torch.Tensor, d_count: Optional[torch.Tensor]) -> None:
+    """a, b: (match_len, num_nodes, ids, parent, count) tensor tuples of the two trees."""
+    B, N = a[2].shape
+    args = [_ptr(t, torch.int32) for t in (*a, *b)]
+    code = _lib.war_draft_pick(B, N, *args, _ptr(d_source, torch.int32), _ptr(d_match_len, torch.int32),
+                               _ptr(d_num_nodes, torch.int32), _ptr(d_ids, torch.int32), _ptr(d_parent, torch.int32),
+                               _ptr(d_count, torch.int32), _stream())
+    _check("war_draft_pick", code)
 
 
 def attn_params(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, page_table: torch.Tensor, scale: float,

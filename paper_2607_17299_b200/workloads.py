@@ -203,6 +203,31 @@ def make_request_tails(cfg: WorkloadConfig, ctx_len: Optional[np.ndarray] = None
     return tails, tail_len
 
 
+def make_request_contexts(cfg: WorkloadConfig, ctx_len: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Whole contexts of the live requests, back to back (int32) with int64 bounds [B+1]: the final stretch of each is
+    the one `make_request_tails` synthesises (so the last P tokens agree with its tails), the part before it comes
+    from the same span recipe on a seed stream of its own.  Templates recur inside a context, which is the
+    self-repetition that drafting from the own context feeds on."""
+    cdf = zipf_cdf(cfg.vocab)
+    templates = make_templates(cfg, cdf)
+    tmpl_flat, tmpl_off = _flatten(templates)
+    rng = np.random.Generator(np.random.PCG64(seed_streams(cfg)[2]))
+    rng_head = np.random.Generator(np.random.PCG64(seed_streams(cfg)[2].spawn(1)[0]))
+    if ctx_len is None:
+        ctx_len = context_lengths(cfg)
+    parts = []
+    for i in range(cfg.B):
+        n = int(min(ctx_len[i], max(2048, 2 * cfg.tmpl_hi)))
+        seq = _span_sequence(rng, n, cfg, templates, tmpl_flat, tmpl_off, cdf)
+        head = int(ctx_len[i]) - n
+        if head > 0:
+            parts.append(_span_sequence(rng_head, head, cfg, templates, tmpl_flat, tmpl_off, cdf))
+        parts.append(seq)
+    off = np.zeros(cfg.B + 1, dtype=np.int64)
+    off[1:] = np.cumsum(np.asarray(ctx_len[:cfg.B], dtype=np.int64))
+    return np.concatenate(parts).astype(np.int32), off
+
+
 # ----------------------------------------------------------------------------------------------
 # bf16 tensors: counter hash -> table of normal quantiles (exact integer ops, any torch device)
 # ----------------------------------------------------------------------------------------------
