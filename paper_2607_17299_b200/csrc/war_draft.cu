@@ -825,8 +825,11 @@ war_draft_select_kernel(CandArrays ca, int B, int C, int N, int32_t* __restrict_
         if (o_len < 0) take = false;
         else if (len < 0) take = true;
         else {
-            const long long l = o_num * den, r = num * o_den;            // o_num / o_den against num / den
-            take = l > r || (l == r && o_best < best);
+            // o_num / o_den against num / den by 128-bit products (counts may need 31 bits, sums 37)
+            const unsigned long long l_hi = __umul64hi((unsigned long long)o_num, (unsigned long long)den), l_lo = (unsigned long long)o_num * (unsigned long long)den;
+            const unsigned long long r_hi = __umul64hi((unsigned long long)num, (unsigned long long)o_den), r_lo = (unsigned long long)num * (unsigned long long)o_den;
+            const bool gt = l_hi > r_hi || (l_hi == r_hi && l_lo > r_lo), eq = l_hi == r_hi && l_lo == r_lo;
+            take = gt || (eq && o_best < best);
         }
         if (take) { len = o_len; den = o_den; num = o_num; best = o_best; }
     }

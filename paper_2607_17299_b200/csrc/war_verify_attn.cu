@@ -29,8 +29,8 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     __shared__ uint16_t s_order[kMaxPlanB];   // request at each sorted position
     __shared__ uint8_t s_n[kMaxPlanB];        // validated slot count
     __shared__ int s_red[32];
-    __shared__ long long s_sum[32];
-    __shared__ int s_chunk_tiles, s_total, s_one_wave;
+    __shared__ long long s_sum[32], s_sum2[32];
+    __shared__ int s_chunk_tiles, s_total, s_one_wave, s_cstar;
     __shared__ long long s_tot;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -118,33 +118,84 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     }
     __syncthreads();
     const int chunk_tiles = s_chunk_tiles;
-    // Little work (few requests): one unit per CTA instead of many short ones.  Every (request, kv head, row block)
-    // gets a share of the CTAs in proportion to its tiles, rounded down; if that fits the grid it is used: one
-    // pipeline fill and one epilogue per CTA, and far fewer partials to merge.
+    // Little work (few requests): the default chunk (about kTargetUnits units) would cut every request into short
+    // units, and a unit costs about six tiles on top of its own (pipeline fill, Q load, partials written and merged;
+    // calibrated on 2 to 32 requests).
+    // Up to 32 requests, one warp therefore looks for the chunk length c that minimises the estimated time in tiles
+    //     ceil(units(c) / CTAs) * (c + 6),     units(c) = sum over (request, kv head, row block) of ceil(tiles / c),
+    // over c from the default up to the longest request: a coarse grid of 32 lengths (a lane each, every lane walks
+    // the requests), then finer grids around the best.  This covers "one unit per CTA" (units(c) <= CTAs: one pipeline
+    // fill and one epilogue per CTA) as well as a few long units per CTA, and with a dozen requests of very different
+    // lengths it avoids leaving most CTAs idle while the longest request finishes.  Equal estimates take the longer
+    // chunk (fewer partials).  More requests (only with very few kv heads can that be little work): shares of the grid
+    // in proportion to the tiles, rounded down, if that fits the grid and its longest unit beats the default plan.
     const long long tot_all = s_tot;
+    if (B <= 32) {
+        if (warp == 0) {
+            const int t_mine = lane < B ? s_tiles[lane] : 0;
+            const int t_max = __reduce_max_sync(0xffffffffu, lane < B && s_n[lane] > 0 ? t_mine : 0);
+            int c_lo = max(4, chunk_tiles), c_hi = max(t_max, c_lo), best_c = c_lo;
+            while (true) {
+                const int step = max(1, (c_hi - c_lo + 31) / 32);
+                const int cl = min(c_lo + lane * step, c_hi);
+                long long units = 0;
+                for (int q = 0; q < B; ++q) {
+                    const int n = s_n[q], t = s_tiles[q];
+                    if (n > 0 && t > 0) units += (long long)Hkv * ((G * n + kRowBlock - 1) / kRowBlock) * ((t + cl - 1) / cl);
+                }
+                const long long est = ((units + n_ctas - 1) / n_ctas) * (cl + 6);
+                // smallest estimate, then the longest chunk: est < 2^40, cl < 2^20
+                const long long key = (est << 20) | (long long)((1 << 20) - 1 - cl);
+                long long kmin = key;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+                best_c = (1 << 20) - 1 - (int)(kmin & ((1 << 20) - 1));
+                if (step == 1) break;
+                c_lo = max(c_lo, best_c - step + 1);
+                c_hi = min(c_hi, best_c + step - 1);
+            }
+            if (lane == 0) s_cstar = best_c;
+        }
+        __syncthreads();
+    }
+    const int c_best = s_cstar;
     auto chunks_one_wave = [&](int t) -> int {
         if (t <= 0) return 0;
         long long nc = tot_all > 0 ? (long long)t * n_ctas / tot_all : 1;        // tot_all: the tiles of all such triples
         const int cap = max(1, t / 4);                                           // a chunk keeps at least four tiles
         return (int)max(1ll, min(nc, (long long)cap));
     };
-    {
-        long long mine = 0;
+    if (B > 32) {
+        long long mine = 0, mine_chunked = 0;
+        int longest = 0;
 #pragma unroll
-        for (int k = 0; k < kPer; ++k) mine += (long long)chunks_one_wave(r_tiles[k]) * Hkv * r_rbs[k];
-        for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
-        if (lane == 0) s_sum[warp] = mine;
+        for (int k = 0; k < kPer; ++k) {
+            const int nc = chunks_one_wave(r_tiles[k]);
+            mine += (long long)nc * Hkv * r_rbs[k];
+            if (nc > 0 && r_rbs[k] > 0) longest = max(longest, (r_tiles[k] + nc - 1) / nc);
+            mine_chunked += (long long)((r_tiles[k] + chunk_tiles - 1) / chunk_tiles) * Hkv * r_rbs[k];
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            mine += __shfl_xor_sync(0xffffffffu, mine, o);
+            mine_chunked += __shfl_xor_sync(0xffffffffu, mine_chunked, o);
+            longest = max(longest, __shfl_xor_sync(0xffffffffu, longest, o));
+        }
+        __syncthreads();                                                   // s_sum is read above
+        if (lane == 0) { s_sum[warp] = mine; s_sum2[warp] = mine_chunked; s_red[warp] = longest; }
         __syncthreads();
         if (tid == 0) {
-            long long units = 0;
-            for (int i = 0; i < (int)(blockDim.x >> 5); ++i) units += s_sum[i];
-            s_one_wave = units <= n_ctas;
+            long long units = 0, units_chunked = 0;
+            int lg = 0;
+            for (int i = 0; i < (int)(blockDim.x >> 5); ++i) { units += s_sum[i]; units_chunked += s_sum2[i]; lg = max(lg, s_red[i]); }
+            const long long t_one = lg + 2, t_chunked = ((units_chunked + n_ctas - 1) / n_ctas) * (chunk_tiles + 2);
+            s_one_wave = units <= n_ctas && t_one <= t_chunked;
         }
         __syncthreads();
     }
     const bool one_wave = s_one_wave != 0;
     auto chunks_of = [&](int t) -> int {
         if (t <= 0) return 0;
+        if (B <= 32) return (t + c_best - 1) / c_best;
         return one_wave ? chunks_one_wave(t) : (t + chunk_tiles - 1) / chunk_tiles;
     };
     // longest-first order: position = number of requests that rank before this one
