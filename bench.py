@@ -141,6 +141,9 @@ def main():
     ap.add_argument("--score-lengths", type=int, default=1,
                     help="draft from the best-scoring of this many suffix lengths (war_draft_scored) instead of from the "
                          "longest match (war_draft); 1 = war_draft, the configuration the metric is quoted on")
+    ap.add_argument("--own-context", action="store_true",
+                    help="also draft from each request's own context (war_draft_local, on a second stream beside war_draft) "
+                         "and verify the better-scoring tree of the two (war_draft_pick)")
     ap.add_argument("--cuda-graph", action="store_true",
                     help="replay the step (draft, verify attention, accept) from one captured CUDA graph, as the paper's engine "
                          "does for both modes; the per-kernel breakdown and the roofline then come from a second, eagerly "
@@ -274,8 +277,28 @@ def main():
         draft_ws = torch.empty(war.war_draft_scored_workspace_bytes(cfg.B, cfg.P, N, cfg.topk, args.score_lengths),
                                dtype=torch.uint8, device=dev)
 
+    if args.own_context:
+        h_ctx, h_ctx_off = W.make_request_contexts(cfg, ctx)
+        d_ctx, d_ctx_off = torch.from_numpy(h_ctx).to(dev), torch.from_numpy(h_ctx_off).to(dev)
+        i32 = dict(dtype=torch.int32, device=dev)
+        g_tree = [torch.zeros(cfg.B, **i32), torch.zeros(cfg.B, **i32)] + [torch.zeros((cfg.B, N), **i32) for _ in range(3)]
+        l_tree = [torch.zeros(cfg.B, **i32), torch.zeros(cfg.B, **i32)] + [torch.zeros((cfg.B, N), **i32) for _ in range(3)]
+        d_src = torch.zeros(cfg.B, **i32)
+        local_stream = torch.cuda.Stream()
+        local_done = torch.cuda.Event()
+
     def draft():
-        if args.score_lengths > 1:
+        if args.own_context:
+            # the two drafts share no data: the own-context scan runs beside the index lookup, then the better tree is kept
+            main = torch.cuda.current_stream()
+            local_stream.wait_stream(main)
+            with torch.cuda.stream(local_stream):
+                war.war_draft_local(d_ctx, d_ctx_off, d_tl, cfg.P, N, cfg.topk, 1, *l_tree, args.spec_batch_limit)
+                local_done.record(local_stream)
+            war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, *g_tree, args.spec_batch_limit)
+            main.wait_event(local_done)
+            war.war_draft_pick(g_tree, l_tree, d_src, d_ml, d_nn, d_ids, d_par, d_cnt)
+        elif args.score_lengths > 1:
             war.war_draft_scored(ix, d_tails, d_tl, N, cfg.topk, 1, args.score_lengths, draft_ws, d_ml, d_used, d_nn, d_ids,
                                  d_par, d_cnt, args.spec_batch_limit)
         else:
@@ -466,12 +489,14 @@ def main():
             "config": dict(base_config, kernel="tcgen05" if args.kernel == 0 else "cuda-core",
                            **({"spec_batch_limit": args.spec_batch_limit} if args.spec_batch_limit else {}),
                            **({"score_lengths": args.score_lengths} if args.score_lengths > 1 else {}),
+                           **({"own_context": True, "own_context_share": float(d_src.float().mean().item())}
+                              if args.own_context else {}),
                            **({"launch": "one CUDA graph per step", "eager_ms_per_step": eager_ms / args.steps}
                               if args.cuda_graph else {})),
             "clocks": clocks.summary(),
             "e2e": {"value": verified_all / (e2e_ms / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
-            "gpu_launches": (LAUNCHES_PER_STEP + (args.score_lengths > 1)) * args.steps,
+            "gpu_launches": (LAUNCHES_PER_STEP + (args.score_lengths > 1) + 2 * args.own_context) * args.steps,
             "roofline": ({"bound": "tensor", "achieved": flops / (attn_ms * 1e-3) / 1e12, "peak": peak_tf, "unit": "TFLOP/s",
                           "frac": t_tensor / (attn_ms * 1e-3), "traffic": traffic, "flops_per_launch": flops,
                           "peak_source": "measured (MEASURED_PEAKS.json bf16_tflops_sustained)" if os.path.exists(peaks_path) else "fallback",

@@ -2,14 +2,19 @@
 //
 // The SuffixDecoding method that the paper adopts (Section 3.2) also drafts from the tokens of the running request
 // itself: text a rollout has produced or read once tends to come back inside the same trajectory.  A context changes
-// every step, so no index is kept for it: one CTA per request scans the context (4 bytes per token, a few microseconds
-// even at 10^5 tokens) for the longest suffix that occurs earlier, keeps the 32 most recent occurrences, and warp 0
-// builds the tree from those with one occurrence per lane: a node is a lane mask plus a depth, its continuations are
-// the groups of equal next tokens (`__match_any_sync`), and offers are taken best-first exactly as in war_draft.
+// every step, so no index is kept for it: a cluster of up to 8 CTAs per request scans the context, a slice each (4
+// bytes per token, a few microseconds even at 10^5 tokens), for the longest suffix that occurs earlier and for its 32
+// most recent occurrences; the slices' results meet in the first CTA's shared memory (distributed shared memory and
+// the hardware cluster barrier: no flags, no spinning).  Warp 0 of that CTA builds the tree with one occurrence per
+// lane: a node is a lane mask plus a depth, its continuations are the groups of equal next tokens
+// (`__match_any_sync`), and offers are taken best-first exactly as in war_draft.
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include "war.h"
 #include "war_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -41,7 +46,9 @@ war_draft_local_kernel(const int32_t* __restrict__ ctx, const int64_t* __restric
                        int prob_den, int32_t* __restrict__ match_len, int32_t* __restrict__ num_nodes, int32_t* __restrict__ ids,
                        int32_t* __restrict__ parent, int32_t* __restrict__ count, int* status_word) {
     __shared__ Shared sh;
-    const int b = blockIdx.x;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank(), nblk = (int)cluster.num_blocks();      // the CTAs of a cluster share a request
+    const int b = blockIdx.x / nblk;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int32_t* o_ids = ids + (size_t)b * N;
     int32_t* o_par = parent + (size_t)b * N;
@@ -50,7 +57,7 @@ war_draft_local_kernel(const int32_t* __restrict__ ctx, const int64_t* __restric
     // workload-aware switch, as in war_draft: every CTA counts the running requests itself
     bool plain = false;
     if (tid == 0) { sh.n_running = 0; sh.best_len = 0; sh.n_occ = 0; sh.stop = 0; }
-    __syncthreads();
+    cluster.sync();                                                       // before any CTA touches another one's shared memory
     if (spec_batch_limit > 0) {
         int c = 0;
         for (int i = tid; i < B; i += kThreads) c += tail_len[i] >= 0;
@@ -68,6 +75,7 @@ war_draft_local_kernel(const int32_t* __restrict__ ctx, const int64_t* __restric
     const int32_t* c = ctx + ctx_off[b];
 
     auto finish = [&](int ml, int n) {                                   // all threads: lengths, then the unused slots
+        if (rank != 0) return;                                           // (every early exit is taken by the whole cluster)
         if (tid == 0) { match_len[b] = ml; num_nodes[b] = n; }
         for (int j = n + tid; j < N; j += kThreads) {
             o_ids[j] = -1; o_par[j] = -1;
@@ -75,7 +83,7 @@ war_draft_local_kernel(const int32_t* __restrict__ ctx, const int64_t* __restric
         }
     };
     if (my_tl < 0 || bad) { finish(0, 0); return; }
-    if (tid == 0) { o_ids[0] = L > 0 ? c[L - 1] : -1; o_par[0] = -1; if (o_cnt) o_cnt[0] = 0; }
+    if (tid == 0 && rank == 0) { o_ids[0] = L > 0 ? c[L - 1] : -1; o_par[0] = -1; if (o_cnt) o_cnt[0] = 0; }
     int maxlen = min(min(P, my_tl), L - 1);
     if (plain || maxlen <= 0) { finish(0, 1); return; }
 
@@ -89,17 +97,20 @@ war_draft_local_kernel(const int32_t* __restrict__ ctx, const int64_t* __restric
     }
     if (maxlen == 0) { finish(0, 1); return; }
 
+    // this CTA's slice of the end positions 0 .. L - 2
+    const int slice = (L - 1 + nblk - 1) / nblk;
+    const int s_lo = min(rank * slice, L - 1), s_hi = min(s_lo + slice, L - 1);
     // ---- pass 1: the longest suffix that also ends at some position e <= L - 2 ----
     // (kScanDepth coalesced loads per thread are in flight together: a CTA alone has to cover the latency)
     {
         const int last = sh.pat[0];
         int best = 0;
-        for (int base = 0; base <= L - 2; base += kChunk) {
+        for (int base = s_lo; base < s_hi; base += kChunk) {
             int v[kScanDepth];
 #pragma unroll
             for (int k = 0; k < kScanDepth; ++k) {
                 const int e = base + k * kThreads + tid;
-                v[k] = e <= L - 2 ? c[e] : -1;
+                v[k] = e < s_hi ? c[e] : -1;
             }
 #pragma unroll
             for (int k = 0; k < kScanDepth; ++k) {
@@ -112,19 +123,19 @@ war_draft_local_kernel(const int32_t* __restrict__ ctx, const int64_t* __restric
             }
         }
         best = __reduce_max_sync(0xffffffffu, best);
-        if (lane == 0 && best > 0) atomicMax(&sh.best_len, best);
+        if (lane == 0 && best > 0) atomicMax(cluster.map_shared_rank(&sh.best_len, 0), best);     // the first CTA collects
     }
-    __syncthreads();
-    const int ml = sh.best_len;
-    if (ml == 0) { finish(0, 1); return; }
+    cluster.sync();
+    const int ml = *cluster.map_shared_rank(&sh.best_len, 0);
+    if (ml == 0) { cluster.sync(); finish(0, 1); return; }             // (nobody leaves while its memory may be read)
 
     // ---- pass 2: its most recent occurrences, kChunk positions at a time from the end of the context ----
-    for (int hi = L - 1; hi > 0; hi -= kChunk) {                          // positions [hi - kChunk, hi)
+    for (int hi = s_hi; hi > s_lo; hi -= kChunk) {                        // positions [max(hi - kChunk, s_lo), hi)
         int v[kScanDepth];
 #pragma unroll
         for (int k = 0; k < kScanDepth; ++k) {
             const int e = hi - kChunk + k * kThreads + tid;
-            v[k] = e >= ml - 1 ? c[e] : -1;
+            v[k] = e >= max(ml - 1, s_lo) ? c[e] : -1;
         }
         unsigned hits = 0;
 #pragma unroll
@@ -158,6 +169,22 @@ war_draft_local_kernel(const int32_t* __restrict__ ctx, const int64_t* __restric
         __syncthreads();
         if (sh.stop) break;
     }
+    // the slices' lists meet in the first CTA, most recent slice first
+    cluster.sync();
+    if (rank == 0 && warp == 0 && nblk > 1) {
+        int have = 0, mine = 0;
+        for (int r = nblk - 1; r >= 0 && have < kMaxOcc; --r) {
+            const int n_r = min(*cluster.map_shared_rank(&sh.n_occ, r), kMaxOcc - have);
+            if (lane >= have && lane < have + n_r) mine = cluster.map_shared_rank(sh.occ, r)[lane - have];
+            have += n_r;
+        }
+        __syncwarp();
+        if (lane < have) sh.occ[lane] = mine;
+        if (lane == 0) sh.n_occ = have;
+    }
+    cluster.sync();                                                       // the other CTAs' lists have been read
+    if (rank != 0) return;
+    __syncthreads();
     const int n_occ = sh.n_occ;                                           // >= 1: pass 1 saw one
 
     // ---- the tree: warp 0, one occurrence per lane ----
@@ -280,12 +307,21 @@ extern "C" war_status_t war_draft_local(const int32_t* d_ctx, const int64_t* d_c
     if (!d_ctx || !d_ctx_off || !d_tail_len || !d_match_len || !d_num_nodes || !d_ids || !d_parent) return WAR_ERR_INVALID_ARG;
     int* status_word = war_status_word();
     if (!status_word) return WAR_ERR_CUDA;
-    war_draft_local_kernel<<<p->B, kThreads, 0, stream>>>(d_ctx, d_ctx_off, d_tail_len, p->B, p->P, p->N, p->topk, p->min_match,
-                                                         p->spec_batch_limit, p->spec_factor_num,
-                                                         p->spec_factor_num > 0 ? p->spec_factor_den : 1, p->min_prob_num,
-                                                         p->min_prob_num > 0 ? p->min_prob_den : 1, d_match_len, d_num_nodes,
-                                                         d_ids, d_parent, d_count, status_word);
-    WAR_LAUNCH_CHECK();
+    // CTAs per request: as many as still leave the whole grid a few waves at most
+    const int nblk = p->B <= 128 ? 8 : p->B <= 256 ? 4 : p->B <= 512 ? 2 : 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p->B * nblk);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = nblk; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int fac_den = p->spec_factor_num > 0 ? p->spec_factor_den : 1, prob_den = p->min_prob_num > 0 ? p->min_prob_den : 1;
+    WAR_CUDA_TRY(cudaLaunchKernelEx(&cfg, war_draft_local_kernel, d_ctx, d_ctx_off, d_tail_len, (int)p->B, (int)p->P, (int)p->N,
+                                    (int)p->topk, (int)p->min_match, (int)p->spec_batch_limit, (int)p->spec_factor_num, fac_den,
+                                    (int)p->min_prob_num, prob_den, d_match_len, d_num_nodes, d_ids, d_parent, d_count, status_word));
     return WAR_OK;
 }
 
