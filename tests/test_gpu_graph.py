@@ -129,3 +129,67 @@ def test_one_graph_serves_speculative_and_plain_steps(war):
             assert (o[i, h_nn[i]:] == 7.0).all() and (h_nn[i] == 0 or (o[i, 0] != 7.0).any())
     assert war.war_device_status() == 0
     ix.destroy()
+
+
+def test_drafting_variants_replay_from_a_graph(war):
+    """war_draft_scored, war_draft_local (a cluster launch) and war_draft_pick enqueue work only: captured once,
+    replayed on new inputs in the same buffers, bit-identical to eager calls."""
+    from oracle import draft_oracle as D
+    from oracle import local_draft_oracle as L
+    cfg = W.scaled(W.CONFIGS["tiny"], B=6)
+    dev = U.dev()
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(cfg)
+    ctx_len = np.array([900, 3000, 64, 5000, 1200, 700])
+    h_ctx, h_off = W.make_request_contexts(cfg, ctx_len)
+    ix = U.build_index(war, tok, off, cfg.vocab)
+    B, N, k, P = cfg.B, cfg.N, cfg.topk, cfg.P
+    i32 = dict(dtype=torch.int32, device=dev)
+    d_tails, d_tl = torch.from_numpy(tails).to(dev), torch.from_numpy(tl).to(dev)
+    d_ctx, d_off = torch.from_numpy(h_ctx).to(dev), torch.from_numpy(h_off).to(dev)
+    tree = lambda: [torch.zeros(B, **i32), torch.zeros(B, **i32)] + [torch.zeros((B, N), **i32) for _ in range(3)]
+    s_tree, l_tree, p_tree = tree(), tree(), tree()
+    used, src = torch.zeros(B, **i32), torch.zeros(B, **i32)
+    sws = torch.zeros(war.war_draft_scored_workspace_bytes(B, P, N, k, 3), dtype=torch.uint8, device=dev)
+
+    def drafts():
+        war.war_draft_scored(ix, d_tails, d_tl, N, k, 1, 3, sws, s_tree[0], used, *s_tree[1:])
+        war.war_draft_local(d_ctx, d_off, d_tl, P, N, k, 1, *l_tree)
+        war.war_draft_pick(s_tree, l_tree, src, *p_tree)
+
+    def snapshot():
+        torch.cuda.synchronize()
+        return [t.clone() for t in (used, src, *s_tree, *l_tree, *p_tree)]
+
+    drafts()
+    eager = snapshot()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        drafts()
+    torch.cuda.current_stream().wait_stream(side)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        drafts()
+    for t in (used, src, *s_tree, *l_tree, *p_tree):
+        t.fill_(-3)
+    g.replay()
+    for x, y in zip(snapshot(), eager):
+        assert torch.equal(x, y)
+    # new inputs in the same buffers
+    d_tails.copy_(torch.roll(d_tails, 1, dims=0)); d_tl.copy_(torch.roll(d_tl, 1, dims=0))
+    d_ctx.copy_(torch.roll(d_ctx, 17))
+    g.replay()
+    replayed = snapshot()
+    drafts()
+    for x, y in zip(replayed, snapshot()):
+        assert torch.equal(x, y)
+    # and the replay is the checker's answer
+    t2, l2 = d_tails.cpu().numpy(), d_tl.cpu().numpy()
+    w_s = D.draft_scored_batch(D.Corpus(tok, off), t2, l2, N, k, 3)
+    w_l = L.draft_local_batch(d_ctx.cpu().numpy(), h_off, l2, P, N, k)
+    w_p = L.pick_by_score((w_s[0],) + tuple(w_s[2:]), w_l)
+    for gpu, want in zip([src] + p_tree, w_p):
+        assert np.array_equal(gpu.cpu().numpy(), want)
+    assert war.war_device_status() == 0
+    ix.destroy()
