@@ -1,17 +1,20 @@
 // Draft: longest-suffix match against the suffix array, then best-first expansion of the matched
 // interval into a frequency-ranked token tree.  One CTA per request.
 //
-// Match.  Lane l of warp 0 owns the candidate length l+1: it narrows the first-token bucket of its pattern
-// to the suffix-array interval of the whole pattern with two binary searches.  The longest non-empty
-// interval wins (occurrence is monotone in the length, so it is also the first empty one minus one).
+// Match.  Four lanes own each candidate length 1..32 (warps 0-3 the lower end of the pattern's suffix-array interval,
+// warps 4-7 the upper end): a binary search inside the first token's bucket, pipelined two probes deep.  The longest
+// occurring length wins (occurrence is monotone in the length).
 //
 // Tree.  A node is a suffix-array interval [lo, lo+cnt) whose suffixes share the first `depth` tokens.  Its
 // children are the maximal runs between positions with lcp <= depth; a run's token is the suffix's token at
 // `depth`, its count the run length.  Suffixes that end there (next entry is a separator) sort first, form
 // runs of one, and are skipped.  Runs arrive in ascending token order, so keeping the first-seen run on equal
-// counts is the (count descending, token ascending) rule.  Short intervals are scanned by warp 0, long ones
-// by all warps over contiguous spans whose edge runs are stitched afterwards.  The pool of offered children
-// lives in shared memory; the next slot is its maximum under (count desc, parent slot asc, token asc).
+// counts is the (count descending, token ascending) rule.  Intervals of at most 32 suffixes are expanded in
+// registers, longer ones are answered by the index's memo or scanned (by warp 0, the longest by all warps over
+// contiguous spans whose edge runs are stitched afterwards).  The k offers of a slot form a sorted list in shared
+// memory; the next slot is the best list head under (count desc, parent slot asc), which equals the rule
+// (count desc, parent slot asc, token asc).  Warp 0 drives the expansion and meets the other warps at the block
+// barrier only for the turns that need them.
 #include <climits>
 #include "war_common.cuh"
 #include "war_index.cuh"
