@@ -8,7 +8,7 @@
 // Tiles alternate between two softmax groups, each with its own S/P region, running (max, sum) and O accumulator
 // in TMEM; the two partial results are merged once per unit.  Nothing synchronises the groups per tile.
 // Warp roles:  warp 8   producer: reads the page table, issues one TMA tensor copy per (page, head) into a ring of
-//                       32 KB slots in the order the tensor pipe consumes them (K0 K1 V0 K2 V1 ...); no multicast,
+//                       32 KB slots in the order the tensor pipe consumes them (K0 K1 V0 K2 V1 ...); every CTA loads for itself,
 //                       this GPU's memory only
 //              warp 9   MMA issuer (one lane): S(t+2) is queued right behind PV(t); owns the TMEM allocation
 //              warps 0-3 / 4-7  softmax group 0 / 1: one thread per query row (TMEM lane); the whole row of S is
