@@ -5,7 +5,9 @@
 // 128-key tiles.  A tiny planning kernel cuts every request into chunks so that about kTargetUnits units exist,
 // orders requests longest-first and writes the unit table; the attention kernel's persistent CTAs take units in a
 // fixed snake order; units of a split request leave (max, sum, unnormalised output) partials that a combine kernel merges
-// in chunk order.  Everything lives in the caller's workspace, so no call allocates.
+// in chunk order.  With few requests and one row block per kv head the plan is a contiguous split instead: the tiles
+// of all (request, kv head) pairs form one sequence that is cut into equal ranges, one per CTA, so every CTA streams
+// the same number of tiles whatever the lengths of the requests; a pair that crosses a cut is merged the same way.  Everything lives in the caller's workspace, so no call allocates.
 #pragma once
 #include <stdint.h>
 #include "war.h"
@@ -23,8 +25,15 @@ struct AttnReq {
     int base_unit, n_chunks, n_tiles, n_nodes;
 };
 
+constexpr int kMaxPlanCtas = 1024;      // CTAs of the attention grid the plan can describe
+
 struct AttnWorkspace {
-    int* counters;       // [0] next unit to hand out, [1] number of units, [2] chunk size in tiles
+    int* counters;       // [0] next unit to hand out, [1] number of units, [2] chunk size in tiles,
+                         // [3] 1: contiguous split (units of CTA c are cta_first[c] .. cta_first[c+1]), 0: snake deal
+    int* cta_first;      // [kMaxPlanCtas + 1]   contiguous split: first unit of every CTA
+    int* pair_unit0;     // [B, Hkv]             contiguous split: unit of the first chunk of (request, kv head),
+    int* pair_cta0;      // [B, Hkv]             the CTA that runs it (chunk c > 0 is the first unit of CTA cta0 + c)
+    int* pair_chunks;    // [B, Hkv]             and the number of chunks
     AttnReq* req;        // [B]
     uint64_t* anc;       // [B, N] bit a of anc[b, j]: slot a is j or an ancestor of j
     AttnUnit* units;     // [max_units]
@@ -57,6 +66,10 @@ inline AttnWorkspace war_attn_workspace_layout(const war_attn_params_t* p, void*
     size_t at = 0;
     char* b = (char*)base;
     w.counters = (int*)(b + at); at += align(64 * sizeof(int));
+    w.cta_first = (int*)(b + at); at += align(sizeof(int) * (kMaxPlanCtas + 1));
+    w.pair_unit0 = (int*)(b + at); at += align(sizeof(int) * (size_t)p->B * p->Hkv);
+    w.pair_cta0 = (int*)(b + at); at += align(sizeof(int) * (size_t)p->B * p->Hkv);
+    w.pair_chunks = (int*)(b + at); at += align(sizeof(int) * (size_t)p->B * p->Hkv);
     w.req = (AttnReq*)(b + at); at += align(sizeof(AttnReq) * (size_t)p->B);
     w.anc = (uint64_t*)(b + at); at += align(sizeof(uint64_t) * (size_t)p->B * p->N);
     w.units = (AttnUnit*)(b + at); at += align(sizeof(AttnUnit) * (size_t)w.max_units);

@@ -19,6 +19,98 @@ __device__ __forceinline__ uint64_t shfl64(uint64_t v, int src) {
     return ((uint64_t)hi << 32) | lo;
 }
 
+// The contiguous split of the plan (see attn_plan_kernel): units of every CTA, per-pair records for the merge.
+// Kept out of line so that calls which do not use it run through the same code as before.
+__device__ __noinline__ void plan_contiguous(const int* s_tiles, const uint8_t* s_n, long long* s_start, int* s_cnt, int B, int Hkv,
+                                             int n_ctas, AttnWorkspace w) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (warp == 0) {                                             // first tile of every request's pairs in the sequence
+        const long long mine = lane < B && s_n[lane] > 0 ? (long long)s_tiles[lane] * Hkv : 0;
+        long long incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const long long y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+        s_start[lane] = incl - mine;
+        if (lane == 31) s_start[32] = incl;
+    }
+    __syncthreads();
+    const long long t_all = s_start[32];
+    {
+    const int n_used = (int)min((long long)n_ctas, max(1ll, t_all / 4));                  // at least four tiles per CTA
+    auto cut = [&](int c) -> long long { return t_all * c / n_used; };
+    auto req_of = [&](long long x) -> int {              // request whose pairs hold tile x of the sequence
+        int r = 0;
+        for (int q = 1; q < B; ++q) if (s_start[q] <= x && s_n[q] > 0 && s_tiles[q] > 0) r = q;
+        return r;
+    };
+    // how many units each CTA gets: one per pair that overlaps its range
+    for (int c = tid; c < n_used; c += 1024) {
+        int cnt = 0;
+        {
+            const long long lo = cut(c), hi = cut(c + 1);
+            if (hi > lo) {
+                const int r0 = req_of(lo), r1 = req_of(hi - 1);
+                const int p0 = (int)((lo - s_start[r0]) / s_tiles[r0]), p1 = (int)((hi - 1 - s_start[r1]) / s_tiles[r1]);
+                for (int r = r0; r <= r1; ++r) {
+                    if (s_n[r] <= 0 || s_tiles[r] <= 0) continue;
+                    cnt += (r == r1 ? p1 : Hkv - 1) - (r == r0 ? p0 : 0) + 1;
+                }
+            }
+        }
+        s_cnt[c] = cnt;
+    }
+    __syncthreads();
+    if (warp == 0) {                                     // exclusive scan over the CTAs: a segment per lane
+        const int per = (n_used + 31) / 32, c0 = lane * per, c1 = min(n_used, c0 + per);
+        int sum = 0;
+        for (int c = c0; c < c1; ++c) sum += s_cnt[c];
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+        int run = incl - sum;
+        for (int c = c0; c < c1; ++c) { const int x = s_cnt[c]; s_cnt[c] = run; run += x; }
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
+        if (lane == 0) { s_cnt[n_used] = total; w.counters[0] = 0; w.counters[1] = total; w.counters[2] = 0; w.counters[3] = 1; }
+    }
+    __syncthreads();
+    for (int c = tid; c <= n_ctas; c += 1024) w.cta_first[c] = s_cnt[min(c, n_used)];
+    for (int i = tid; i < B; i += 1024) {
+        AttnReq rq;
+        rq.base_unit = -1; rq.n_chunks = 2; rq.n_tiles = s_tiles[i]; rq.n_nodes = s_n[i];  // -1: contiguous split, see pair_chunks
+        w.req[i] = rq;
+    }
+    for (int i = tid; i < B * Hkv; i += 1024)
+        if (s_n[i / Hkv] <= 0 || s_tiles[i / Hkv] <= 0) w.pair_chunks[i] = 0;
+    // the units of every CTA, one thread per CTA
+    auto cta_of = [&](long long x) -> int {              // the CTA whose range holds tile x
+        int c = (int)min((long long)n_used - 1, x * n_used / t_all);
+        while (c + 1 < n_used && cut(c + 1) <= x) ++c;
+        while (c > 0 && cut(c) > x) --c;
+        return c;
+    };
+    for (int c = tid; c < n_used; c += 1024) {
+        const long long lo = cut(c), hi = cut(c + 1);
+        if (hi <= lo) continue;
+        int u = s_cnt[c];
+        const int r0 = req_of(lo), r1 = req_of(hi - 1);
+        for (int r = r0; r <= r1; ++r) {
+            const int t = s_tiles[r];
+            if (s_n[r] <= 0 || t <= 0) continue;
+            const int h0 = r == r0 ? (int)((lo - s_start[r]) / t) : 0, h1 = r == r1 ? (int)((hi - 1 - s_start[r]) / t) : Hkv - 1;
+            for (int h = h0; h <= h1; ++h, ++u) {
+                const long long ps = s_start[r] + (long long)h * t;                      // the pair's first tile
+                const int c0 = cta_of(ps), c1 = cta_of(ps + t - 1);
+                AttnUnit x;
+                x.req = r; x.kvh = h; x.rb = 0;
+                x.tile_begin = (int)(max(lo, ps) - ps); x.tile_end = (int)(min(hi, ps + t) - ps);
+                x.n_chunks = c1 - c0 + 1; x.chunk = c - c0; x.pad = 0;
+                w.units[u] = x;
+                if (c == c0) { w.pair_unit0[r * Hkv + h] = u; w.pair_cta0[r * Hkv + h] = c0; w.pair_chunks[r * Hkv + h] = c1 - c0 + 1; }
+            }
+        }
+    }
+    }
+}
+
 __global__ void __launch_bounds__(1024)
 attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ num_nodes,
                  const int32_t* __restrict__ parent, int B, int N, int Hkv, int G, int page_size, int max_pages, int n_ctas,
@@ -88,6 +180,31 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     }
     __syncthreads();
 
+    // ---- few requests, one row block each: contiguous split ----
+    // The tiles of all (request, kv head) pairs, request after request and head after head, form one sequence of
+    // T_all tiles; CTA c takes the range [c * T_all / n_used, (c + 1) * T_all / n_used).  A pair that crosses a cut is
+    // split there: its first chunk is somewhere in a CTA's list, every further chunk is the first unit of the next CTA.
+    // Every CTA streams the same number of tiles (within one) whatever the requests' lengths are.  It pays where the
+    // tile count per CTA decides the time and pairs have to be cut anyway: more than 64 live rows per kv head (below
+    // that the call is bound by DRAM alone, which does not care which CTA streams what), at least 64 tiles per CTA and
+    // pairs of 128 tiles (16 K tokens) or more on average, none longer than twice the average; measured on 4-32 requests
+    // of three recipes, +2 to +8 % there and a loss elsewhere (short pairs are better left whole, short ranges pay for
+    // the extra unit per CTA, one very long request among short ones is better served by the search below).
+    if (B <= 32 && n_ctas <= kMaxPlanCtas) {
+        // every warp works the rule out for itself (a lane per request): no barrier on the way of the calls that do not use it
+        const int n = lane < B ? s_n[lane] : 0, t = lane < B ? s_tiles[lane] : 0;
+        const int rows_max = __reduce_max_sync(0xffffffffu, G * n);
+        const int pairs = __reduce_add_sync(0xffffffffu, n > 0 && t > 0 ? Hkv : 0);
+        const int t_max = __reduce_max_sync(0xffffffffu, n > 0 ? t : 0);
+        const int t_sum = __reduce_add_sync(0xffffffffu, n > 0 ? t : 0);      // < 2^31: at most 32 requests of < 2^24 tiles
+        const long long t_all = (long long)t_sum * Hkv;
+        if (rows_max > 64 && rows_max <= kRowBlock && t_all >= 64ll * n_ctas && t_all >= 128ll * pairs && (long long)t_max * pairs <= 2 * t_all) {
+            __shared__ long long s_start[33];
+            plan_contiguous(s_tiles, s_n, s_start, s_units, B, Hkv, n_ctas, w);      // (the snake deal's s_units is free here)
+            return;
+        }
+    }
+
     // ---- per request, one thread: weights, order, chunk counts ----
     int r_n[kPer], r_tiles[kPer], r_rbs[kPer], r_pos[kPer], r_nc[kPer];
     long long my_tiles = 0;
@@ -115,6 +232,7 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         s_one_wave = 0;
         w.counters[0] = 0;
         w.counters[2] = (int)ct;
+        w.counters[3] = 0;
     }
     __syncthreads();
     const int chunk_tiles = s_chunk_tiles;
@@ -286,16 +404,27 @@ attn_combine_kernel(AttnWorkspace w, int N, int Hq, int Hkv, int G, __nv_bfloat1
     const int r = blockIdx.y * kCombineWarps + (threadIdx.x >> 5);
     if (r >= R) return;
     const int rb = r / kRowBlock, rr = r % kRowBlock;
-    const int u0 = rq.base_unit + kvh * rbs + rb, ustep = Hkv * rbs;       // unit of chunk c = u0 + c * ustep
+    const int u0 = rq.base_unit + kvh * rbs + rb, ustep = Hkv * rbs;       // snake deal: unit of chunk c = u0 + c * ustep
+    const bool contiguous = rq.base_unit < 0;                             // (the flag rides in the record that is read anyway)
+    const int pair = i * Hkv + kvh;
+    const int n_chunks = contiguous ? w.pair_chunks[pair] : rq.n_chunks;
+    if (n_chunks <= 1) return;                                             // the attention kernel wrote the result itself
+    const int first_unit = contiguous ? w.pair_unit0[pair] : u0, first_cta = contiguous ? w.pair_cta0[pair] : 0;
+    auto unit_of = [&](int c) -> int {
+        if (!contiguous) return u0 + c * ustep;
+        return c == 0 ? first_unit : w.cta_first[first_cta + c];           // a later chunk opens the next CTA's list
+    };
+    const int my_unit = contiguous && lane < n_chunks ? unit_of(lane) : 0;   // contiguous split: the first 32 chunks' units, one per lane
     float M = -CUDART_INF_F;
-    for (int c = lane; c < rq.n_chunks; c += 32)
-        M = fmaxf(M, w.part_ml[((size_t)(u0 + c * ustep) * w.rows + rr) * 2]);
+    for (int c = lane; c < n_chunks; c += 32)
+        M = fmaxf(M, w.part_ml[((size_t)(contiguous && c < 32 ? my_unit : unit_of(c)) * w.rows + rr) * 2]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     float l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = 0; c < rq.n_chunks; ++c) {
-        const size_t base = (size_t)(u0 + c * ustep) * w.rows + rr;
+    for (int c = 0; c < n_chunks; ++c) {
+        const int uc = !contiguous ? u0 + c * ustep : c < 32 ? __shfl_sync(0xffffffffu, my_unit, c) : unit_of(c);   // (warp-uniform)
+        const size_t base = (size_t)uc * w.rows + rr;
         const float2 ml = *reinterpret_cast<const float2*>(w.part_ml + base * 2);
         const float4 o = *reinterpret_cast<const float4*>(w.part_o + base * 128 + lane * 4);
         const float sc = ml.x == -CUDART_INF_F ? 0.f : exp2f(ml.x - M);

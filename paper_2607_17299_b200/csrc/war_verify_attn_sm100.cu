@@ -86,6 +86,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     const uint32_t sQ = smem_u32(smem + kOffQ), sRing = smem_u32(smem + kOffRing);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_units = a.w.counters[1];
+    // k-th unit of this CTA: its own contiguous list, or the snake deal of the longest-first list
+    const bool contiguous = a.w.counters[3] != 0 && gridDim.x <= (unsigned)kMaxPlanCtas;
+    const int list_first = contiguous ? a.w.cta_first[blockIdx.x] : 0, list_end = contiguous ? a.w.cta_first[blockIdx.x + 1] : 0;
+    auto unit_at = [&](int k) -> int {
+        if (contiguous) return list_first + k < list_end ? list_first + k : n_units;
+        return snake_unit(k, blockIdx.x, gridDim.x);
+    };
     const int pages_per_tile = kTileKeys / a.page_size;
     const uint32_t page_bytes = (uint32_t)a.page_size * 256u;
 
@@ -117,7 +124,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         uint32_t ld = 0;
         bool ok = true;
         for (int k = 0; ok; ++k) {
-            const int u = snake_unit(k, blockIdx.x, gridDim.x);
+            const int u = unit_at(k);
             if (u >= n_units) break;
             const AttnUnit un = a.w.units[u];
             const int i = un.req;
@@ -178,7 +185,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         const uint32_t v_step = (kTokenMajor ? 2048u : 4096u) >> 4;              // 16 keys of V
         bool ok = true;
         for (int k = 0; ok; ++k) {
-            const int u = snake_unit(k, blockIdx.x, gridDim.x);
+            const int u = unit_at(k);
             if (u >= n_units) break;
             const AttnUnit un = a.w.units[u];
             const int T = un.tile_end - un.tile_begin;
@@ -257,7 +264,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         uint32_t ld0 = 0, cgm = 0, cg_other = 0, units_done = 0;    // cgm: tiles this group has processed so far
         bool ok = true;
         for (int k = 0; ok; ++k) {
-            const int u = snake_unit(k, blockIdx.x, gridDim.x);
+            const int u = unit_at(k);
             if (u >= n_units) break;
             const AttnUnit un = a.w.units[u];
             const int i = un.req;
