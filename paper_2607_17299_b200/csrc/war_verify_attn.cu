@@ -20,46 +20,56 @@ __device__ __forceinline__ uint64_t shfl64(uint64_t v, int src) {
 }
 
 // The contiguous split of the plan (see attn_plan_kernel): units of every CTA, per-pair records for the merge.
-// Kept out of line so that calls which do not use it run through the same code as before.
-__device__ __noinline__ void plan_contiguous(const int* s_tiles, const uint8_t* s_n, long long* s_start, int* s_cnt, int B, int Hkv,
-                                             int n_ctas, AttnWorkspace w) {
+// Kept out of line so that calls which do not use it run through the same code as before.  All positions are 32-bit
+// (the caller checked that the sequence has fewer than 2^31 tiles) and the cuts are worked out once, one 64-bit division
+// per CTA in parallel: everything after that is additions, comparisons and 32-bit divisions.
+__device__ __noinline__ void plan_contiguous(const int* s_tiles, const uint8_t* s_n, int* s_start, int* s_cnt, int* s_cut, int B,
+                                             int Hkv, int n_ctas, AttnWorkspace w) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (warp == 0) {                                             // first tile of every request's pairs in the sequence
-        const long long mine = lane < B && s_n[lane] > 0 ? (long long)s_tiles[lane] * Hkv : 0;
-        long long incl = mine;
+        const int mine = lane < B && s_n[lane] > 0 ? s_tiles[lane] * Hkv : 0;
+        int incl = mine;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const long long y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
         s_start[lane] = incl - mine;
         if (lane == 31) s_start[32] = incl;
     }
     __syncthreads();
-    const long long t_all = s_start[32];
-    {
-    const int n_used = (int)min((long long)n_ctas, max(1ll, t_all / 4));                  // at least four tiles per CTA
-    auto cut = [&](int c) -> long long { return t_all * c / n_used; };
-    auto req_of = [&](long long x) -> int {              // request whose pairs hold tile x of the sequence
+    const int t_all = s_start[32];
+    const int n_used = min(n_ctas, max(1, t_all / 4));           // at least four tiles per CTA
+    for (int c = tid; c <= n_used; c += 1024) s_cut[c] = (int)((long long)t_all * c / n_used);
+    __syncthreads();
+    auto req_of = [&](int x) -> int {                            // request whose pairs hold tile x of the sequence
         int r = 0;
         for (int q = 1; q < B; ++q) if (s_start[q] <= x && s_n[q] > 0 && s_tiles[q] > 0) r = q;
         return r;
     };
-    // how many units each CTA gets: one per pair that overlaps its range
-    for (int c = tid; c < n_used; c += 1024) {
+    auto cta_of = [&](int x) -> int {                            // the CTA whose range holds tile x (ranges are equal within one)
+        int c = min(n_used - 1, x / max(1, t_all / n_used));       // a guess in 32 bits, then at most a few steps
+        while (c + 1 < n_used && s_cut[c + 1] <= x) ++c;
+        while (c > 0 && s_cut[c] > x) --c;
+        return c;
+    };
+    // the units of every CTA, one thread per CTA: first how many (one per pair that overlaps its range), then, after
+    // a scan, the units themselves
+    int r0 = 0, r1 = -1, h_first = 0, h_last = 0, lo = 0, hi = 0;
+    if (tid < n_used) {
+        lo = s_cut[tid]; hi = s_cut[tid + 1];
+        if (hi > lo) {
+            r0 = req_of(lo); r1 = req_of(hi - 1);
+            h_first = (lo - s_start[r0]) / s_tiles[r0]; h_last = (hi - 1 - s_start[r1]) / s_tiles[r1];
+        }
+    }
+    for (int c = tid; c < n_used; c += 1024) {                   // (n_used <= 1024: one pass)
         int cnt = 0;
-        {
-            const long long lo = cut(c), hi = cut(c + 1);
-            if (hi > lo) {
-                const int r0 = req_of(lo), r1 = req_of(hi - 1);
-                const int p0 = (int)((lo - s_start[r0]) / s_tiles[r0]), p1 = (int)((hi - 1 - s_start[r1]) / s_tiles[r1]);
-                for (int r = r0; r <= r1; ++r) {
-                    if (s_n[r] <= 0 || s_tiles[r] <= 0) continue;
-                    cnt += (r == r1 ? p1 : Hkv - 1) - (r == r0 ? p0 : 0) + 1;
-                }
-            }
+        for (int r = r0; r <= r1; ++r) {
+            if (s_n[r] <= 0 || s_tiles[r] <= 0) continue;
+            cnt += (r == r1 ? h_last : Hkv - 1) - (r == r0 ? h_first : 0) + 1;
         }
         s_cnt[c] = cnt;
     }
     __syncthreads();
-    if (warp == 0) {                                     // exclusive scan over the CTAs: a segment per lane
+    if (warp == 0) {                                             // exclusive scan over the CTAs: a segment per lane
         const int per = (n_used + 31) / 32, c0 = lane * per, c1 = min(n_used, c0 + per);
         int sum = 0;
         for (int c = c0; c < c1; ++c) sum += s_cnt[c];
@@ -80,34 +90,25 @@ __device__ __noinline__ void plan_contiguous(const int* s_tiles, const uint8_t* 
     }
     for (int i = tid; i < B * Hkv; i += 1024)
         if (s_n[i / Hkv] <= 0 || s_tiles[i / Hkv] <= 0) w.pair_chunks[i] = 0;
-    // the units of every CTA, one thread per CTA
-    auto cta_of = [&](long long x) -> int {              // the CTA whose range holds tile x
-        int c = (int)min((long long)n_used - 1, x * n_used / t_all);
-        while (c + 1 < n_used && cut(c + 1) <= x) ++c;
-        while (c > 0 && cut(c) > x) --c;
-        return c;
-    };
-    for (int c = tid; c < n_used; c += 1024) {
-        const long long lo = cut(c), hi = cut(c + 1);
-        if (hi <= lo) continue;
+    if (tid < n_used && hi > lo) {
+        const int c = tid;
         int u = s_cnt[c];
-        const int r0 = req_of(lo), r1 = req_of(hi - 1);
         for (int r = r0; r <= r1; ++r) {
             const int t = s_tiles[r];
             if (s_n[r] <= 0 || t <= 0) continue;
-            const int h0 = r == r0 ? (int)((lo - s_start[r]) / t) : 0, h1 = r == r1 ? (int)((hi - 1 - s_start[r]) / t) : Hkv - 1;
+            const int h0 = r == r0 ? h_first : 0, h1 = r == r1 ? h_last : Hkv - 1;
             for (int h = h0; h <= h1; ++h, ++u) {
-                const long long ps = s_start[r] + (long long)h * t;                      // the pair's first tile
-                const int c0 = cta_of(ps), c1 = cta_of(ps + t - 1);
+                const int ps = s_start[r] + h * t;                                       // the pair's first tile
+                // a pair that starts in this range and ends in it is whole; otherwise look the two ends up
+                const int c0 = ps >= lo ? c : cta_of(ps), c1 = ps + t <= hi ? c : cta_of(ps + t - 1);
                 AttnUnit x;
                 x.req = r; x.kvh = h; x.rb = 0;
-                x.tile_begin = (int)(max(lo, ps) - ps); x.tile_end = (int)(min(hi, ps + t) - ps);
+                x.tile_begin = max(lo, ps) - ps; x.tile_end = min(hi, ps + t) - ps;
                 x.n_chunks = c1 - c0 + 1; x.chunk = c - c0; x.pad = 0;
                 w.units[u] = x;
                 if (c == c0) { w.pair_unit0[r * Hkv + h] = u; w.pair_cta0[r * Hkv + h] = c0; w.pair_chunks[r * Hkv + h] = c1 - c0 + 1; }
             }
         }
-    }
     }
 }
 
@@ -198,9 +199,9 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         const int t_max = __reduce_max_sync(0xffffffffu, n > 0 ? t : 0);
         const int t_sum = __reduce_add_sync(0xffffffffu, n > 0 ? t : 0);      // < 2^31: at most 32 requests of < 2^24 tiles
         const long long t_all = (long long)t_sum * Hkv;
-        if (rows_max > 64 && rows_max <= kRowBlock && t_all >= 64ll * n_ctas && t_all >= 128ll * pairs && (long long)t_max * pairs <= 2 * t_all) {
-            __shared__ long long s_start[33];
-            plan_contiguous(s_tiles, s_n, s_start, s_units, B, Hkv, n_ctas, w);      // (the snake deal's s_units is free here)
+        if (rows_max > 64 && rows_max <= kRowBlock && t_all >= 64ll * n_ctas && t_all < (1ll << 31) && t_all >= 128ll * pairs && (long long)t_max * pairs <= 2 * t_all) {
+            __shared__ int s_start[33];
+            plan_contiguous(s_tiles, s_n, s_start, s_units, s_units + kMaxPlanCtas + 8, B, Hkv, n_ctas, w);   // (the snake deal's s_units is free here)
             return;
         }
     }
