@@ -112,6 +112,8 @@ __device__ __noinline__ void plan_contiguous(const int* s_tiles, const uint8_t* 
     }
 }
 
+constexpr int kSearchMaxB = 64;           // up to this many requests the chunk length is searched (see below)
+
 __global__ void __launch_bounds__(1024)
 attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ num_nodes,
                  const int32_t* __restrict__ parent, int B, int N, int Hkv, int G, int page_size, int max_pages, int n_ctas,
@@ -249,10 +251,11 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     // chunk (fewer partials).  More requests (only with very few kv heads can that be little work): shares of the grid
     // in proportion to the tiles, rounded down, if that fits the grid and its longest unit beats the default plan.
     const long long tot_all = s_tot;
-    if (B <= 32) {
+    if (B <= kSearchMaxB) {
         if (warp == 0) {
-            const int t_mine = lane < B ? s_tiles[lane] : 0;
-            const int t_max = __reduce_max_sync(0xffffffffu, lane < B && s_n[lane] > 0 ? t_mine : 0);
+            int t_mine = 0;
+            for (int q = lane; q < B; q += 32) if (s_n[q] > 0) t_mine = max(t_mine, s_tiles[q]);
+            const int t_max = __reduce_max_sync(0xffffffffu, t_mine);
             int c_lo = max(4, chunk_tiles), c_hi = max(t_max, c_lo), best_c = c_lo;
             while (true) {
                 const int step = max(1, (c_hi - c_lo + 31) / 32);
@@ -284,7 +287,7 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         const int cap = max(1, t / 4);                                           // a chunk keeps at least four tiles
         return (int)max(1ll, min(nc, (long long)cap));
     };
-    if (B > 32) {
+    if (B > kSearchMaxB) {
         long long mine = 0, mine_chunked = 0;
         int longest = 0;
 #pragma unroll
@@ -314,7 +317,7 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     const bool one_wave = s_one_wave != 0;
     auto chunks_of = [&](int t) -> int {
         if (t <= 0) return 0;
-        if (B <= 32) return (t + c_best - 1) / c_best;
+        if (B <= kSearchMaxB) return (t + c_best - 1) / c_best;
         return one_wave ? chunks_one_wave(t) : (t + chunk_tiles - 1) / chunk_tiles;
     };
     // longest-first order: position = number of requests that rank before this one
