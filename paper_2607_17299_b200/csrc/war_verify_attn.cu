@@ -27,15 +27,17 @@ __device__ __noinline__ void plan_contiguous(const int* s_tiles, const uint8_t* 
                                              int Hkv, int n_ctas, AttnWorkspace w) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (warp == 0) {                                             // first tile of every request's pairs in the sequence
-        const int mine = lane < B && s_n[lane] > 0 ? s_tiles[lane] * Hkv : 0;
-        int incl = mine;
+        const int q0 = 2 * lane, q1 = 2 * lane + 1;              // two requests per lane: B <= 64
+        const int m0 = q0 < B && s_n[q0] > 0 ? s_tiles[q0] * Hkv : 0, m1 = q1 < B && s_n[q1] > 0 ? s_tiles[q1] * Hkv : 0;
+        int incl = m0 + m1;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
-        s_start[lane] = incl - mine;
-        if (lane == 31) s_start[32] = incl;
+        s_start[q0] = incl - m0 - m1;
+        s_start[q1] = incl - m1;
+        if (lane == 31) s_start[64] = incl;
     }
     __syncthreads();
-    const int t_all = s_start[32];
+    const int t_all = s_start[64];
     const int n_used = min(n_ctas, max(1, t_all / 4));           // at least four tiles per CTA
     for (int c = tid; c <= n_used; c += 1024) s_cut[c] = (int)((long long)t_all * c / n_used);
     __syncthreads();
@@ -193,16 +195,21 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     // pairs of 128 tiles (16 K tokens) or more on average, none longer than twice the average; measured on 4-32 requests
     // of three recipes, +2 to +8 % there and a loss elsewhere (short pairs are better left whole, short ranges pay for
     // the extra unit per CTA, one very long request among short ones is better served by the search below).
-    if (B <= 32 && n_ctas <= kMaxPlanCtas) {
-        // every warp works the rule out for itself (a lane per request): no barrier on the way of the calls that do not use it
-        const int n = lane < B ? s_n[lane] : 0, t = lane < B ? s_tiles[lane] : 0;
-        const int rows_max = __reduce_max_sync(0xffffffffu, G * n);
-        const int pairs = __reduce_add_sync(0xffffffffu, n > 0 && t > 0 ? Hkv : 0);
-        const int t_max = __reduce_max_sync(0xffffffffu, n > 0 ? t : 0);
-        const int t_sum = __reduce_add_sync(0xffffffffu, n > 0 ? t : 0);      // < 2^31: at most 32 requests of < 2^24 tiles
+    if (B <= 64 && n_ctas <= kMaxPlanCtas) {
+        // every warp works the rule out for itself (two requests per lane): no barrier on the way of the calls that do not use it
+        int n_mx = 0, prs = 0, t_mx = 0, t_sm = 0;
+        for (int q = lane; q < B; q += 32) {
+            const int n = s_n[q], t = s_tiles[q];
+            n_mx = max(n_mx, n);
+            if (n > 0 && t > 0) { prs += Hkv; t_mx = max(t_mx, t); t_sm += t; }
+        }
+        const int rows_max = G * __reduce_max_sync(0xffffffffu, n_mx);
+        const int pairs = __reduce_add_sync(0xffffffffu, prs);
+        const int t_max = __reduce_max_sync(0xffffffffu, t_mx);
+        const int t_sum = __reduce_add_sync(0xffffffffu, t_sm);               // < 2^31: at most 64 requests of < 2^24 tiles
         const long long t_all = (long long)t_sum * Hkv;
         if (rows_max > 64 && rows_max <= kRowBlock && t_all >= 64ll * n_ctas && t_all < (1ll << 31) && t_all >= 128ll * pairs && (long long)t_max * pairs <= 2 * t_all) {
-            __shared__ int s_start[33];
+            __shared__ int s_start[65];
             plan_contiguous(s_tiles, s_n, s_start, s_units, s_units + kMaxPlanCtas + 8, B, Hkv, n_ctas, w);   // (the snake deal's s_units is free here)
             return;
         }
