@@ -192,7 +192,7 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     // Every CTA streams the same number of tiles (within one) whatever the requests' lengths are.  It pays where the
     // tile count per CTA decides the time and pairs have to be cut anyway: more than 64 live rows per kv head (below
     // that the call is bound by DRAM alone, which does not care which CTA streams what), at least 64 tiles per CTA and
-    // pairs of 128 tiles (16 K tokens) or more on average, none longer than twice the average; measured on 4-32 requests
+    // pairs of 128 tiles (16 K tokens) or more on average, none longer than twice the average; measured on 4-64 requests
     // of three recipes, +2 to +8 % there and a loss elsewhere (short pairs are better left whole, short ranges pay for
     // the extra unit per CTA, one very long request among short ones is better served by the search below).
     if (B <= 64 && n_ctas <= kMaxPlanCtas) {
@@ -249,7 +249,7 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     // Little work (few requests): the default chunk (about kTargetUnits units) would cut every request into short
     // units, and a unit costs about six tiles on top of its own (pipeline fill, Q load, partials written and merged;
     // calibrated on 2 to 32 requests).
-    // Up to 32 requests, one warp therefore looks for the chunk length c that minimises the estimated time in tiles
+    // Up to 64 requests, one warp therefore looks for the chunk length c that minimises the estimated time in tiles
     //     ceil(units(c) / CTAs) * (c + 6),     units(c) = sum over (request, kv head, row block) of ceil(tiles / c),
     // over c from the default up to the longest request: a coarse grid of 32 lengths (a lane each, every lane walks
     // the requests), then finer grids around the best.  This covers "one unit per CTA" (units(c) <= CTAs: one pipeline
