@@ -70,3 +70,12 @@ def test_full_size_sampled(war, name, sample):
     longest, shortest = int(np.argmax(ctx)), int(np.argmin(ctx))
     ml, nn, alen = _step(war, cfg, sample=sorted(set(sample + [longest, shortest])))
     torch.cuda.empty_cache()
+
+
+def test_contiguous_split_beyond_32_requests(war):
+    """48 requests of the Low recipe (128 query rows per kv head, pairs of 128-256 tiles): the attention plan cuts the
+    whole tile sequence into equal ranges, two requests per planning lane; sampled requests against the checker."""
+    cfg = W.scaled(W.CONFIGS["low"], B=48)
+    ctx = W.context_lengths(cfg)
+    _step(war, cfg, sample=sorted({0, 23, 47, int(np.argmax(ctx)), int(np.argmin(ctx))}))
+    torch.cuda.empty_cache()
