@@ -258,12 +258,17 @@ def main():
     del d_tok
     attn = W.make_attention_inputs(cfg, ctx, device=dev)
     B, N = cfg.B, cfg.N
-    d_tails = torch.from_numpy(tails).to(dev)
-    d_tl = torch.from_numpy(tl).to(dev)
     i32 = dict(dtype=torch.int32, device=dev)
-    d_ml, d_nn = torch.zeros(B, **i32), torch.zeros(B, **i32)
-    d_ids, d_par, d_cnt = torch.zeros((B, N), **i32), torch.zeros((B, N), **i32), torch.zeros((B, N), **i32)
-    d_alen, d_path, d_bonus = torch.zeros(B, **i32), torch.zeros((B, N), **i32), torch.zeros(B, **i32)
+    # the step's small integer inputs (tails, their lengths, the target model's tokens) share one allocation as well
+    P_ = tails.shape[1]
+    d_in = torch.zeros(B * (P_ + 1 + N), **i32)
+    d_tails, d_tl, d_target = d_in[:B * P_].view(B, P_), d_in[B * P_:B * (P_ + 1)], d_in[B * (P_ + 1):].view(B, N)
+    d_tails.copy_(torch.from_numpy(tails)); d_tl.copy_(torch.from_numpy(tl))
+    # the step's small integer results live side by side in one allocation, so the end-to-end leg reads them back with one copy
+    d_small = torch.zeros(B * (3 + 3 * N), **i32)
+    d_nn, d_alen, d_bonus = d_small[0:B], d_small[B:2 * B], d_small[2 * B:3 * B]
+    d_ids, d_par, d_path = (d_small[3 * B + k * B * N:3 * B + (k + 1) * B * N].view(B, N) for k in range(3))
+    d_ml, d_cnt = torch.zeros(B, **i32), torch.zeros((B, N), **i32)
     d_out = torch.zeros_like(attn.q)
     d_lse = torch.zeros(attn.q.shape[:3], dtype=torch.float32, device=dev)
     scale = 1.0 / float(np.sqrt(cfg.D))
@@ -314,7 +319,7 @@ def main():
     draft_cold_ms = cold0.elapsed_time(cold1)
     h_ids, h_par, h_nn = d_ids.cpu().numpy(), d_par.cpu().numpy(), d_nn.cpu().numpy()
     targets = W.make_targets(cfg, h_ids, h_par, h_nn, 0)
-    d_target = torch.from_numpy(targets).to(dev)
+    d_target.copy_(torch.from_numpy(targets))
 
     def step(attn_events=None):
         draft()
@@ -388,11 +393,10 @@ def main():
 
     # ---- end to end: per-step inputs start in pinned host memory, results are read back ----
     pin = lambda t: t.cpu().pin_memory()
-    h_q, h_tails, h_tl, h_target = pin(attn.q), pin(d_tails), pin(d_tl), pin(d_target)
-    r_alen, r_path, r_bonus = pin(d_alen), pin(d_path), pin(d_bonus)
-    r_ids, r_par, r_nn, r_out = pin(d_ids), pin(d_par), pin(d_nn), pin(d_out)
-    h2d = sum(t.numel() * t.element_size() for t in (h_q, h_tails, h_tl, h_target))
-    d2h = sum(t.numel() * t.element_size() for t in (r_alen, r_path, r_bonus, r_ids, r_par, r_nn, r_out))
+    h_q, h_in = pin(attn.q), pin(d_in)
+    r_small, r_out = pin(d_small), pin(d_out)                 # trees, accepted paths and bonus tokens; attention output
+    h2d = sum(t.numel() * t.element_size() for t in (h_q, h_in))
+    d2h = sum(t.numel() * t.element_size() for t in (r_small, r_out))
 
     # the queries are only needed by the verification: their copy runs on a second stream beside the draft call
     copy_stream = torch.cuda.Stream()
@@ -401,7 +405,7 @@ def main():
     overlap_q = h_q.numel() * h_q.element_size() >= (4 << 20)   # for a small batch the extra stream costs more than it hides
 
     def e2e_step():
-        d_tails.copy_(h_tails, non_blocking=True); d_tl.copy_(h_tl, non_blocking=True)
+        d_in.copy_(h_in, non_blocking=True)
         if overlap_q:
             copy_stream.wait_stream(main_stream)            # the previous step's readers of q are done
             with torch.cuda.stream(copy_stream):
@@ -409,16 +413,14 @@ def main():
                 q_ready.record(copy_stream)
         else:
             attn.q.copy_(h_q, non_blocking=True)
-        d_target.copy_(h_target, non_blocking=True)
         draft()
         if overlap_q:
             main_stream.wait_event(q_ready)
         war.war_verify_attn(attn.q, attn.k_pool, attn.v_pool, attn.page_table, attn.prefix_len, d_nn, d_par, params, ws,
                             d_out, d_lse)
         war.war_accept(d_ids, d_par, d_nn, d_target, 0, d_alen, d_path, d_bonus)
-        for dst, src in ((r_alen, d_alen), (r_path, d_path), (r_bonus, d_bonus), (r_ids, d_ids), (r_par, d_par),
-                         (r_nn, d_nn), (r_out, d_out)):
-            dst.copy_(src, non_blocking=True)
+        r_small.copy_(d_small, non_blocking=True)
+        r_out.copy_(d_out, non_blocking=True)
         torch.cuda.synchronize()                        # the caller needs the accepted tokens before the next step
 
     for _ in range(2):
