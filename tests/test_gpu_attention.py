@@ -278,3 +278,42 @@ def test_random_shapes_against_the_checker(war, seed):
         _, raw1 = _check(war, cfg, ctx, nn, parent, 0, scale=scale, a=a)
         _, _, raw2 = U.run_attn(war, a, nn, parent, scale, 0)
         assert torch.equal(raw1, raw2)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_mid_size_batches_through_every_plan(war, seed):
+    """2-64 requests of four length mixes (long and uniform: the contiguous split when the trees have more than 64
+    rows; short; lognormal; one very long among short ones: the chunk-length search), random trees, sampled requests
+    against the fp64 checker."""
+    rng = np.random.default_rng(7000 + seed)
+    B = int(rng.integers(2, 65))
+    Hkv, G, N, pg = int(rng.choice([2, 4, 8])), int(rng.choice([2, 4])), int(rng.integers(4, 33)), int(rng.choice([16, 32]))
+    kind = seed % 4
+    if kind == 0:
+        ctx = rng.integers(16000, 30000, B)
+    elif kind == 1:
+        ctx = rng.integers(200, 9000, B)
+    elif kind == 2:
+        ctx = np.clip(np.exp(rng.normal(np.log(6000), 0.8, B)), 130, 40000).astype(int)
+    else:
+        ctx = np.concatenate([rng.integers(500, 3000, B - 1), rng.integers(30000, 60000, 1)])
+    budget = 3e9                                                        # bytes of K/V held on the device
+    if ctx.sum() * Hkv * 512 > budget:
+        ctx = (ctx * (budget / (ctx.sum() * Hkv * 512))).astype(int) + 130
+    cfg = W.scaled(W.CONFIGS["low"], B=B, N=N, Hkv=Hkv, Hq=Hkv * G, page_size=pg)
+    a = W.make_attention_inputs(cfg, np.asarray(ctx), device=U.dev())
+    nn = rng.integers(1, N + 1, B).astype(np.int32)
+    par = np.full((B, N), -1, np.int32)
+    for i in range(B):
+        for j in range(1, nn[i]):
+            par[i, j] = int(rng.integers(0, j))
+    scale = 1.0 / np.sqrt(cfg.D)
+    got, got_lse, _ = U.run_attn(war, a, nn, par, scale, 0)
+    sample = sorted({0, B - 1, int(np.argmax(ctx)), int(rng.integers(0, B))})
+    want = A.verify_attention(a.q, a.k_pool, a.v_pool, a.page_table.cpu().numpy(), a.prefix_len.cpu().numpy(), nn, par, scale,
+                              requests=sample)
+    for i in sample:
+        U.assert_attention_close(got[i], got_lse[i], want[i][0], want[i][1], int(nn[i]))
+    assert war.war_device_status() == 0
+    del a
+    torch.cuda.empty_cache()
