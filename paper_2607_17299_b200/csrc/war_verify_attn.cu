@@ -134,15 +134,28 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     // ---- per request, one warp: validate, ancestor masks by pointer jumping, tile count ----
     // Lane l holds slots l and l + 32.  After round r a slot's mask covers its 2^r nearest ancestors-or-self and its
     // pointer is the 2^r-th ancestor (the root points at itself), so 6 rounds cover any tree of 64 slots.
+    // The parent row is requested together with the slot count (all N entries exist; the ones past n are ignored), and
+    // the next request's while this one is worked on: the warp waits for one memory latency in all, not two per request.
+    const int j0 = lane, j1 = lane + 32;
+    int nx_q0 = 0, nx_q1 = 0, nx_n = 0, nx_pl = 0;
+    if (warp < B) {
+        const int32_t* prow = parent + (size_t)warp * N;
+        nx_q0 = j0 < N ? prow[j0] : 0; nx_q1 = j1 < N ? prow[j1] : 0;
+        nx_n = num_nodes[warp]; nx_pl = prefix_len[warp];
+    }
     for (int i = warp; i < B; i += 32) {
-        int n = num_nodes[i];
-        const int pl = prefix_len[i];
+        const int q0 = nx_q0, q1 = nx_q1;
+        int n = nx_n;
+        const int pl = nx_pl;
+        if (i + 32 < B) {
+            const int32_t* prow = parent + (size_t)(i + 32) * N;
+            nx_q0 = j0 < N ? prow[j0] : 0; nx_q1 = j1 < N ? prow[j1] : 0;
+            nx_n = num_nodes[i + 32]; nx_pl = prefix_len[i + 32];
+        }
         bool bad = n < 0 || n > N || pl < 0;
         if (!bad && n > 0) {
-            const int32_t* prow = parent + (size_t)i * N;
-            const int j0 = lane, j1 = lane + 32;
-            int p0 = (j0 > 0 && j0 < n) ? prow[j0] : 0;
-            int p1 = (j1 < n) ? prow[j1] : 0;
+            int p0 = (j0 > 0 && j0 < n) ? q0 : 0;
+            int p1 = (j1 < n) ? q1 : 0;
             const bool bad_l = (j0 > 0 && j0 < n && (p0 < 0 || p0 >= j0)) || (j1 < n && (p1 < 0 || p1 >= j1));
             bad = __any_sync(0xffffffffu, bad_l);
             if (!bad) {
@@ -391,7 +404,11 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         const int c = local / (Hkv * rbs), rem = local % (Hkv * rbs);
         AttnUnit x;
         x.req = i; x.kvh = rem / rbs; x.rb = rem % rbs;
-        x.tile_begin = (int)((long long)t * c / nc); x.tile_end = (int)((long long)t * (c + 1) / nc);
+        if (t < 32768 && nc < 32768) {                              // 32-bit arithmetic is enough (and several times faster)
+            x.tile_begin = (int)((unsigned)t * (unsigned)c / (unsigned)nc); x.tile_end = (int)((unsigned)t * (unsigned)(c + 1) / (unsigned)nc);
+        } else {
+            x.tile_begin = (int)((long long)t * c / nc); x.tile_end = (int)((long long)t * (c + 1) / nc);
+        }
         x.n_chunks = nc; x.chunk = c; x.pad = 0;
         w.units[u] = x;
     }
