@@ -237,8 +237,16 @@ war_status_t war_draft_pick(int32_t B, int32_t N,
  * (Hq/Hkv) * N <= 512, scale > 0; anything else returns WAR_ERR_UNSUPPORTED / WAR_ERR_INVALID_ARG.
  * Rows j >= num_nodes[b] of d_out / d_lse are left untouched.
  * d_workspace: war_verify_attn_workspace_bytes(params) bytes of device memory, 256-byte aligned, private to
- * the call while it runs (split-KV partial results and the work list live there).
- *   kernel: 0 = default (tensor-core path), 1 = plain CUDA-core path kept for A/B checks.
+ * the call while it runs (split-KV partial results, their arrival counters and the work list live there); its
+ * contents before the call do not matter.
+ *   kernel: 0 = default: the tensor-core kernel; with up to 64 requests (the low-load regime the step exists for)
+ *               the whole call is ONE kernel launch: every thread block works out its own share of the work from
+ *               prefix_len / num_nodes, and a request that was split between blocks is merged by one of them once
+ *               its last piece is there (in a fixed order: results do not depend on timing).  With more requests a
+ *               planning launch precedes the kernel and a combine launch follows it.
+ *           1 = plain CUDA-core kernel, 2 = tensor-core kernel always with the separate planning and combine
+ *               launches; both kept for A/B checks (0 and 2 give the same bits).
+ * Contexts (max_pages_per_req * page_size) must stay below 2^30 tokens.
  * ------------------------------------------------------------------------------------------------ */
 typedef struct {
     int32_t B, N, Hq, Hkv, D, page_size, max_pages_per_req, kernel;
@@ -266,9 +274,9 @@ war_status_t war_verify_attn(const void* d_q, const void* d_kpool, const void* d
  *     WAR_ERR_CAPACITY and launches nothing.
  *   - The first call on each device looks up the array's device address (with that device current); make that
  *     first call before starting any stream capture.
- *   - All calls on a device share the one array, and it keeps the previous call's contents (nothing in it needs
- *     clearing: every call rewrites what it reads).  Two calls that overlap on the GPU, e.g. on two streams,
- *     race on it; run them in stream order.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents (the caller clears
+ *     nothing: a call rewrites what it reads, or recognises it as left over from an earlier call).  Two calls that
+ *     overlap on the GPU, e.g. on two streams, race on it; run them in stream order.
  * ------------------------------------------------------------------------------------------------ */
 #define WAR_VERIFY_ATTN_NOALLOC_MAX_BYTES (64u * 1024u * 1024u)
 war_status_t war_verify_attn_noalloc(const void* d_q, const void* d_kpool, const void* d_vpool,

@@ -1,0 +1,317 @@
+// The verify-attention plan worked out by every CTA for itself (library-internal, device code).
+//
+// With up to kFusedMaxB requests the work decomposition of war_attn_plan.cuh is a closed form of at most 64
+// (prefix_len, num_nodes) pairs, so a separate planning launch costs more than it saves: every persistent CTA of the
+// attention kernel reads those pairs, validates the trees and takes the same decisions as attn_plan_kernel
+// (contiguous split, or searched chunk length + longest-first snake deal).  What stays behind is a table of a few
+// hundred bytes in shared memory from which every warp role derives the CTA's next unit when it gets there; nothing
+// of the plan goes through global memory.
+//
+// A unit of a split (request, kv head, row block) leaves its partial result in a slot of the workspace that every
+// CTA can name without a table:
+//   snake deal        slot = the unit's index in the longest-first list (chunk c of a triple is u0 + c * ustep)
+//   contiguous split  a split pair's first chunk is the LAST unit of its CTA c0 (slot 2*c0 + 1), every further chunk
+//                     is the FIRST unit of the next CTA (slot 2*(c0 + c))
+// The CTA that ran chunk 0 of a split triple merges all its chunks, in chunk order, once its own units are done.
+#pragma once
+#include "war_attn_plan.cuh"
+#include "war_common.cuh"
+
+constexpr int kFusedMaxB = 64;
+constexpr int kFusedMaxCtas = 192;          // a pair can be cut into as many chunks as there are CTAs (see kFusedMaxChunks)
+constexpr int kFusedThreads = 384;
+constexpr int kFusedMaxUnitsTotal = 60000;     // unit offsets are kept as 16-bit numbers
+
+struct FusedPlan {                        // resident in shared memory for the whole kernel
+    int tiles[kFusedMaxB];                // 128-key tiles per request (0: not running or rejected)
+    union {
+        struct {
+            uint16_t pos_base[kFusedMaxB + 2];   // snake deal: first unit of the request at each sorted position
+            uint16_t nc[kFusedMaxB];             // chunks per request
+        } s;
+        int start[kFusedMaxB + 1];        // contiguous split: first tile of each request's pairs in the sequence
+    } u;
+    uint8_t n[kFusedMaxB];                // validated slot count per request
+    uint8_t pos_req[kFusedMaxB];          // snake deal: request at each sorted position (longest first)
+    int mode;                             // 0 snake deal, 1 contiguous split
+    int total;                            // snake deal: number of units
+    int t_all, n_used;                    // contiguous split: tiles in the sequence, CTAs that get a range,
+    int cut_base, cut_rem;                //   t_all / n_used and t_all % n_used
+    int lo, hi, r0, h0;                   // contiguous split: this CTA's range and the pair that holds its first tile
+};
+static_assert(sizeof(FusedPlan) <= 704, "the plan table shares 768 bytes of shared memory");
+
+struct FusedPlanScratch {                 // only while the plan is made (lives in the idle ring)
+    int keys[64];
+    int weight[kFusedMaxB];               // units per chunk of a request: kv heads x row blocks (0: no work)
+    int units_by_pos[kFusedMaxB];
+};
+
+// Host-side rule for taking this path: few requests, and unit offsets that fit 16 bits (the snake deal creates at
+// most kTargetUnits + one unit per (request, kv head, row block)).
+inline bool war_attn_fused_ok(const war_attn_params_t* p, int row_blocks, int n_ctas) {
+    return p->B <= kFusedMaxB && n_ctas <= kFusedMaxCtas && n_ctas >= 1 && p->Hkv <= 255 && p->N <= 255 &&
+           (long long)p->max_pages_per_req * p->page_size < (1ll << 30) &&
+           (long long)kTargetUnits + (long long)p->B * p->Hkv * row_blocks <= kFusedMaxUnitsTotal;
+}
+
+#ifdef __CUDACC__
+namespace fused_plan {
+
+struct Unit {
+    int req, kvh, rb, tile_begin, tile_end, n_chunks, chunk, n_nodes;
+    int slot_base, slot_stride, bump;     // partial of chunk c: slot_base + c * slot_stride (+ bump for c == 0)
+};
+
+// Walks the units of one CTA in the order they are run.  Every warp role keeps its own cursor.
+struct Cursor {
+    int k, r, h;
+};
+
+__device__ __forceinline__ int snake_unit(int k, int cta, int ctas) { return k * ctas + ((k & 1) ? ctas - 1 - cta : cta); }
+
+// ceil(x / d) for 0 <= x, 0 < d, x + d <= 2^24, without an integer division
+__device__ __forceinline__ int ceil_div_small(int x, int d) {
+    int q = __float2int_rz(__fdividef((float)(x + d - 1), (float)d));
+    const int r = (x + d - 1) - q * d;
+    q += (r >= d) - (r < 0);
+    return q;
+}
+
+// The chunk length for up to kFusedMaxB requests: the c in [c_lo, max(c_lo, t_max)] that minimises the estimated time
+//     ceil(units(c) / CTAs) * (c + 6)  tiles,     units(c) = sum over requests of weight * ceil(tiles / c)
+// (a unit costs about six tiles on top of its own: pipeline fill, Q load, partials written and merged).  Equal
+// estimates take the longer chunk.  The first kThreads threads of the block evaluate one candidate each: every length
+// of the range if there are that few, else every step-th one, followed by every length within a step of the best.
+// Called by all threads of the block (block barriers inside); blocks of different sizes find the same length.
+// `keys` is shared scratch of 64 entries.  tiles < 2^23, units(c_lo) < 2^24.
+template <int kThreads>
+__device__ __forceinline__ int chunk_search(const int* tiles, const int* weight, int B, int c_lo, int t_max, int n_ctas,
+                                            int* keys) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int lo = c_lo, hi = max(t_max, c_lo), result = lo;
+#pragma unroll 1
+    while (true) {
+        const int step = (hi - lo + kThreads) / kThreads;          // 1 when every length has a thread
+        const int cl = min(lo + tid * step, hi);
+        int est = 0x7fffffff;
+        if (tid < kThreads) {
+            int units = 0;                                          // (entries from B up to the next multiple of 4 have weight 0)
+#pragma unroll 1
+            for (int q = 0; q < B; q += 4) {
+                int part[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) part[k] = weight[q + k] * ceil_div_small(max(tiles[q + k], 0), cl);
+                units += (part[0] + part[1]) + (part[2] + part[3]);
+            }
+            const int waves = ceil_div_small(units, n_ctas);
+            const long long e = (long long)waves * (cl + 6);
+            est = e < 0x7fffffffll ? (int)e : 0x7ffffffe;
+        }
+        // smallest estimate, then the longest chunk
+        const int est_w = __reduce_min_sync(0xffffffffu, est);
+        const int cl_w = __reduce_max_sync(0xffffffffu, est == est_w ? cl : 0);
+        __syncthreads();                                            // (the previous round's keys have been read)
+        if (lane == 0) { keys[2 * warp] = est_w; keys[2 * warp + 1] = cl_w; }
+        __syncthreads();
+        int best_e = 0x7fffffff;
+        result = 0;
+#pragma unroll 1
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+            const int e = keys[2 * w], c = keys[2 * w + 1];
+            if (e < best_e || (e == best_e && c > result)) { best_e = e; result = c; }
+        }
+        if (step == 1) break;
+        lo = max(lo, result - step + 1);
+        hi = min(hi, result + step - 1);
+    }
+    return result;
+}
+
+// The contiguous split (the tiles of all (request, kv head) pairs as one sequence, cut into equal ranges, a CTA each)
+// balances the CTAs to within one tile and gives every CTA at most two split units, but a range pays for an extra
+// unit wherever a pair ends inside it.  Measured on 4 to 64 requests of three recipes it wins from about 48 tiles per
+// CTA on (one row block per kv head); below that the searched chunk length does better.
+__host__ __device__ __forceinline__ bool contiguous_split_pays(int rows_max, long long t_all, int n_ctas) {
+    return rows_max <= kRowBlock && t_all >= 48ll * n_ctas && t_all < (1ll << 31);
+}
+
+constexpr int kFusedMaxChunks = 192;      // chunks per request at most (what the merge of a row group can hold at once)
+__device__ __forceinline__ int chunk_floor(int t_max) { return max(4, (t_max + kFusedMaxChunks - 1) / kFusedMaxChunks); }
+
+// contiguous split: first tile of CTA c's range = floor(t_all * c / n_used), in 32-bit arithmetic
+// (t_all = cut_base * n_used + cut_rem, cut_rem * c < 2^20)
+__device__ __forceinline__ int cut_at(const FusedPlan* pl, int c) {
+    return pl->cut_base * c + (int)((unsigned)(pl->cut_rem * c) / (unsigned)pl->n_used);
+}
+
+__device__ __forceinline__ void cursor_init(const FusedPlan* pl, Cursor& c) { c.k = 0; c.r = pl->r0; c.h = pl->h0; }
+
+// The CTA's next unit (false: none left).
+__device__ __forceinline__ bool next_unit(const FusedPlan* pl, Cursor& c, int B, int Hkv, int G, Unit& un) {
+    const int cta = blockIdx.x, n_ctas = gridDim.x;
+    if (pl->mode == 0) {
+        const int u = snake_unit(c.k, cta, n_ctas);
+        if (u >= pl->total) return false;
+        int lo = 0, hi = B - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if ((int)pl->u.s.pos_base[mid] <= u) lo = mid; else hi = mid - 1;
+        }
+        const int i = pl->pos_req[lo];
+        const int t = pl->tiles[i], n = pl->n[i], nc = pl->u.s.nc[i];
+        const int rbs = (G * n + kRowBlock - 1) / kRowBlock;
+        const int local = u - (int)pl->u.s.pos_base[lo];
+        const int per = Hkv * rbs;
+        const int ch = local / per, rem = local - ch * per;
+        un.req = i; un.kvh = rem / rbs; un.rb = rem - un.kvh * rbs; un.n_nodes = n;
+        if (t < 32768 && nc < 32768) {
+            un.tile_begin = (int)((unsigned)t * (unsigned)ch / (unsigned)nc); un.tile_end = (int)((unsigned)t * (unsigned)(ch + 1) / (unsigned)nc);
+        } else {
+            un.tile_begin = (int)((long long)t * ch / nc); un.tile_end = (int)((long long)t * (ch + 1) / nc);
+        }
+        un.n_chunks = nc; un.chunk = ch;
+        un.slot_base = u - ch * per; un.slot_stride = per; un.bump = 0;
+        ++c.k;
+        return true;
+    }
+    // contiguous split: the pairs that overlap [lo, hi), one after the other
+    const int lo = pl->lo, hi = pl->hi;
+    if (c.r >= B) return false;
+    const int t = pl->tiles[c.r];
+    const int ps = pl->u.start[c.r] + c.h * t;
+    if (ps >= hi) return false;
+    auto cta_of = [&](int x) -> int {                 // the CTA whose range [cut(c), cut(c+1)) holds tile x
+        int cc = min(pl->n_used - 1, (int)((unsigned)x / (unsigned)max(1, pl->cut_base)));
+        while (cc + 1 < pl->n_used && cut_at(pl, cc + 1) <= x) ++cc;
+        while (cc > 0 && cut_at(pl, cc) > x) --cc;
+        return cc;
+    };
+    const int c0 = ps >= lo ? cta : cta_of(ps), c1 = ps + t <= hi ? cta : cta_of(ps + t - 1);
+    un.req = c.r; un.kvh = c.h; un.rb = 0; un.n_nodes = pl->n[c.r];
+    un.tile_begin = max(lo, ps) - ps; un.tile_end = min(hi, ps + t) - ps;
+    un.n_chunks = c1 - c0 + 1; un.chunk = cta - c0;
+    un.slot_base = 2 * c0; un.slot_stride = 2; un.bump = 1;
+    ++c.k;
+    if (++c.h == Hkv) {
+        c.h = 0;
+        do { ++c.r; } while (c.r < B && (pl->n[c.r] == 0 || pl->tiles[c.r] <= 0));
+    }
+    return true;
+}
+
+// Executed by all kFusedThreads threads of the CTA (it contains block barriers).  The code below runs once per CTA
+// and launch, straight from a cold instruction cache, so its cost is its length: it reads only the two numbers per
+// request the plan depends on (the parent arrays are checked by the warps that use them, unit by unit), keeps to
+// 32-bit arithmetic and rolled loops, and has two block barriers on the contiguous path and five on the other.
+__device__ __noinline__ static void make(const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ num_nodes,
+                                        int B, int N, int Hkv, int G, int page_size, int max_pages,
+                                        FusedPlanScratch* sc, FusedPlan* pl, int* status_word) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_ctas = gridDim.x, cta = blockIdx.x;
+    if (tid < kFusedMaxB) {
+        int n = 0, tiles = 0;
+        if (tid < B) {
+            n = num_nodes[tid];
+            const int pfx = prefix_len[tid];
+            if (n < 0 || n > N || pfx < 0) { war_set_device_status(status_word, WAR_ERR_BAD_TREE); n = 0; }
+            if (n > 0) {
+                const long long L = (long long)pfx + n;
+                if (L > (long long)max_pages * page_size) { war_set_device_status(status_word, WAR_ERR_BAD_PAGE); n = 0; }
+                else tiles = (int)((L + kTileKeys - 1) >> 7);
+            }
+        }
+        pl->tiles[tid] = tiles;
+        pl->n[tid] = (uint8_t)n;
+        sc->weight[tid] = n > 0 && tiles > 0 ? Hkv * ((G * n + kRowBlock - 1) / kRowBlock) : 0;
+    }
+    __syncthreads();
+
+    // ---- the same choice as attn_plan_kernel makes for up to 64 requests (every warp for itself) ----
+    int n_mx = 0, prs = 0, t_mx = 0, t_sm = 0;
+    long long w_sm = 0;
+    for (int q = lane; q < B; q += 32) {
+        const int w = sc->weight[q], t = pl->tiles[q];
+        if (w > 0) { n_mx = max(n_mx, (int)pl->n[q]); prs += Hkv; t_mx = max(t_mx, t); t_sm += t; w_sm += (long long)t * w; }
+    }
+    const int rows_max = G * __reduce_max_sync(0xffffffffu, n_mx);
+    const int pairs = __reduce_add_sync(0xffffffffu, prs);
+    const int t_max = __reduce_max_sync(0xffffffffu, t_mx);
+    const int t_sum = __reduce_add_sync(0xffffffffu, t_sm);
+    // all tiles, weighted by kv heads and row blocks (the sum of the lanes' numbers in two 32-bit pieces)
+    const long long tot = ((long long)__reduce_add_sync(0xffffffffu, (unsigned)(w_sm >> 24)) << 24) +
+                          (long long)__reduce_add_sync(0xffffffffu, (unsigned)(w_sm & 0xffffff));
+    const long long t_all_ll = (long long)t_sum * Hkv;
+    const bool contiguous = contiguous_split_pays(rows_max, t_all_ll, n_ctas);
+
+    if (contiguous) {
+        // The tiles of all (request, kv head) pairs form one sequence; CTA c takes [cut(c), cut(c+1)), cut(c) = t_all * c / n_used.
+        if (warp == 0) {
+            const int a0 = 2 * lane, a1 = 2 * lane + 1;
+            const int m0 = sc->weight[a0] > 0 ? pl->tiles[a0] * Hkv : 0, m1 = sc->weight[a1] > 0 ? pl->tiles[a1] * Hkv : 0;
+            int incl = m0 + m1;
+#pragma unroll 1
+            for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+            pl->u.start[a0] = incl - m0 - m1;
+            pl->u.start[a1] = incl - m1;
+            if (lane == 31) pl->u.start[64] = incl;
+            __syncwarp();
+            const int t_all = __shfl_sync(0xffffffffu, incl, 31);
+            const int n_used = min(n_ctas, max(1, t_all / 4));
+            if (lane == 0) {
+                pl->mode = 1; pl->total = 0; pl->t_all = t_all; pl->n_used = n_used;
+                pl->cut_base = (int)((unsigned)t_all / (unsigned)n_used); pl->cut_rem = t_all - pl->cut_base * n_used;
+            }
+            __syncwarp();
+            // this CTA's range and the pair that holds its first tile (lanes look at requests lane and lane + 32)
+            int lo = 0, hi = 0;
+            if (cta < n_used) { lo = cut_at(pl, cta); hi = cut_at(pl, cta + 1); }
+            int best = -1;
+            for (int q = lane; q < B; q += 32)
+                if (sc->weight[q] > 0 && pl->u.start[q] <= lo) best = max(best, q);
+            best = __reduce_max_sync(0xffffffffu, best);
+            if (lane == 0) {
+                pl->lo = lo; pl->hi = hi;
+                if (hi > lo && best >= 0) { pl->r0 = best; pl->h0 = (int)((unsigned)(lo - pl->u.start[best]) / (unsigned)pl->tiles[best]); }
+                else { pl->r0 = B; pl->h0 = 0; }
+            }
+        }
+        __syncthreads();
+        return;
+    }
+
+    // ---- searched chunk length (see chunk_search), never more than kFusedMaxChunks chunks per request ----
+    long long ct = (tot + kTargetUnits - 1) / kTargetUnits;
+    if (ct < kMinChunkTiles) ct = kMinChunkTiles;
+    const int chunk_tiles = (int)ct;
+    const int best_c = chunk_search<kFusedThreads>(pl->tiles, sc->weight, B, max(chunk_floor(t_max), chunk_tiles), t_max, n_ctas, sc->keys);
+    const int c_best = best_c;
+    // ---- longest-first order, units per request, their offsets ----
+    if (tid < B) {
+        const int t = pl->tiles[tid];
+        int pos = 0;
+        for (int q = 0; q < B; ++q) {
+            const int tq = pl->tiles[q];
+            pos += (tq > t) || (tq == t && q < tid);
+        }
+        const int nc = t > 0 ? ceil_div_small(t, c_best) : 0;
+        pl->u.s.nc[tid] = (uint16_t)nc;
+        pl->pos_req[pos] = (uint8_t)tid;
+        sc->units_by_pos[pos] = nc * sc->weight[tid];
+    }
+    __syncthreads();
+    if (warp == 0) {                                             // exclusive scan over the sorted positions, two per lane
+        const int a0 = 2 * lane, a1 = 2 * lane + 1;
+        const int m0 = a0 < B ? sc->units_by_pos[a0] : 0, m1 = a1 < B ? sc->units_by_pos[a1] : 0;
+        int incl = m0 + m1;
+#pragma unroll 1
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+        pl->u.s.pos_base[a0] = (uint16_t)(incl - m0 - m1);
+        pl->u.s.pos_base[a1] = (uint16_t)(incl - m1);
+        if (lane == 31) { pl->mode = 0; pl->total = incl; pl->r0 = 0; pl->h0 = 0; pl->lo = 0; pl->hi = 0; pl->t_all = 0; pl->n_used = 0; }
+    }
+    __syncthreads();
+}
+
+}  // namespace fused_plan
+#endif

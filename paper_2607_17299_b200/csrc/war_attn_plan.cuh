@@ -14,7 +14,7 @@
 
 constexpr int kTileKeys = 128;          // planning granularity in keys
 constexpr int kRowBlock = 128;          // query rows per unit
-constexpr int kTargetUnits = 148 * 8;   // aim: several units per SM
+constexpr int kTargetUnits = 148 * 8;   // aim: several units per SM of a B200 (a tuning constant of the plan, not a launch size)
 constexpr int kMinChunkTiles = 8;       // never cut finer than 1024 keys
 constexpr int kMaxPlanB = 4096;
 
@@ -34,6 +34,8 @@ struct AttnWorkspace {
     int* pair_unit0;     // [B, Hkv]             contiguous split: unit of the first chunk of (request, kv head),
     int* pair_cta0;      // [B, Hkv]             the CTA that runs it (chunk c > 0 is the first unit of CTA cta0 + c)
     int* pair_chunks;    // [B, Hkv]             and the number of chunks
+    unsigned long long* pair_count;   // [B, Hkv, row_blocks]  one-launch path: (call number << 16) | units of a split
+                                      // triple that have left their partial result
     AttnReq* req;        // [B]
     uint64_t* anc;       // [B, N] bit a of anc[b, j]: slot a is j or an ancestor of j
     AttnUnit* units;     // [max_units]
@@ -59,7 +61,7 @@ inline AttnWorkspace war_attn_workspace_layout(const war_attn_params_t* p, void*
     AttnWorkspace w;
     const int G = p->Hq / p->Hkv;
     const int R = G * p->N;
-    w.rows = R < kRowBlock ? R : kRowBlock;
+    w.rows = ((R < kRowBlock ? R : kRowBlock) + 1) & ~1;        // even: a unit's (max, sum) block starts on a 16-byte boundary
     w.row_blocks = (R + kRowBlock - 1) / kRowBlock;
     w.max_units = kTargetUnits + p->B * p->Hkv * w.row_blocks;
     auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
@@ -70,6 +72,7 @@ inline AttnWorkspace war_attn_workspace_layout(const war_attn_params_t* p, void*
     w.pair_unit0 = (int*)(b + at); at += align(sizeof(int) * (size_t)p->B * p->Hkv);
     w.pair_cta0 = (int*)(b + at); at += align(sizeof(int) * (size_t)p->B * p->Hkv);
     w.pair_chunks = (int*)(b + at); at += align(sizeof(int) * (size_t)p->B * p->Hkv);
+    w.pair_count = (unsigned long long*)(b + at); at += align(sizeof(unsigned long long) * (size_t)p->B * p->Hkv * w.row_blocks);
     w.req = (AttnReq*)(b + at); at += align(sizeof(AttnReq) * (size_t)p->B);
     w.anc = (uint64_t*)(b + at); at += align(sizeof(uint64_t) * (size_t)p->B * p->N);
     w.units = (AttnUnit*)(b + at); at += align(sizeof(AttnUnit) * (size_t)w.max_units);
@@ -83,6 +86,9 @@ inline AttnWorkspace war_attn_workspace_layout(const war_attn_params_t* p, void*
 war_status_t war_attn_launch_simple(const void* q, const void* k, const void* v, const int32_t* page_table,
                                     const int32_t* prefix_len, const war_attn_params_t* p, const AttnWorkspace& w,
                                     void* out, float* lse, int* status_word, cudaStream_t s);
+// fused: the kernel plans for itself and merges split units itself (one launch, see war_attn_fused_plan.cuh)
 war_status_t war_attn_launch_sm100(const void* q, const void* k, const void* v, const int32_t* page_table,
-                                   const int32_t* prefix_len, const war_attn_params_t* p, const AttnWorkspace& w,
+                                   const int32_t* prefix_len, const int32_t* num_nodes, const int32_t* parent,
+                                   const war_attn_params_t* p, const AttnWorkspace& w, bool fused,
                                    void* out, float* lse, int* status_word, cudaStream_t s);
+int war_attn_sm_count();                 // SMs of the current device (0 on error)

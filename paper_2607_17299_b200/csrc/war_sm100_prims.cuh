@@ -59,6 +59,12 @@ __device__ __forceinline__ void tma_load_block(uint32_t dst, const CUtensorMap* 
         ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(block) : "memory");
 }
 
+// plain (untiled) bulk copy global -> shared: both addresses 16-byte aligned, size a multiple of 16 bytes
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
 // token-major pools: tensor (d, token, head, page); one copy brings 64 dims of every token of one (page, head)
 __device__ __forceinline__ void tma_load_half_page(uint32_t dst, const CUtensorMap* map, int d0, int head, int page, uint64_t* bar) {
     asm volatile(

@@ -4,6 +4,7 @@
 #include <math_constants.h>
 #include "war_common.cuh"
 #include "war_attn_plan.cuh"
+#include "war_attn_fused_plan.cuh"
 
 namespace {
 
@@ -202,12 +203,8 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     // The tiles of all (request, kv head) pairs, request after request and head after head, form one sequence of
     // T_all tiles; CTA c takes the range [c * T_all / n_used, (c + 1) * T_all / n_used).  A pair that crosses a cut is
     // split there: its first chunk is somewhere in a CTA's list, every further chunk is the first unit of the next CTA.
-    // Every CTA streams the same number of tiles (within one) whatever the requests' lengths are.  It pays where the
-    // tile count per CTA decides the time and pairs have to be cut anyway: more than 64 live rows per kv head (below
-    // that the call is bound by DRAM alone, which does not care which CTA streams what), at least 64 tiles per CTA and
-    // pairs of 128 tiles (16 K tokens) or more on average, none longer than twice the average; measured on 4-64 requests
-    // of three recipes, +2 to +8 % there and a loss elsewhere (short pairs are better left whole, short ranges pay for
-    // the extra unit per CTA, one very long request among short ones is better served by the search below).
+    // Every CTA streams the same number of tiles (within one) whatever the requests' lengths are.  When it pays:
+    // fused_plan::contiguous_split_pays (the one-launch path takes the same decision in every CTA).
     if (B <= 64 && n_ctas <= kMaxPlanCtas) {
         // every warp works the rule out for itself (two requests per lane): no barrier on the way of the calls that do not use it
         int n_mx = 0, prs = 0, t_mx = 0, t_sm = 0;
@@ -221,7 +218,8 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         const int t_max = __reduce_max_sync(0xffffffffu, t_mx);
         const int t_sum = __reduce_add_sync(0xffffffffu, t_sm);               // < 2^31: at most 64 requests of < 2^24 tiles
         const long long t_all = (long long)t_sum * Hkv;
-        if (rows_max > 64 && rows_max <= kRowBlock && t_all >= 64ll * n_ctas && t_all < (1ll << 31) && t_all >= 128ll * pairs && (long long)t_max * pairs <= 2 * t_all) {
+        (void)pairs; (void)t_max;
+        if (fused_plan::contiguous_split_pays(rows_max, t_all, n_ctas)) {
             __shared__ int s_start[65];
             plan_contiguous(s_tiles, s_n, s_start, s_units, s_units + kMaxPlanCtas + 8, B, Hkv, n_ctas, w);   // (the snake deal's s_units is free here)
             return;
@@ -262,42 +260,26 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
     // Little work (few requests): the default chunk (about kTargetUnits units) would cut every request into short
     // units, and a unit costs about six tiles on top of its own (pipeline fill, Q load, partials written and merged;
     // calibrated on 2 to 32 requests).
-    // Up to 64 requests, one warp therefore looks for the chunk length c that minimises the estimated time in tiles
+    // Up to 64 requests, the block therefore looks for the chunk length c that minimises the estimated time in tiles
     //     ceil(units(c) / CTAs) * (c + 6),     units(c) = sum over (request, kv head, row block) of ceil(tiles / c),
-    // over c from the default up to the longest request: a coarse grid of 32 lengths (a lane each, every lane walks
-    // the requests), then finer grids around the best.  This covers "one unit per CTA" (units(c) <= CTAs: one pipeline
-    // fill and one epilogue per CTA) as well as a few long units per CTA, and with a dozen requests of very different
-    // lengths it avoids leaving most CTAs idle while the longest request finishes.  Equal estimates take the longer
+    // over c from the default up to the longest request (fused_plan::chunk_search, the routine the one-launch path
+    // runs in every CTA, so both paths cut the requests the same way).  This covers "one unit per CTA" (units(c) <=
+    // CTAs: one pipeline fill and one epilogue per CTA) as well as a few long units per CTA, and with a dozen requests
+    // of very different lengths it avoids leaving most CTAs idle while the longest request finishes.  Equal estimates take the longer
     // chunk (fewer partials).  More requests (only with very few kv heads can that be little work): shares of the grid
     // in proportion to the tiles, rounded down, if that fits the grid and its longest unit beats the default plan.
     const long long tot_all = s_tot;
     if (B <= kSearchMaxB) {
-        if (warp == 0) {
-            int t_mine = 0;
-            for (int q = lane; q < B; q += 32) if (s_n[q] > 0) t_mine = max(t_mine, s_tiles[q]);
-            const int t_max = __reduce_max_sync(0xffffffffu, t_mine);
-            int c_lo = max(4, chunk_tiles), c_hi = max(t_max, c_lo), best_c = c_lo;
-            while (true) {
-                const int step = max(1, (c_hi - c_lo + 31) / 32);
-                const int cl = min(c_lo + lane * step, c_hi);
-                long long units = 0;
-                for (int q = 0; q < B; ++q) {
-                    const int n = s_n[q], t = s_tiles[q];
-                    if (n > 0 && t > 0) units += (long long)Hkv * ((G * n + kRowBlock - 1) / kRowBlock) * ((t + cl - 1) / cl);
-                }
-                const long long est = ((units + n_ctas - 1) / n_ctas) * (cl + 6);
-                // smallest estimate, then the longest chunk: est < 2^40, cl < 2^20
-                const long long key = (est << 20) | (long long)((1 << 20) - 1 - cl);
-                long long kmin = key;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
-                best_c = (1 << 20) - 1 - (int)(kmin & ((1 << 20) - 1));
-                if (step == 1) break;
-                c_lo = max(c_lo, best_c - step + 1);
-                c_hi = min(c_hi, best_c + step - 1);
-            }
-            if (lane == 0) s_cstar = best_c;
-        }
+        __shared__ int s_keys[64];
+        __shared__ int s_weight[kSearchMaxB];
+        int t_mine = 0;
+        for (int q = lane; q < B; q += 32) if (s_n[q] > 0) t_mine = max(t_mine, s_tiles[q]);
+        const int t_max = __reduce_max_sync(0xffffffffu, t_mine);
+        if (tid < kSearchMaxB) s_weight[tid] = tid < B && s_n[tid] > 0 && s_tiles[tid] > 0 ? Hkv * ((G * s_n[tid] + kRowBlock - 1) / kRowBlock) : 0;
+        if (tid >= B && tid < kSearchMaxB) s_tiles[tid] = 0;
+        __syncthreads();
+        const int best_c = fused_plan::chunk_search<kFusedThreads>(s_tiles, s_weight, B, max(fused_plan::chunk_floor(t_max), chunk_tiles), t_max, n_ctas, s_keys);
+        if (tid == 0) s_cstar = best_c;
         __syncthreads();
     }
     const int c_best = s_cstar;
@@ -601,12 +583,13 @@ attn_simple_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
 war_status_t check_params(const war_attn_params_t* p) {
     if (!p) return WAR_ERR_INVALID_ARG;
     if (p->B < 0 || p->N < 1 || p->N > 64 || p->Hq < 1 || p->Hkv < 1 || p->Hq % p->Hkv != 0 || p->max_pages_per_req < 0 ||
-        p->num_pages < 0 || p->kernel < 0 || p->kernel > 1 || !(p->scale > 0.f))
+        p->num_pages < 0 || p->kernel < 0 || p->kernel > 2 || !(p->scale > 0.f))
         return WAR_ERR_INVALID_ARG;
     // a 128-key tile is a whole number of pages, and a page is a whole number of 8-token groups of the tile layout
     if (p->D != 128 || (p->page_size != 8 && p->page_size != 16 && p->page_size != 32 && p->page_size != 64 && p->page_size != 128))
         return WAR_ERR_UNSUPPORTED;
     if ((p->Hq / p->Hkv) * p->N > 512 || p->B > kMaxPlanB) return WAR_ERR_UNSUPPORTED;
+    if ((long long)p->max_pages_per_req * p->page_size >= (1ll << 30)) return WAR_ERR_UNSUPPORTED;    // contexts below 2^30 tokens
     const int layout = war_attn_pool_layout(p->k_strides, p);                 // both pools in the same one of the two layouts
     if (layout < 0 || war_attn_pool_layout(p->v_strides, p) != layout) return WAR_ERR_UNSUPPORTED;
     return WAR_OK;
@@ -618,7 +601,9 @@ war_status_t war_attn_launch_simple(const void* q, const void* k, const void* v,
                                     const int32_t* prefix_len, const war_attn_params_t* p, const AttnWorkspace& w,
                                     void* out, float* lse, int* status_word, cudaStream_t s) {
     const int G = p->Hq / p->Hkv;
-    attn_simple_kernel<<<148 * 4, 128, 0, s>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, page_table,
+    const int n_sm = war_attn_sm_count();
+    if (n_sm <= 0) return WAR_ERR_CUDA;
+    attn_simple_kernel<<<n_sm * 4, 128, 0, s>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, page_table,
                                               prefix_len, p->N, p->Hq, p->Hkv, G, p->page_size, p->max_pages_per_req,
                                               (long long)p->k_strides[0], (long long)p->k_strides[1], (long long)p->k_strides[2],
                                               (long long)p->num_pages, p->scale * kLog2e, w, (__nv_bfloat16*)out, lse, status_word);
@@ -648,18 +633,22 @@ extern "C" war_status_t war_verify_attn(const void* d_q, const void* d_kpool, co
     if (!status_word) return WAR_ERR_CUDA;
     const AttnWorkspace w = war_attn_workspace_layout(p, d_workspace);
     const int G = p->Hq / p->Hkv;
-    static int sm_count[64] = {0};
-    int dev = 0;
-    WAR_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return WAR_ERR_UNSUPPORTED;
-    if (!sm_count[dev]) WAR_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+    const int n_sm = war_attn_sm_count();
+    if (n_sm <= 0) return WAR_ERR_CUDA;
+    // Few requests (the low-load regime the step exists for): one launch.  Every CTA of the attention kernel plans
+    // for itself and the last CTA to finish a split unit's triple merges it, so the planning and combine launches
+    // and the gaps around them disappear.
+    if (p->kernel == 0 && war_attn_fused_ok(p, w.row_blocks, n_sm))
+        return war_attn_launch_sm100(d_q, d_kpool, d_vpool, d_page_table, d_prefix_len, d_num_nodes, d_parent, p, w, true, d_out,
+                                     d_lse, status_word, stream);
     attn_plan_kernel<<<1, 1024, 0, stream>>>(d_prefix_len, d_num_nodes, d_parent, p->B, p->N, p->Hkv, G, p->page_size,
-                                            p->max_pages_per_req, sm_count[dev], w, status_word);
+                                            p->max_pages_per_req, n_sm, w, status_word);
     WAR_LAUNCH_CHECK();
     if (p->kernel == 1)
         st = war_attn_launch_simple(d_q, d_kpool, d_vpool, d_page_table, d_prefix_len, p, w, d_out, d_lse, status_word, stream);
     else
-        st = war_attn_launch_sm100(d_q, d_kpool, d_vpool, d_page_table, d_prefix_len, p, w, d_out, d_lse, status_word, stream);
+        st = war_attn_launch_sm100(d_q, d_kpool, d_vpool, d_page_table, d_prefix_len, d_num_nodes, d_parent, p, w, false, d_out,
+                                   d_lse, status_word, stream);
     if (st != WAR_OK) return st;
     attn_combine_kernel<<<dim3(p->B * p->Hkv, (G * p->N + kCombineWarps - 1) / kCombineWarps), kCombineWarps * 32, 0, stream>>>(
         w, p->N, p->Hq, p->Hkv, G, (__nv_bfloat16*)d_out, d_lse);

@@ -51,9 +51,10 @@ extern "C" war_status_t war_verify_attn_noalloc(const void* d_q, const void* d_k
     void* scratch = nullptr;
     const war_status_t st = scratch_for_current_device(&scratch);
     if (st != WAR_OK) return st;
-    // Nothing in the scratch has to start at zero: the planning kernel of every call rewrites the counters, the
-    // per-request records and the work list before anything reads them, and partial results are only read for
-    // units written earlier in the same call.
+    // Nothing in the scratch has to start at zero.  On the one-launch path the arrival counters of split units carry
+    // the number of the call that wrote them, so what an earlier call left reads as "nothing yet"; on the three-launch
+    // path the planning kernel writes counters, per-request records and the work list before anything reads them.
+    // Partial results are only read for units written earlier in the same call.
     return war_verify_attn(d_q, d_kpool, d_vpool, d_page_table, d_prefix_len, d_num_nodes, d_parent, params, scratch,
                            d_out, d_lse, stream);
 }

@@ -16,7 +16,7 @@ from tests import gpu_util as U
 
 pytestmark = pytest.mark.gpu
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
-KERNELS = [0, 1]
+KERNELS = [0, 1, 2]          # 0 default (one launch for up to 64 requests), 1 plain CUDA-core kernel, 2 tensor-core kernel with separate plan / combine launches
 
 
 @pytest.fixture(scope="module")
@@ -280,6 +280,41 @@ def test_random_shapes_against_the_checker(war, seed):
         assert torch.equal(raw1, raw2)
 
 
+@pytest.mark.parametrize("kernel", [0, 2])
+def test_workspace_contents_do_not_matter(war, kernel):
+    """The workspace is scratch: whatever it holds before the call (zeros, ones, a pattern, another call's leftovers,
+    noise), the results are the same bits.  On the one-launch path this is what the call numbers in the arrival
+    counters of split requests are for; the contexts are long enough that every request is split."""
+    rng = np.random.default_rng(77)
+    cfg = W.scaled(W.CONFIGS["low"], B=5, N=12)
+    ctx = np.array([9000, 14000, 700, 20000, 4100])
+    a = W.make_attention_inputs(cfg, ctx, device=U.dev())
+    nn, parent = _random_trees(rng, cfg.B, cfg.N)
+    d_nn, d_par = torch.from_numpy(nn).to(U.dev()), torch.from_numpy(parent).to(U.dev())
+    params = war.attn_params(a.q, a.k_pool, a.v_pool, a.page_table, 0.088, kernel)
+    n_bytes = war.war_verify_attn_workspace_bytes(params)
+    outs = []
+    fills = [lambda n: torch.zeros(n, dtype=torch.uint8, device=U.dev()),
+             lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device=U.dev()),
+             lambda n: torch.full((n,), 0xA5, dtype=torch.uint8, device=U.dev()),
+             lambda n: torch.randint(0, 256, (n,), dtype=torch.uint8, device=U.dev())]
+    for fill in fills:
+        ws = fill(n_bytes)
+        for _ in range(2):                                                    # the second call finds the first one's leftovers
+            out = torch.full(a.q.shape, 7.0, dtype=torch.bfloat16, device=U.dev())
+            lse = torch.full(a.q.shape[:3], 7.0, dtype=torch.float32, device=U.dev())
+            war.war_verify_attn(a.q, a.k_pool, a.v_pool, a.page_table, a.prefix_len, d_nn, d_par, params, ws, out, lse)
+            torch.cuda.synchronize()
+            outs.append((out, lse))
+    for out, lse in outs[1:]:
+        assert torch.equal(out, outs[0][0]) and torch.equal(lse, outs[0][1])
+    assert war.war_device_status() == 0
+    want = A.verify_attention(a.q, a.k_pool, a.v_pool, a.page_table.cpu().numpy(), a.prefix_len.cpu().numpy(), nn, parent, 0.088)
+    got, got_lse = outs[0][0].float().cpu().numpy(), outs[0][1].cpu().numpy()
+    for i in range(cfg.B):
+        U.assert_attention_close(got[i], got_lse[i], want[i][0], want[i][1], int(nn[i]))
+
+
 @pytest.mark.parametrize("seed", range(12))
 def test_mid_size_batches_through_every_plan(war, seed):
     """2-64 requests of four length mixes (long and uniform: the contiguous split when the trees have more than 64
@@ -308,7 +343,11 @@ def test_mid_size_batches_through_every_plan(war, seed):
         for j in range(1, nn[i]):
             par[i, j] = int(rng.integers(0, j))
     scale = 1.0 / np.sqrt(cfg.D)
-    got, got_lse, _ = U.run_attn(war, a, nn, par, scale, 0)
+    got, got_lse, raw = U.run_attn(war, a, nn, par, scale, 0)
+    # the one-launch path (every CTA plans for itself, the last CTA of a split unit merges) takes the same decisions as
+    # the three-launch path and adds the partials in the same order: the bits are the same
+    got3, got3_lse, raw3 = U.run_attn(war, a, nn, par, scale, 2)
+    assert torch.equal(raw, raw3) and (got_lse == got3_lse).all()
     sample = sorted({0, B - 1, int(np.argmax(ctx)), int(rng.integers(0, B))})
     want = A.verify_attention(a.q, a.k_pool, a.v_pool, a.page_table.cpu().numpy(), a.prefix_len.cpu().numpy(), nn, par, scale,
                               requests=sample)

@@ -45,10 +45,11 @@ def _both(war, cfg, ctx, seed):
     lse = torch.full(a.q.shape[:3], 3.0, dtype=torch.float32, device=dev)
     war.war_verify_attn_noalloc(a.q, a.k_pool, a.v_pool, a.page_table, a.prefix_len, d_nn, d_par, params, out, lse)
     torch.cuda.synchronize()
-    np.testing.assert_allclose(out.float().cpu().numpy(), ref_out.float().cpu().numpy(), atol=1e-2, rtol=1e-2)
-    np.testing.assert_allclose(lse.cpu().numpy(), ref_lse.cpu().numpy(), atol=1e-3, rtol=1e-4)
+    # the two entry points run the same kernels on the same plan: the same bits, not merely close ones
+    assert torch.equal(out, ref_out) and torch.equal(lse, ref_lse)
     assert (ref_out.float() != 3.0).any()
     assert war.war_device_status() == 0
+    return a, nn, parent, scale, out, lse
 
 
 def test_matches_the_workspace_entry_point_on_two_calls_in_a_row(war):
@@ -58,6 +59,18 @@ def test_matches_the_workspace_entry_point_on_two_calls_in_a_row(war):
     cfg2 = W.scaled(W.CONFIGS["tiny"], B=3, N=8, page_size=32)
     _both(war, cfg2, np.array([700, 5000, 64]), seed=2)
     _both(war, cfg1, np.array([100, 200, 300, 400, 500, 4000]), seed=3)
+
+
+def test_matches_the_cpu_checker(war):
+    """The allocation-free entry point against the fp64 checker itself (not only against the other entry point)."""
+    from oracle import attention_oracle as A
+    from tests import gpu_util as U
+    cfg = W.scaled(W.CONFIGS["tiny"], B=4, N=16)
+    a, nn, parent, scale, out, lse = _both(war, cfg, np.array([3000, 129, 4096, 640]), seed=4)
+    want = A.verify_attention(a.q, a.k_pool, a.v_pool, a.page_table.cpu().numpy(), a.prefix_len.cpu().numpy(), nn, parent, scale)
+    got, got_lse = out.float().cpu().numpy(), lse.cpu().numpy()
+    for i in range(cfg.B):
+        U.assert_attention_close(got[i], got_lse[i], want[i][0], want[i][1], int(nn[i]))
 
 
 def test_refuses_shapes_beyond_the_fixed_scratch(war):
