@@ -1,7 +1,7 @@
 /*
  * war.h -- C ABI of the batched SuffixDecoding speculate-and-verify step for one B200 (sm_100a).
  *
- * The paper (WAR: Workload-Aware Rollouts, Section 3 overview and Section 3.2 "SuffixDecoding") speeds up
+ * The paper (WAR: Workload-Aware Rollouts, Section 3 overview and Section 3.3 "SuffixDecoding") speeds up
  * low-load agentic RL rollouts with model-free speculative decoding: a cache of previously generated
  * trajectories is matched against each live request's current token pattern to produce draft tokens, the
  * target model verifies all drafts in one forward pass, and the request advances by every accepted token.
@@ -59,9 +59,8 @@ typedef struct CUstream_st* war_stream_t;      /* same type as cudaStream_t */
 typedef struct war_index war_index_t;          /* opaque; lives on the device that was current at build */
 
 /* ------------------------------------------------------------------------------------------------
- * Trajectory cache (paper Section 3.2: SuffixDecoding "caches token-sequence patterns from previously
- * generated trajectories"; the "external update interface" adds newly generated trajectories after each
- * RL step).  Trajectory t is d_tokens[h_offsets[t] .. h_offsets[t+1]); token ids must lie in [0, vocab)
+ * Trajectory cache (paper Section 3.3: SuffixDecoding keeps the token patterns of the trajectories generated so
+ * far; an update interface outside the decode loop adds the new trajectories after each RL step).  Trajectory t is d_tokens[h_offsets[t] .. h_offsets[t+1]); token ids must lie in [0, vocab)
  * (checked on the device: WAR_ERR_INVALID_ARG, nothing added).
  * Inside the index the trajectories are joined with one unique negative separator each, so no match ever
  * straddles two trajectories.  The suffix array is ordered to depth max_depth (>= P + N of every later
@@ -71,8 +70,8 @@ typedef struct war_index war_index_t;          /* opaque; lives on the device th
  * war_index_append leaves the index answering every query exactly as a fresh build over the old
  * trajectories followed by the new ones would.  Exceeding the capacity returns WAR_ERR_CAPACITY and
  * leaves the index unchanged.  Both calls synchronise `stream` before returning.
- * Updating without blocking the drafts (the paper updates the cache "asynchronously" so that it does not block
- * the pipeline, Section 3.2): the index keeps two sets of (suffix array, LCP, buckets).  war_index_append builds
+ * Updating without blocking the drafts (the paper updates the cache asynchronously so that it does not block
+ * the pipeline, Section 3.3): the index keeps two sets of (suffix array, LCP, buckets).  war_index_append builds
  * the new set beside the published one and publishes it just before it returns; the corpus is only written
  * behind what the published set refers to.  So ONE thread may run war_index_append (on its own stream) while other
  * threads keep calling war_draft on other streams: a war_draft call uses the set that is published at the moment
@@ -86,7 +85,7 @@ war_status_t war_index_build(const int32_t* d_tokens, const int64_t* h_offsets, 
 war_status_t war_index_append(war_index_t* ix, const int32_t* d_tokens, const int64_t* h_offsets, int32_t T,
                               war_stream_t stream);
 
-/* Windowed cache (the paper keeps the cache's "memory overhead" modest, Section 3.2, without naming a policy; this
+/* Windowed cache (the paper keeps the cache's memory overhead modest, Section 3.3, without naming a policy; this
  * is the simplest one): removes the n_oldest trajectories that were added first.  Afterwards every query answers
  * exactly as a fresh build on the remaining trajectories would.  The suffix array is filtered, not sorted again
  * (the remaining suffixes keep their order); LCP and buckets are recomputed.  Synchronises `stream`; allocates
@@ -121,8 +120,8 @@ war_status_t war_index_info(const war_index_t* ix, war_index_info_t* out);
 war_status_t war_index_destroy(war_index_t* ix);
 
 /* ------------------------------------------------------------------------------------------------
- * Draft (paper Section 3: SuffixDecoding "matches the current token pattern against [the historical
- * trajectories] to generate draft tokens").  For each of B requests:
+ * Draft (paper Section 3: SuffixDecoding drafts by matching the request's current tokens against the stored
+ * trajectories).  For each of B requests:
  *   match   the largest l <= min(P, tail_len) such that the last l tokens of the tail occur contiguously
  *           inside one stored trajectory (0 if none);
  *   tree    slot 0 = the last tail token, count[0] = occurrences of the matched string.  Every further slot
@@ -135,15 +134,15 @@ war_status_t war_index_destroy(war_index_t* ix);
  * entries are read.  Tail tokens outside [0, vocab) never match.
  * Outputs: d_match_len [B], d_num_nodes [B], d_ids / d_parent / d_count [B, N] (d_count may be NULL).
  * Unused slots are written as ids = -1, parent = -1, count = 0.
- * Workload-aware switch (paper Section 3.2, "adaptive enabling and disabling" of speculation "according to the
- * current batch size", with "stateless mode switching"; Section 5.3: beyond a batch of about 16 speculation
+ * Workload-aware switch (paper Section 3.3: speculation is enabled and disabled according to the
+ * current batch size, and switching between the modes carries no state; Section 5.3: beyond a batch of about 16 speculation
  * costs more than it gains).  A request with tail_len[b] < 0 is not running: num_nodes = 0, match_len = 0.  The
  * effective batch size is the number of running requests, counted on the device in this call.  When
  * spec_batch_limit > 0 and the effective batch size exceeds it, nothing is looked up and every running request
  * gets the root alone (num_nodes = 1, match_len = 0, count = 0), so the step that follows is a plain decode step
  * through the same calls: no state is kept between calls and one captured CUDA graph serves both modes.
  * spec_batch_limit = 0 always speculates.
- * Two thresholds of the SuffixDecoding method the paper builds on (Section 3.2 takes that method's code base; the
+ * Two thresholds of the SuffixDecoding method the paper builds on (Section 3.3 takes that method's code base; the
  * paper itself names neither), both exact integer rules, both off when their numerator is 0:
  *   spec_factor_num / spec_factor_den   the tree has at most 1 + floor(match_len * num / den) slots, so a longer
  *                                       match earns a larger tree (den >= 1)
@@ -162,7 +161,7 @@ war_status_t war_draft(const war_index_t* ix, const int32_t* d_tail, const int32
                        int32_t* d_match_len, int32_t* d_num_nodes,
                        int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream);
 
-/* Drafting from the best-scoring of several suffix lengths (a variant of the SuffixDecoding method that Section 3.2
+/* Drafting from the best-scoring of several suffix lengths (a variant of the SuffixDecoding method that Section 3.3
  * adopts; the paper does not spell it out).  Candidates are the suffix lengths match_len, match_len - 1, ...,
  * n_lengths of them (1 <= n_lengths <= 32), never below max(1, min_match); every shorter suffix of an occurring
  * string occurs too, usually more often.  Each candidate gets its own tree by the rules of war_draft (its own root
@@ -184,7 +183,7 @@ war_status_t war_draft_scored(const war_index_t* ix, const int32_t* d_tail, cons
                               int32_t* d_match_len, int32_t* d_used_len, int32_t* d_num_nodes,
                               int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream);
 
-/* Drafting from each request's own context (a part of the SuffixDecoding method that Section 3.2 adopts; the paper
+/* Drafting from each request's own context (a part of the SuffixDecoding method that Section 3.3 adopts; the paper
  * does not spell it out): text a rollout has produced or read once tends to come back inside the same trajectory.
  * d_ctx holds the contexts of all requests back to back (int32 token ids), d_ctx_off [B+1] (int64, DEVICE memory)
  * their bounds: request b owns c = d_ctx[d_ctx_off[b] .. d_ctx_off[b+1]), L tokens, the last one being the root of
@@ -220,8 +219,8 @@ war_status_t war_draft_pick(int32_t B, int32_t N,
                             int32_t* d_ids, int32_t* d_parent, int32_t* d_count, war_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
- * Verification attention (paper Section 3.2: the predicted tokens "are then verified by the target model"
- * in "a single forward pass"; Sections 2.3 / 5.3: this needs auxiliary attention-mask / tree-mask handling).
+ * Verification attention (paper Section 3.3: the target model then verifies the predicted tokens
+ * in one forward pass; Sections 2.3 / 5.3: this needs auxiliary attention-mask / tree-mask handling).
  * For request b, slot j < num_nodes[b], query head h (kv head h / (Hq/Hkv)):
  *     visible = { 0 .. prefix_len[b]-1 }  U  { prefix_len[b] + a : a == j or a is an ancestor of j }
  *     out[b,j,h,:] = sum_c softmax_c(scale * <q[b,j,h,:], K[c,:]>) * V[c,:]      (c over visible)
@@ -286,8 +285,8 @@ war_status_t war_verify_attn_noalloc(const void* d_q, const void* d_kpool, const
                                      war_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
- * Accept (paper Section 2.3: drafts are verified "while preserving the target output distribution";
- * Section 3.2: the rollout advances "by multiple tokens ... when the drafts are accepted").  The caller
+ * Accept (paper Section 2.3: verifying drafts leaves the target model's output distribution unchanged;
+ * Section 3.3: with accepted drafts a request advances by several tokens at once).  The caller
  * supplies the target model's own token choices; a draft slot is accepted iff every slot on its root path
  * equals the target's choice there.
  *   target_mode 0: d_target_ids[b, p] is the token the target emits AFTER slot p; slot j matches iff
@@ -301,8 +300,8 @@ war_status_t war_accept(const int32_t* d_ids, const int32_t* d_parent, const int
                         int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, war_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
- * Commit (completes the step of paper Section 3.2: the rollout advances "by multiple tokens in a single forward
- * pass when the drafts are accepted"; the paper does not spell the bookkeeping out).  After war_accept, makes the
+ * Commit (completes the step of paper Section 3.3: with accepted drafts a request advances by several tokens
+ * in one forward pass; the paper does not spell the bookkeeping out).  After war_accept, makes the
  * accepted path the end of each request's context, so that the next war_draft / war_verify_attn can run on the
  * same buffers:
  *   KV cache    the K/V rows of the accepted slots (logical positions prefix_len + slot) move to positions
@@ -317,9 +316,10 @@ war_status_t war_accept(const int32_t* d_ids, const int32_t* d_parent, const int
  * d_accept_path [B, N] as written by war_accept (slots strictly increasing).  Pools: bf16, D = 128, strides in
  * elements as in war_attn_params_t with unit stride along d and the others multiples of 8 (rows are moved 16
  * bytes at a time); both pools are modified in place.
+ * A request that is not running (tail_len[b] < 0, see war_draft) is left untouched and is no error.
  * A request whose path is malformed or whose rows lie beyond max_pages_per_req is left untouched and
  * WAR_ERR_BAD_TREE is recorded in the device status word; a page id outside [0, num_pages) records
- * WAR_ERR_BAD_PAGE and that row is skipped.  Enqueues two kernels on `stream`; does not synchronise.
+ * WAR_ERR_BAD_PAGE and the move of that row is skipped (its destination keeps what it held).  Enqueues two kernels on `stream`; does not synchronise.
  * ------------------------------------------------------------------------------------------------ */
 typedef struct {
     int32_t B, N, P;                 /* requests, slots per tree, tail window */
@@ -331,6 +331,17 @@ war_status_t war_commit(const int32_t* d_ids, const int32_t* d_accept_len, const
                         const int32_t* d_bonus, void* d_kpool, void* d_vpool, const int32_t* d_page_table,
                         const war_commit_params_t* params, int32_t* d_prefix_len, int32_t* d_tail,
                         int32_t* d_tail_len, war_stream_t stream);
+
+/* Diagnostic, no counterpart in the paper: exercises the bounded waits of the attention kernel without the kernel.
+ * Every wait inside the tensor-core kernel (on a tile that has not arrived, on a result that is not ready) gives up
+ * after a time budget, records WAR_ERR_TIMEOUT in the device status word and tells the other waiters of its thread
+ * block to stop, so that a lost signal ends the call with an error instead of hanging the GPU.  This call launches
+ * one small thread block in which one warp waits, with a budget of budget_us microseconds (1 .. 1 000 000), on a
+ * barrier that nobody will ever complete, and a second warp waits on the same barrier with the kernel's ordinary
+ * budget (2 s).  Expected afterwards: d_result [4] (int64, device) = { 0, 0, t0, t1 } -- both waits gave up, the
+ * first after about budget_us (t0, t1 in nanoseconds), the second released by the first, not by its own budget --
+ * and war_device_status reads WAR_ERR_TIMEOUT.  The kernel returns normally; later calls work as before. */
+war_status_t war_selftest_bounded_wait(int32_t budget_us, int64_t* d_result, war_stream_t stream);
 
 /* Reads and clears the sticky device status word (synchronises `stream`).  *h_status receives a
  * war_status_t value: WAR_OK, or the first device-side problem seen since the last read. */

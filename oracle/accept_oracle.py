@@ -1,8 +1,8 @@
 """Longest accepted root path by enumeration (test infrastructure).
 
-Verification is lossless (paper, Section 2.3: speculative decoding verifies drafts "while preserving the
-target output distribution"; Section 3.2: the rollout advances "by multiple tokens in a single forward pass
-when the drafts are accepted"): the step may only emit tokens the target model itself chose.  With the target's
+Verification is lossless (paper, Section 2.3: checking the drafts leaves the target model's output distribution
+as it is; Section 3.3: a request moves ahead by several tokens per forward pass whenever drafts are accepted): the
+step may only emit tokens the target model itself chose.  With the target's
 choices supplied as ids, a draft slot is accepted exactly when every slot on its root path equals the
 target's choice at that point.
 

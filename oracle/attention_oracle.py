@@ -1,8 +1,8 @@
 """Tree-masked GQA verification attention in fp64 (test infrastructure).
 
-The verifier scores all draft tokens of a request in one forward pass (paper, Section 3.2: predicted tokens
-"are then verified by the target model ... in a single forward pass"; Sections 2.3 and 5.3 name the
-auxiliary attention / tree mask this needs).  The attention of that pass, for request i, slot j, query head h
+The verifier scores all draft tokens of a request in one forward pass (paper, Section 3.3: the target model
+checks the predicted tokens together, in one pass; Sections 2.3 and 5.3 name the auxiliary attention / tree mask
+this needs).  The attention of that pass, for request i, slot j, query head h
 (kv head g = h // G):
 
     visible(j) = { all prefix positions 0 .. prefix_len-1 }  U  { prefix_len + a : a == j or a is an ancestor of j }

@@ -1,8 +1,8 @@
 """Advancing a request by its accepted tokens, written out plainly (test infrastructure).
 
-A speculate-and-verify step ends by making the accepted tokens part of the request (paper, Section 3.2: the
-rollout advances "by multiple tokens in a single forward pass when the drafts are accepted"; Section 2.3: the
-rejected drafts leave no trace, the output is the target model's own).  The paper does not spell the
+A speculate-and-verify step ends by making the accepted tokens part of the request (paper, Section 3.3: with accepted
+drafts a request moves ahead by several tokens in one forward pass; Section 2.3: the rejected drafts leave no trace,
+the output is the target model's own).  The paper does not spell the
 bookkeeping out; this is the reading used here, in the slot convention of the draft tree (slot 0 = the
 request's last context token, whose K/V sits at logical position prefix_len, slot j at prefix_len + j):
 

@@ -1,8 +1,8 @@
 """Longest-suffix match and draft-tree construction by brute force (test infrastructure).
 
-What is computed (paper, Section 3: SuffixDecoding "stores the historical trajectories and matches the
-current token pattern against them to generate draft tokens"; Section 3.2: it "caches token-sequence
-patterns from previously generated trajectories" and predicts likely next tokens from them):
+What is computed (paper, Section 3: SuffixDecoding keeps the trajectories generated so far and drafts by
+matching the request's current tokens against them; Section 3.3: the cache holds the token patterns of earlier
+trajectories, and likely next tokens are predicted from them):
 
   match   the largest l <= min(P, tail_len) such that the last l context tokens occur contiguously inside
           ONE stored trajectory (occurrences never straddle two trajectories);
@@ -138,7 +138,7 @@ def build_draft_tree(corpus: Corpus, tail: np.ndarray, match_len: int, ends: np.
                      min_match: int = 1, spec_factor=(0, 1), min_prob=(0, 1)):
     """Returns (ids, parent, count) int32 arrays of length num_nodes (see module docstring for the rules).
 
-    Two thresholds of the SuffixDecoding method the paper builds on (Section 3.2 takes that method's code base;
+    Two thresholds of the SuffixDecoding method the paper builds on (Section 3.3 takes that method's code base;
     the paper itself names neither), both exact integer rules:
       spec_factor (a, b), a > 0: the tree has at most 1 + floor(match_len * a / b) slots (a longer match earns a
                   larger tree); (0, .) = no such cap.
@@ -207,7 +207,7 @@ def tree_score(count: np.ndarray) -> Tuple[int, int]:
 def draft_scored(corpus: Corpus, tail: np.ndarray, tail_len: int, N: int, k: int, n_lengths: int, min_match: int = 1,
                  spec_factor=(0, 1), min_prob=(0, 1)):
     """Draft from the best-scoring of several suffix lengths instead of from the longest match alone (a variant of
-    the SuffixDecoding method the paper adopts in Section 3.2; the paper itself does not spell it out).
+    the SuffixDecoding method the paper adopts in Section 3.3; the paper itself does not spell it out).
 
     Candidates are the lengths match_len, match_len - 1, ..., down n_lengths of them, never below max(1, min_match)
     (every shorter suffix of an occurring string occurs too).  Each candidate gets its own tree by the rules of
@@ -259,7 +259,7 @@ def draft_batch(corpus: Corpus, tails: np.ndarray, tail_len: np.ndarray, N: int,
                 spec_batch_limit: int = 0, spec_factor=(0, 1), min_prob=(0, 1)):
     """Batched form with the library's output convention: unused slots hold ids = -1, parent = -1, count = 0.
 
-    Workload-aware switch (paper, Section 3.2, "adaptive enabling and disabling" by the current batch size, and
+    Workload-aware switch (paper, Section 3.3: speculation is switched on and off by the current batch size, and
     Section 5.3: beyond a batch of about 16 speculation costs more than it gains): a request with
     tail_len < 0 is not running (no tree at all); the effective batch size is the number of running requests;
     when spec_batch_limit > 0 and the effective batch size exceeds it, nothing is looked up and every running

@@ -1,7 +1,7 @@
 """Drafting from the request's own context, and the choice between two draft trees (test infrastructure).
 
-The SuffixDecoding method that the paper adopts (Section 3.2: it "caches token-sequence patterns from previously
-generated trajectories") keeps, besides the cache of finished trajectories, the tokens of the running request itself:
+The SuffixDecoding method that the paper adopts (Section 3.3: a cache of the token patterns of earlier
+trajectories) keeps, besides the cache of finished trajectories, the tokens of the running request itself:
 text that a rollout has produced or read once (a file, a tool result) tends to come back inside the same trajectory.
 The paper does not spell this part out; the rules below are this build's reading and are listed in the design notes.
 

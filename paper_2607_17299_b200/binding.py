@@ -28,6 +28,7 @@ STATUS_NAMES = {0: "WAR_OK", 1: "WAR_ERR_INVALID_ARG", 2: "WAR_ERR_OOM", 3: "WAR
 EXPORTS = ["war_index_build", "war_index_append", "war_index_evict", "war_index_export_bytes", "war_index_export",
            "war_index_import", "war_index_info", "war_index_destroy", "war_draft", "war_draft_scored_workspace_bytes", "war_draft_scored", "war_draft_local", "war_draft_pick",
            "war_verify_attn_workspace_bytes", "war_verify_attn", "war_verify_attn_noalloc", "war_accept", "war_commit", "war_device_status",
+           "war_selftest_bounded_wait",
            "war_status_string"]
 
 
@@ -342,6 +343,15 @@ def war_commit(d_ids: torch.Tensor, d_accept_len: torch.Tensor, d_accept_path: t
                            _ptr(page_table, torch.int32), C.byref(p), _ptr(d_prefix_len, torch.int32),
                            _ptr(d_tail, torch.int32), _ptr(d_tail_len, torch.int32), _stream())
     _check("war_commit", code)
+
+
+_lib.war_selftest_bounded_wait.restype = C.c_int
+_lib.war_selftest_bounded_wait.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
+
+
+def war_selftest_bounded_wait(budget_us: int, d_result: torch.Tensor) -> None:
+    """d_result: int64 [4] CUDA tensor; see include/war.h."""
+    _check("war_selftest_bounded_wait", _lib.war_selftest_bounded_wait(int(budget_us), _ptr(d_result, torch.int64), _stream()))
 
 
 def war_device_status() -> int:

@@ -60,6 +60,7 @@ war_commit_kv_kernel(const int32_t* __restrict__ accept_len, const int32_t* __re
     // item = (move d, K or V, 16-byte piece); a move whose row is already in place is skipped on both sides
     const int items = k * 2 * kPiecesPerRow;
     uint4 buf[kMaxPerThread];
+    unsigned have = 0;                                           // bit r: buf[r] holds a row piece that was really read
 #pragma unroll
     for (int r = 0; r < kMaxPerThread; ++r) {
         const int it = threadIdx.x + r * kKvThreads;
@@ -68,7 +69,7 @@ war_commit_kv_kernel(const int32_t* __restrict__ accept_len, const int32_t* __re
             const int d = it / (2 * kPiecesPerRow), which = (it / kPiecesPerRow) & 1, piece = it % kPiecesPerRow;
             if (s_path[d] != d + 1) {
                 const uint4* src = row_ptr(which, pl + s_path[d]);
-                if (src) buf[r] = src[piece];
+                if (src) { buf[r] = src[piece]; have |= 1u << r; }
             }
         }
     }
@@ -78,7 +79,7 @@ war_commit_kv_kernel(const int32_t* __restrict__ accept_len, const int32_t* __re
         const int it = threadIdx.x + r * kKvThreads;
         if (it < items) {
             const int d = it / (2 * kPiecesPerRow), which = (it / kPiecesPerRow) & 1, piece = it % kPiecesPerRow;
-            if (s_path[d] != d + 1) {
+            if (s_path[d] != d + 1 && ((have >> r) & 1u)) {        // a row whose source page was bad is skipped, not zeroed
                 uint4* dst = row_ptr(which, pl + 1 + d);
                 if (dst) dst[piece] = buf[r];
             }
@@ -94,6 +95,7 @@ __global__ void war_commit_ctx_kernel(const int32_t* __restrict__ ids, const int
     const int lane = threadIdx.x & 31;
     if (b >= B) return;
     const int k = accept_len[b], pl = prefix_len[b], tl = tail_len[b], bn = bonus[b];
+    if (tl < 0) return;                                                    // not running (see war_draft): nothing to advance
     bool ok = pl >= 0 && tl >= 0 && tl <= P && path_ok(accept_path + (size_t)b * N, k, N);
     if (ok && k > 0) ok = (pl + accept_path[(size_t)b * N + k - 1]) / page_size < max_pages;
     if (!ok) {

@@ -1,6 +1,6 @@
 // war_draft_local: draft trees from each request's own context, and war_draft_pick: the choice between two trees.
 //
-// The SuffixDecoding method that the paper adopts (Section 3.2) also drafts from the tokens of the running request
+// The SuffixDecoding method that the paper adopts (Section 3.3) also drafts from the tokens of the running request
 // itself: text a rollout has produced or read once tends to come back inside the same trajectory.  A context changes
 // every step, so no index is kept for it: a cluster of up to 8 CTAs per request scans the context, a slice each (4
 // bytes per token, a few microseconds even at 10^5 tokens), for the longest suffix that occurs earlier and for its 32

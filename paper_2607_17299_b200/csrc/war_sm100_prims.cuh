@@ -34,16 +34,19 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     return t;
 }
 
-// Bounded wait.  Returns false when the CTA is aborting (this wait ran out of time, or another one did).
+// Bounded wait.  Returns false when the CTA is aborting (this wait ran out of time, or another one did): the
+// waiter that runs out of its budget records WAR_ERR_TIMEOUT and raises the CTA's abort flag, which ends every
+// other wait of the CTA the next time it looks.  Nothing traps and nothing spins for ever.
 template <class BarsT>
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, BarsT* bars, int* status_word) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, BarsT* bars, int* status_word,
+                                          unsigned long long budget_ns = kWaitBudgetNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     unsigned spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 255u) == 0) {
             if (*(volatile int*)&bars->abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitBudgetNs) {
+            if (global_timer_ns() - t0 > budget_ns) {
                 war_set_device_status(status_word, WAR_ERR_TIMEOUT);
                 atomicExch(&bars->abort_flag, 1);
                 return false;

@@ -925,6 +925,39 @@ war_status_t device_setup(int dev) {
 
 }  // namespace
 
+namespace {
+// Self-test of the bounded waits (see war.h): one CTA, an mbarrier nobody ever arrives on.  Warp 0 waits on it with
+// the caller's budget through the same mbar_wait the attention kernel uses, runs out of it, records WAR_ERR_TIMEOUT
+// and raises the abort flag; warp 1 waits on the same barrier with the kernel's ordinary (long) budget and is
+// released by that flag.  result = { warp 0's wait returned true?, warp 1's, ns warp 0 waited, ns warp 1 waited }.
+struct SelftestBars { uint64_t never; int abort_flag; };
+__global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(unsigned long long budget_ns, long long* result, int* status_word) {
+    __shared__ SelftestBars bars;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        mbar_init(&bars.never, 1);
+        bars.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const unsigned long long t0 = global_timer_ns();
+    const bool ok = warp == 0 ? mbar_wait(&bars.never, 0u, &bars, status_word, budget_ns)
+                              : mbar_wait(&bars.never, 0u, &bars, status_word);
+    const unsigned long long dt = global_timer_ns() - t0;
+    if (lane == 0) { result[warp] = ok ? 1 : 0; result[2 + warp] = (long long)dt; }
+}
+
+}  // namespace
+
+extern "C" war_status_t war_selftest_bounded_wait(int32_t budget_us, int64_t* d_result, war_stream_t stream) {
+    if (!d_result || budget_us < 1 || budget_us > 1000000) return WAR_ERR_INVALID_ARG;
+    int* status_word = war_status_word();
+    if (!status_word) return WAR_ERR_CUDA;
+    bounded_wait_selftest_kernel<<<1, 64, 0, stream>>>((unsigned long long)budget_us * 1000ull, (long long*)d_result, status_word);
+    WAR_LAUNCH_CHECK();
+    return WAR_OK;
+}
+
 int war_attn_sm_count() {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return 0; }

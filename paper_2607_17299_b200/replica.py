@@ -3,7 +3,7 @@
 The step itself needs no exchange: every rank (one process per GPU = one rollout replica) holds the whole
 trajectory index and its own requests and KV cache.  The one exchange the method has is at the end of an RL step,
 when every replica must add the trajectories that ALL replicas finished in that step to its own index (the paper's
-cross-worker suffix-cache synchronisation, Section 3.2).  `gather_trajectories` does that with plain
+cross-worker suffix-cache synchronisation, Section 3.3).  `gather_trajectories` does that with plain
 `torch.distributed` collectives into each rank's own memory, in rank order, so that every rank appends the same
 trajectories in the same order; `append_step_trajectories` then calls the library's `war_index_append`.
 """

@@ -356,3 +356,28 @@ def test_mid_size_batches_through_every_plan(war, seed):
     assert war.war_device_status() == 0
     del a
     torch.cuda.empty_cache()
+
+
+def test_a_wait_that_runs_out_ends_with_an_error_not_a_hang(war):
+    """Every wait inside the tensor-core kernel has a time budget.  The library's self-test runs the same wait routine
+    on a barrier that nobody completes: the waiter gives up after its budget (here 1 ms instead of the kernel's 2 s),
+    WAR_ERR_TIMEOUT is recorded, a second waiter is released by the first one's abort flag long before its own budget,
+    the kernel returns normally, and the library works afterwards."""
+    d = U.dev()
+    assert war.war_device_status() == 0
+    res = torch.full((4,), -1, dtype=torch.int64, device=d)
+    war.war_selftest_bounded_wait(1000, res)
+    torch.cuda.synchronize()
+    ok0, ok1, ns0, ns1 = res.cpu().tolist()
+    assert ok0 == 0 and ok1 == 0                                     # both waits gave up
+    assert 1_000_000 <= ns0 < 200_000_000                            # the first after its budget (not the 2 s default)
+    assert ns1 < 200_000_000                                         # the second because the first raised the flag
+    assert war.war_device_status() == 5                              # WAR_ERR_TIMEOUT, read and cleared
+    assert war.war_device_status() == 0
+    with pytest.raises(war.WarError):
+        war.war_selftest_bounded_wait(0, res)
+    # the context is intact: an ordinary call right after
+    rng = np.random.default_rng(5)
+    cfg = W.scaled(W.CONFIGS["tiny"], B=3, N=8)
+    nn, parent = _random_trees(rng, cfg.B, cfg.N)
+    _check(war, cfg, np.array([900, 130, 2500]), nn, parent, 0)

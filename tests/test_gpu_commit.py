@@ -139,6 +139,36 @@ def test_malformed_paths_and_pages_are_reported(war):
     war.war_commit(t(ids), t(np.array([0, 2, 0, 0], np.int32)), t(path), t(bonus), k_pool, v_pool, t(pt_bad), d_pl, t(tail), t(tl))
     torch.cuda.synchronize()
     assert war.war_device_status() == 8                                        # WAR_ERR_BAD_PAGE
+    # a bad SOURCE page with a good destination: the destination row keeps what it held (it is not zeroed)
+    pt_src = pt.copy(); pt_src[1, (41 + 7) // pg] = -5                         # slot 7 of request 1 lives on its own page
+    assert (41 + 7) // pg != (41 + 1) // pg
+    path2 = np.full((B, N), -1, np.int32); path2[1, 0] = 7
+    kb, vb = k_pool.clone(), v_pool.clone()
+    war.war_commit(t(ids), t(np.array([0, 1, 0, 0], np.int32)), t(path2), t(bonus), k_pool, v_pool, t(pt_src), t(pl), t(tail), t(tl))
+    torch.cuda.synchronize()
+    assert war.war_device_status() == 8
+    assert torch.equal(k_pool, kb) and torch.equal(v_pool, vb)
+
+
+def test_not_running_requests_are_left_alone(war):
+    """tail_len < 0 marks a request that is not running (war_draft gives it no tree, war_accept an empty result):
+    the commit must not touch it and must not report it as malformed."""
+    rng = np.random.default_rng(8)
+    B, N, Hkv, pg, P = 3, 8, 2, 16, 8
+    pl = np.array([40, 41, 42], np.int32)
+    k_pool, v_pool, pt = _pool(rng, B, pl + N, Hkv, pg)
+    ids = rng.integers(0, 50, (B, N)).astype(np.int32)
+    alen = np.array([1, 0, 0], np.int32)
+    path = np.full((B, N), -1, np.int32); path[0, 0] = 3
+    bonus = np.array([9, -1, 4], np.int32)
+    tail = rng.integers(0, 50, (B, P)).astype(np.int32); tl = np.array([P, -1, 2], np.int32)
+    t = lambda x: torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).to(DEV)
+    d_pl, d_tail, d_tl = t(pl), t(tail), t(tl)
+    war.war_commit(t(ids), t(alen), t(path), t(bonus), k_pool, v_pool, t(pt), d_pl, d_tail, d_tl)
+    torch.cuda.synchronize()
+    assert war.war_device_status() == 0
+    assert d_pl.cpu().tolist() == [42, 41, 43] and d_tl.cpu().tolist() == [P, -1, 3]
+    assert torch.equal(d_tail.cpu()[1], torch.from_numpy(tail[1]))
 
 
 def test_steps_in_a_row(war):

@@ -1,6 +1,6 @@
 """The three calls of a step enqueue work and return without touching the host, so a whole step can be captured
 in a CUDA graph and replayed (the paper's engine keeps separate CUDA graphs for speculative and plain decoding,
-Section 3.2).  Replays must reproduce the eager results bit for bit, also after the inputs change in place."""
+Section 3.3).  Replays must reproduce the eager results bit for bit, also after the inputs change in place."""
 import numpy as np
 import pytest
 import torch
@@ -75,7 +75,7 @@ def test_step_replays_from_a_cuda_graph(war):
 
 
 def test_one_graph_serves_speculative_and_plain_steps(war):
-    """Workload-aware switch inside a captured step (paper Section 3.2: adaptive enabling by batch size, stateless
+    """Workload-aware switch inside a captured step (paper Section 3.3: adaptive enabling by batch size, stateless
     switching, CUDA-graph compatibility): the number of running requests is read on the device, so the same graph
     speculates while few requests run and does plain decode steps (root-only trees) when many do."""
     from oracle import draft_oracle as D
@@ -97,10 +97,16 @@ def test_one_graph_serves_speculative_and_plain_steps(war):
     params = war.attn_params(a.q, a.k_pool, a.v_pool, a.page_table, 1.0 / np.sqrt(cfg.D), 0)
     ws = war.new_workspace(params, dev)
 
+    # the commit works on copies (made inside the step), so that every replay starts from the same request state
+    c_k, c_v = a.k_pool.clone(), a.v_pool.clone()
+    c_pl, c_tails, c_tl = a.prefix_len.clone(), d_tails.clone(), d_tl.clone()
+
     def step():
         war.war_draft(ix, d_tails, d_tl, N, cfg.topk, 1, ml, nn, ids, par, cnt, limit)
         war.war_verify_attn(a.q, a.k_pool, a.v_pool, a.page_table, a.prefix_len, nn, par, params, ws, out, None)
         war.war_accept(ids, par, nn, target, 0, alen, path, bonus)
+        c_pl.copy_(a.prefix_len); c_tails.copy_(d_tails); c_tl.copy_(d_tl)
+        war.war_commit(ids, alen, path, bonus, c_k, c_v, a.page_table, c_pl, c_tails, c_tl)
 
     step()
     torch.cuda.synchronize()
@@ -127,6 +133,13 @@ def test_one_graph_serves_speculative_and_plain_steps(war):
         o = out.float().cpu().numpy()
         for i in range(B):                                             # rows beyond num_nodes are never written
             assert (o[i, h_nn[i]:] == 7.0).all() and (h_nn[i] == 0 or (o[i, 0] != 7.0).any())
+        # the commit leaves requests that are not running alone (and does not call them malformed) and advances the others
+        h_cpl, h_ctl, h_ct = c_pl.cpu().numpy(), c_tl.cpu().numpy(), c_tails.cpu().numpy()
+        h_pl, h_alen = a.prefix_len.cpu().numpy(), alen.cpu().numpy()
+        assert (h_cpl[running:] == h_pl[running:]).all() and (h_ctl[running:] == -1).all()
+        assert (h_ct[running:] == tails[running:]).all()
+        assert (h_cpl[:running] == h_pl[:running] + h_alen[:running] + 1).all()
+        assert war.war_device_status() == 0
     assert war.war_device_status() == 0
     ix.destroy()
 

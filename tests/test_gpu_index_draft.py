@@ -351,7 +351,7 @@ def test_node_budget_and_probability_threshold(war, spec_factor, min_prob):
 
 def test_drafts_keep_running_while_the_index_is_updated(war):
     """war_index_append builds the new arrays beside the published ones and publishes them when they are complete
-    (the paper updates the cache asynchronously so that the update does not block the pipeline, Section 3.2).  One
+    (the paper updates the cache asynchronously so that the update does not block the pipeline, Section 3.3).  One
     thread drafts in a loop on its own stream while another appends twice; every draft result must equal the
     brute-force checker's answer on one of the three corpus states, and the states must appear in order."""
     import threading

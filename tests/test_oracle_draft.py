@@ -182,7 +182,7 @@ def test_tree_invariants_on_tiny_workload(tiny):
 
 def test_trajectory_order_does_not_matter(tiny):
     """Every worker must draft the same tokens once the caches hold the same trajectories, in whatever order
-    they arrived (paper Section 3.2, cross-worker synchronisation)."""
+    they arrived (paper Section 3.3, cross-worker synchronisation)."""
     cfg, tok, off, tails, tl, _ = tiny
     rng = np.random.default_rng(11)
     order = rng.permutation(cfg.n_traj)
