@@ -74,10 +74,15 @@ typedef struct war_index war_index_t;          /* opaque; lives on the device th
  * the pipeline, Section 3.3): the index keeps two sets of (suffix array, LCP, buckets).  war_index_append builds
  * the new set beside the published one and publishes it just before it returns; the corpus is only written
  * behind what the published set refers to.  So ONE thread may run war_index_append (on its own stream) while other
- * threads keep calling war_draft on other streams: a war_draft call uses the set that is published at the moment
- * it is called, and that set stays intact until the NEXT update starts.  The caller makes sure that update does
- * not start before those drafts have finished (an event, or one update per step).  Two updates must not
- * overlap each other.  Cost: 5 more bytes per token of capacity.
+ * threads keep calling war_draft on other streams: a draft kernel takes the set that is published at the moment
+ * it STARTS on the device (it reads the published set's number from device memory), and that set stays intact
+ * until the NEXT update starts.  The caller makes sure that update does not start before those drafts have
+ * finished (an event, or one update per step).  Two updates must not overlap each other.  Cost: 5 more bytes per
+ * token of capacity.
+ * CUDA graphs: because the set is chosen on the device, a captured war_draft / war_draft_scored launch keeps
+ * answering from the current index after any number of war_index_append / war_index_evict calls; nothing has to
+ * be captured again.  (The graph holds the index handle's device addresses: destroy the index only when the graph
+ * is no longer replayed.)
  * ------------------------------------------------------------------------------------------------ */
 war_status_t war_index_build(const int32_t* d_tokens, const int64_t* h_offsets, int32_t T,
                              int32_t vocab, int32_t max_depth, int64_t capacity_tokens,

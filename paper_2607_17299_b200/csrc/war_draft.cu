@@ -236,14 +236,20 @@ struct Shared {
 // grid fits the SMs anyway, which is the low-load case where this kernel's latency matters most.
 template <int kCtasPerSm>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
-war_draft_kernel(const int32_t* __restrict__ corpus, const int32_t* __restrict__ sa, const uint8_t* __restrict__ lcp,
-                 const int32_t* __restrict__ bucket, int32_t* memo, int vocab, const int32_t* __restrict__ tail,
+war_draft_kernel(const int32_t* __restrict__ corpus, const war_index_view* __restrict__ view, int vocab, const int32_t* __restrict__ tail,
                  const int32_t* __restrict__ tail_len, int B, int P, int N, int K, int min_match, int spec_batch_limit,
                  int fac_num, int fac_den, int prob_num, int prob_den, int32_t* __restrict__ match_len, int32_t* __restrict__ num_nodes, int32_t* __restrict__ ids,
                  int32_t* __restrict__ parent, int32_t* __restrict__ count, int32_t* __restrict__ cand_len) {
     __shared__ Shared sh;
     const int b = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // The index arrays come from the set that is published NOW (not when the launch was enqueued or captured): the
+    // request for them goes out first and is in flight while the tail is read.
+    const war_index_arrays arrays = view->set[*(const volatile unsigned int*)&view->cur & 1u];
+    const int32_t* __restrict__ sa = arrays.sa;
+    const uint8_t* __restrict__ lcp = arrays.lcp;
+    const int32_t* __restrict__ bucket = arrays.bucket;
+    int32_t* memo = arrays.memo;
     // Scoring several suffix lengths: CTA (b, c) drafts request b from the suffix that is c tokens shorter than the
     // longest match and leaves its tree in row b * gridDim.y + c of the candidate arrays (all output pointers then
     // address those); a second kernel picks the winner.  With one candidate per request the row is the request.
@@ -854,15 +860,14 @@ war_status_t launch_draft(const war_index_t* ix, const int32_t* d_tail, const in
     const int dev = ix->device;
     if (dev < 0 || dev >= 64) return WAR_ERR_INVALID_ARG;
     if (!sm_count[dev]) WAR_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
-    const war_index_arrays arr = const_cast<war_index_t*>(ix)->published();       // a complete index, also during an update
     const dim3 grid(p->B, n_cand);
     const int fac_den = p->spec_factor_num > 0 ? p->spec_factor_den : 1, prob_den = p->min_prob_num > 0 ? p->min_prob_den : 1;
     if ((long long)p->B * n_cand <= sm_count[dev])
-        war_draft_kernel<1><<<grid, kThreads, 0, stream>>>(ix->corpus, arr.sa, arr.lcp, arr.bucket, arr.memo, ix->vocab, d_tail, d_tail_len,
+        war_draft_kernel<1><<<grid, kThreads, 0, stream>>>(ix->corpus, ix->d_view, ix->vocab, d_tail, d_tail_len,
                                                           p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, p->spec_factor_num,
                                                           fac_den, p->min_prob_num, prob_den, match_len, num_nodes, ids, parent, count, cand_len);
     else
-        war_draft_kernel<2><<<grid, kThreads, 0, stream>>>(ix->corpus, arr.sa, arr.lcp, arr.bucket, arr.memo, ix->vocab, d_tail, d_tail_len,
+        war_draft_kernel<2><<<grid, kThreads, 0, stream>>>(ix->corpus, ix->d_view, ix->vocab, d_tail, d_tail_len,
                                                           p->B, p->P, p->N, p->topk, p->min_match, p->spec_batch_limit, p->spec_factor_num,
                                                           fac_den, p->min_prob_num, prob_den, match_len, num_nodes, ids, parent, count, cand_len);
     WAR_LAUNCH_CHECK();

@@ -234,8 +234,7 @@ war_status_t finish_index(war_index* ix, cudaStream_t s) {
     bucket_from_sa_kernel<<<grid_for(M + 1), kThreads, 0, s>>>(ix->corpus, a.sa, M, ix->vocab, a.bucket);
     WAR_LAUNCH_CHECK();
     WAR_CUDA_TRY(cudaMemsetAsync(a.memo, 0, sizeof(int32_t) * kMemoEntries * kMemoInts, s));   // it described another suffix array
-    WAR_CUDA_TRY(cudaStreamSynchronize(s));
-    ix->publish();
+    WAR_CUDA_TRY(ix->publish(s));
     return WAR_OK;
 }
 
@@ -244,8 +243,7 @@ war_status_t rebuild(war_index* ix, cudaStream_t s) {
     const int64_t M = ix->M;
     if (M == 0) {
         WAR_CUDA_TRY(cudaMemsetAsync(ix->shadow().bucket, 0, sizeof(int32_t) * (ix->vocab + 1), s));
-        WAR_CUDA_TRY(cudaStreamSynchronize(s));
-        ix->publish();
+        WAR_CUDA_TRY(ix->publish(s));
         return WAR_OK;
     }
     const war_status_t st = sort_suffixes(ix->corpus, M, ix->T, ix->vocab, ix->max_depth, ix->shadow().sa, s);
@@ -436,8 +434,7 @@ war_status_t evict_oldest(war_index* ix, int32_t n, cudaStream_t s) {
     ix->T -= n;
     if (M == 0) {
         WAR_CUDA_TRY(cudaMemsetAsync(ix->shadow().bucket, 0, sizeof(int32_t) * (ix->vocab + 1), s));
-        WAR_CUDA_TRY(cudaStreamSynchronize(s));
-        ix->publish();
+        WAR_CUDA_TRY(ix->publish(s));
         return WAR_OK;
     }
     return finish_index(ix, s);
@@ -472,6 +469,13 @@ extern "C" war_status_t war_index_build(const int32_t* d_tokens, const int64_t* 
         if (e == cudaSuccess) e = cudaMemsetAsync(ix->set[k].bucket, 0, sizeof(int32_t) * (vocab + 1), stream);
     }
     if (e == cudaSuccess) e = cudaMemsetAsync(ix->corpus, 0xff, sizeof(int32_t) * (cap + 128), stream);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ix->d_view, sizeof(war_index_view));
+    if (e == cudaSuccess) {
+        war_index_view v;
+        v.set[0] = ix->set[0]; v.set[1] = ix->set[1]; v.cur = (unsigned int)ix->cur;
+        e = cudaMemcpyAsync(ix->d_view, &v, sizeof(v), cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(stream);            // (v is a local)
+    }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         war_index_destroy(ix);
@@ -584,12 +588,11 @@ extern "C" war_status_t war_index_import(const void* h_src, size_t bytes, int64_
     at += pad8(M);
     if (e == cudaSuccess) e = cudaMemcpyAsync(a.bucket, at, sizeof(int32_t) * ((size_t)h.vocab + 1), cudaMemcpyHostToDevice, stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(a.memo, 0, sizeof(int32_t) * kMemoEntries * kMemoInts, stream);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) { (void)cudaGetLastError(); war_index_destroy(ix); return WAR_ERR_CUDA; }
     try { ix->bounds.assign(bounds, bounds + h.T + 1); } catch (...) { war_index_destroy(ix); return WAR_ERR_OOM; }
     ix->M = h.M;
     ix->T = h.T;
-    ix->publish();
+    if (ix->publish(stream) != cudaSuccess) { (void)cudaGetLastError(); war_index_destroy(ix); return WAR_ERR_CUDA; }
     *out = ix;
     return WAR_OK;
 }
@@ -613,6 +616,7 @@ extern "C" war_status_t war_index_info(const war_index_t* ix, war_index_info_t* 
 extern "C" war_status_t war_index_destroy(war_index_t* ix) {
     if (!ix) return WAR_OK;
     if (ix->corpus) cudaFree(ix->corpus);
+    if (ix->d_view) cudaFree(ix->d_view);
     for (int k = 0; k < 2; ++k) {
         if (ix->set[k].sa) cudaFree(ix->set[k].sa);
         if (ix->set[k].lcp) cudaFree(ix->set[k].lcp);

@@ -1,6 +1,7 @@
 // The index object behind war_index_t (library-internal).
 #pragma once
 #include <stdint.h>
+#include <cuda_runtime.h>
 #include <mutex>
 #include <vector>
 
@@ -21,10 +22,19 @@ struct war_index_arrays {
 constexpr int kMemoEntries = 1 << 16;
 constexpr int kMemoInts = 32;             // 128 bytes per entry
 
+// What a draft kernel needs of the index, readable on the device: both array sets (their addresses never change after
+// the build) and the number of the published one.  Kernels take the published set through this view when they START,
+// not when they are enqueued, so a launch captured in a CUDA graph follows the index through later updates.
+struct war_index_view {
+    war_index_arrays set[2];
+    unsigned int cur;            // written in stream order by every publication
+};
+
 struct war_index {
     int32_t* corpus = nullptr;   // [capacity + slack] trajectories joined by unique negative separators
     war_index_arrays set[2];
-    int cur = 0;                 // published set; guarded by `lock` together with the pointers handed to queries
+    war_index_view* d_view = nullptr;   // device copy of (set, cur)
+    int cur = 0;                 // published set (host copy); guarded by `lock` together with the pointers handed to queries
     std::mutex lock;
     int64_t M = 0;               // corpus entries in use
     int64_t capacity = 0;
@@ -36,5 +46,15 @@ struct war_index {
 
     war_index_arrays published() { std::lock_guard<std::mutex> g(lock); return set[cur]; }
     war_index_arrays& shadow() { return set[cur ^ 1]; }                  // only the (single) updater touches it
-    void publish() { std::lock_guard<std::mutex> g(lock); cur ^= 1; }
+    // Publication: the device view first (on the updater's stream, behind everything that built the set; the caller
+    // synchronises that stream before it reports success), then the host copy.
+    cudaError_t publish(cudaStream_t s) {
+        const unsigned int next = (unsigned int)(cur ^ 1);
+        cudaError_t e = cudaMemcpyAsync(&d_view->cur, &next, sizeof(next), cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) return e;
+        std::lock_guard<std::mutex> g(lock);
+        cur ^= 1;
+        return cudaSuccess;
+    }
 };

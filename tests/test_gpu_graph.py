@@ -206,3 +206,59 @@ def test_drafting_variants_replay_from_a_graph(war):
         assert np.array_equal(gpu.cpu().numpy(), want)
     assert war.war_device_status() == 0
     ix.destroy()
+
+
+def test_a_captured_draft_follows_the_index_through_updates(war):
+    """The draft kernel picks the published set of index arrays when it starts, from device memory, so a launch that
+    was captured before an update answers from the updated index when it is replayed: capture, append, replay, append
+    again (the first captured set is being rebuilt now), evict, replay -- every replay equals the checker on the corpus
+    as it is at that moment."""
+    from oracle import draft_oracle as D
+    dev = U.dev()
+    cfg = W.scaled(W.CONFIGS["tiny"], B=8, n_traj=40)
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(cfg)
+    N, k = cfg.N, cfg.topk
+    first, second = 20, 30                                            # 20 trajectories, then +10, then +10
+    cap = len(tok) + cfg.n_traj
+    ix = U.build_index(war, tok[:off[first]], off[:first + 1], cfg.vocab, max_depth=cfg.P + N, capacity=cap)
+    i32 = dict(dtype=torch.int32, device=dev)
+    d_tails, d_tl = torch.from_numpy(tails).to(dev), torch.from_numpy(tl).to(dev)
+    ml, nn = torch.zeros(cfg.B, **i32), torch.zeros(cfg.B, **i32)
+    ids, par, cnt = (torch.zeros((cfg.B, N), **i32) for _ in range(3))
+
+    def draft():
+        war.war_draft(ix, d_tails, d_tl, N, k, 1, ml, nn, ids, par, cnt)
+
+    def check(n_from, n_to):
+        torch.cuda.synchronize()
+        o = off[n_from:n_to + 1] - off[n_from]
+        want = D.draft_batch(D.Corpus(tok[off[n_from]:off[n_to]], o), tails, tl, N, k)
+        for got, w in zip((ml, nn, ids, par, cnt), want):
+            assert np.array_equal(got.cpu().numpy(), w), (n_from, n_to)
+
+    draft()
+    check(0, first)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        draft()
+    torch.cuda.current_stream().wait_stream(side)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        draft()
+    g.replay()
+    check(0, first)
+    d_tok = torch.from_numpy(tok).to(dev)
+    war.war_index_append(ix, d_tok[off[first]:off[second]], off[first:second + 1] - off[first])
+    g.replay()
+    check(0, second)
+    war.war_index_append(ix, d_tok[off[second]:], off[second:] - off[second])
+    g.replay()
+    check(0, cfg.n_traj)
+    war.war_index_evict(ix, 5)
+    g.replay()
+    check(5, cfg.n_traj)
+    assert war.war_device_status() == 0
+    del g
+    ix.destroy()
