@@ -375,3 +375,30 @@ def make_targets(cfg: WorkloadConfig, ids: np.ndarray, parent: np.ndarray, num_n
             if c >= 0:
                 out[i, p] = (ids[i, c] + 1 + shift[i, p]) % cfg.vocab if flip[i, p] else ids[i, c]
     return out
+
+
+def make_targets_device(cfg: WorkloadConfig, ids: torch.Tensor, parent: torch.Tensor, num_nodes: torch.Tensor,
+                        step: int) -> torch.Tensor:
+    """Per-slot target ids (mode 0 of `make_targets`) made on the device from device-resident trees, for benchmark
+    steps whose trees change from step to step: a slot with children agrees with its lowest-numbered child with
+    probability 1 - mismatch, otherwise it is a different token; a leaf gets a uniform random token.  Randomness is
+    a counter hash of (step, request, slot).  This stands in for the target model's sampled tokens; it is input
+    generation, not part of the method."""
+    B, N = ids.shape
+    dev = ids.device
+    j = torch.arange(N, device=dev, dtype=torch.int64).expand(B, N)
+    live = (j >= 1) & (j < num_nodes.to(torch.int64)[:, None])
+    first_child = torch.full((B, N), N, dtype=torch.int64, device=dev)
+    first_child.scatter_reduce_(1, parent.clamp(min=0).to(torch.int64), torch.where(live, j, torch.full_like(j, N)), "amin",
+                                include_self=True)
+    has = first_child < N
+    child_id = ids.to(torch.int64).gather(1, first_child.clamp(max=N - 1))
+    idx = torch.arange(B * N, device=dev, dtype=torch.int64).view(B, N) + (int(step) + 1) * (1 << 24)
+    h = _mix(idx * (-7046029254386353131) + (int(seed_streams(cfg)[5].entropy) & 0xFFFF))
+    u = ((h >> 40) & 0xFFFFFF).to(torch.float64) / float(1 << 24)
+    shift = (h >> 8) & 0x7FFFFFFF
+    flip = u < cfg.mismatch
+    rnd = shift % cfg.vocab
+    wrong = (child_id + 1 + shift % (cfg.vocab - 1)) % cfg.vocab
+    out = torch.where(has, torch.where(flip, wrong, child_id), rnd)
+    return out.to(torch.int32)

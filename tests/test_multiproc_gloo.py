@@ -38,6 +38,7 @@ def _worker(rank, world, port, out_dir):
     try:
         tok, off = _rank_trajectories(rank)
         all_tok, all_off = replica.gather_trajectories(tok, off, "cpu")
+        all_tok = all_tok.numpy()
         # drafts from the merged history, for a fixed set of probes
         corpus = D.Corpus(all_tok, all_off)
         rng = np.random.default_rng(7)
@@ -71,6 +72,20 @@ def test_trajectory_exchange_and_sharding(tmp_path):
     assert (res[2] == r0["ids"]).all() and (res[3] == r0["parent"]).all() and (res[4] == r0["count"]).all()
     shards = [np.load(tmp_path / f"shard{r}.npy") for r in range(world)]
     assert np.concatenate(shards).tolist() == list(range(11)) and abs(len(shards[0]) - len(shards[1])) <= 1
+
+
+def test_one_rank_alone_needs_no_process_group():
+    tok, off = _rank_trajectories(1)
+    got_tok, got_off = replica.gather_trajectories(tok, off, "cpu")
+    assert (got_tok.numpy() == tok).all() and (got_off == off).all()
+    with pytest.raises(ValueError):
+        replica.gather_trajectories(tok[:-1], off, "cpu")
+
+
+def test_kv_head_shards_cover_the_heads():
+    assert [replica.kv_head_shard(8, r, 4) for r in range(4)] == [slice(0, 2), slice(2, 4), slice(4, 6), slice(6, 8)]
+    with pytest.raises(ValueError):
+        replica.kv_head_shard(8, 0, 3)
 
 
 def test_window_eviction_policy():
