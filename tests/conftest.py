@@ -10,6 +10,7 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on a B200)")
+    config.addinivalue_line("markers", "slow: a full-size case that takes about a minute (deselect with -m 'gpu and not slow')")
 
 
 def pytest_collection_modifyitems(config, items):

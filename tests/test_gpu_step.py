@@ -19,14 +19,15 @@ def war():
     return binding
 
 
-def _step(war, cfg, sample, kernel=0):
+def _step(war, cfg, sample, kernel=0, draft_sample=None):
+    """`sample`: requests whose attention is checked; `draft_sample`: requests whose trees are checked (default: the same)."""
     tok, off = W.make_corpus(cfg)
     tails, tl = W.make_request_tails(cfg)
     ctx = W.context_lengths(cfg)
     ix = U.build_index(war, tok, off, cfg.vocab, max_depth=cfg.P + cfg.N)
     ml, nn, ids, par, cnt = U.run_draft(war, ix, tails, tl, cfg.N, cfg.topk)
     corpus = D.Corpus(tok, off)
-    for i in sample:                                                    # brute-force scan per sampled request
+    for i in (sample if draft_sample is None else draft_sample):        # brute-force scan per sampled request
         m, ends = D.longest_suffix_match(corpus, tails[i], int(tl[i]))
         a, b, c = D.build_draft_tree(corpus, tails[i], m, ends, cfg.N, cfg.topk)
         n = len(a)
@@ -69,6 +70,18 @@ def test_full_size_sampled(war, name, sample):
     ctx = W.context_lengths(cfg)
     longest, shortest = int(np.argmax(ctx)), int(np.argmin(ctx))
     ml, nn, alen = _step(war, cfg, sample=sorted(set(sample + [longest, shortest])))
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.slow
+def test_high_workload_every_request(war):
+    """The configuration the metric is quoted on, in full: match lengths, trees and counts of all 256 requests against
+    the brute-force checker, acceptance of all 256 by path enumeration, attention of 32 requests (every eighth, plus
+    the longest and the shortest context) against the fp64 checker."""
+    cfg = W.CONFIGS["high"]
+    ctx = W.context_lengths(cfg)
+    sample = sorted(set(range(0, cfg.B, 8)) | {int(np.argmax(ctx)), int(np.argmin(ctx))})
+    _step(war, cfg, sample=sample, draft_sample=list(range(cfg.B)))
     torch.cuda.empty_cache()
 
 
