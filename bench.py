@@ -265,6 +265,20 @@ class Workload:
         self.index_stats["index_append"] = {"trajectories": k_new, "tokens": int(off[-1] - off[cfg.n_traj - k_new]),
                                             "seconds": time.perf_counter() - t0}
         self.index_stats["index_tokens"] = int(len(tok))
+        # the same amount once more as a stream-ordered update (the oldest trajectories leave first to make room): how
+        # long the host is held (enqueue) and how long the stream is busy with it
+        for _ in range(2):                                     # (the first call grows the allocator's pool; the second is what an engine sees)
+            war.war_index_evict(ix, k_new)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            e0.record()
+            war.war_index_append_async(ix, d_tok, off[:k_new + 1])
+            e1.record()
+            host_s = time.perf_counter() - t0
+            torch.cuda.synchronize()
+        self.index_stats["index_append_async"] = {"trajectories": k_new, "tokens": int(off[k_new]), "host_seconds": host_s,
+                                                  "stream_seconds": 1e-3 * e0.elapsed_time(e1)}
         return ix
 
     def _buffers(self, B):

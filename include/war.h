@@ -69,7 +69,8 @@ typedef struct war_index war_index_t;          /* opaque; lives on the device th
  *                    life of the index, appends included.
  * war_index_append leaves the index answering every query exactly as a fresh build over the old
  * trajectories followed by the new ones would.  Exceeding the capacity returns WAR_ERR_CAPACITY and
- * leaves the index unchanged.  Both calls synchronise `stream` before returning.
+ * leaves the index unchanged.  Both calls synchronise `stream` before returning (war_index_append_async, below,
+ * does not).
  * Updating without blocking the drafts (the paper updates the cache asynchronously so that it does not block
  * the pipeline, Section 3.3): the index keeps two sets of (suffix array, LCP, buckets).  war_index_append builds
  * the new set beside the published one and publishes it just before it returns; the corpus is only written
@@ -89,6 +90,28 @@ war_status_t war_index_build(const int32_t* d_tokens, const int64_t* h_offsets, 
                              war_stream_t stream, war_index_t** out);
 war_status_t war_index_append(war_index_t* ix, const int32_t* d_tokens, const int64_t* h_offsets, int32_t T,
                               war_stream_t stream);
+
+/* war_index_append as a stream-ordered operation (paper Section 3.3: the cache is updated asynchronously, off the
+ * critical path of training): the call only ENQUEUES the update on `stream` and returns; it never synchronises the
+ * host, so one host thread can start the update on a side stream and go on launching steps on its main stream.
+ * The new set of index arrays is built behind the work already in `stream` and published by the last kernel of the
+ * update; a draft kernel that starts after that point answers from the grown index, one that starts earlier from
+ * the old one (either way from a complete index), and the result is the one war_index_append gives.
+ *   - Scratch comes from CUDA's stream-ordered allocator (cudaMallocAsync on `stream`), sized from the token and
+ *     trajectory counts the host knows; the library lets the device's default memory pool keep what it frees.
+ *   - The host-side state of the handle (war_index_info, the capacity check of the next update) advances at once;
+ *     whatever uses the handle next -- another update, war_index_evict, war_index_export, destroying it -- must be
+ *     ordered behind this one: enqueue it on the same stream, or wait for the stream first.  d_tokens must stay
+ *     valid until the update has run; h_offsets may be reused when the call returns.
+ *   - Nobody reads a flag back, so a token id outside [0, vocab) cannot make the call fail: it is stored as an
+ *     end-of-trajectory mark (it matches nothing and nothing continues into it) and WAR_ERR_INVALID_ARG is
+ *     recorded in the device status word.
+ *   - At most 65 535 trajectories per call (WAR_ERR_UNSUPPORTED beyond); capacity as in war_index_append.  If the
+ *     call returns an error, nothing has been published and the handle is as before.
+ * The rule for updates beside running drafts is the one above: the set the drafts read stays intact until the NEXT
+ * update starts. */
+war_status_t war_index_append_async(war_index_t* ix, const int32_t* d_tokens, const int64_t* h_offsets, int32_t T,
+                                    war_stream_t stream);
 
 /* Windowed cache (the paper keeps the cache's memory overhead modest, Section 3.3, without naming a policy; this
  * is the simplest one): removes the n_oldest trajectories that were added first.  Afterwards every query answers

@@ -25,7 +25,7 @@ WAR_OK = 0
 STATUS_NAMES = {0: "WAR_OK", 1: "WAR_ERR_INVALID_ARG", 2: "WAR_ERR_OOM", 3: "WAR_ERR_CAPACITY", 4: "WAR_ERR_CUDA",
                 5: "WAR_ERR_TIMEOUT", 6: "WAR_ERR_UNSUPPORTED", 7: "WAR_ERR_BAD_TREE", 8: "WAR_ERR_BAD_PAGE"}
 
-EXPORTS = ["war_index_build", "war_index_append", "war_index_evict", "war_index_export_bytes", "war_index_export",
+EXPORTS = ["war_index_build", "war_index_append", "war_index_append_async", "war_index_evict", "war_index_export_bytes", "war_index_export",
            "war_index_import", "war_index_info", "war_index_destroy", "war_draft", "war_draft_scored_workspace_bytes", "war_draft_scored", "war_draft_local", "war_draft_pick",
            "war_verify_attn_workspace_bytes", "war_verify_attn", "war_verify_attn_noalloc", "war_accept", "war_commit", "war_device_status",
            "war_selftest_bounded_wait",
@@ -64,6 +64,8 @@ _lib.war_index_build.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C
                                  C.POINTER(C.c_void_p)]
 _lib.war_index_append.restype = C.c_int
 _lib.war_index_append.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+_lib.war_index_append_async.restype = C.c_int
+_lib.war_index_append_async.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
 _lib.war_index_evict.restype = C.c_int
 _lib.war_index_evict.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
 _lib.war_index_export_bytes.restype = C.c_size_t
@@ -165,6 +167,13 @@ def war_index_append(ix: Index, d_tokens: torch.Tensor, h_offsets) -> None:
     off = _offsets(h_offsets)
     _check("war_index_append", _lib.war_index_append(ix.handle, _ptr(d_tokens, torch.int32), off.ctypes.data,
                                                      len(off) - 1, _stream()))
+
+
+def war_index_append_async(ix: Index, d_tokens: torch.Tensor, h_offsets) -> None:
+    """Enqueues the append on the current stream and returns; keep d_tokens alive until that stream has run it."""
+    off = _offsets(h_offsets)
+    _check("war_index_append_async", _lib.war_index_append_async(ix.handle, _ptr(d_tokens, torch.int32), off.ctypes.data,
+                                                                 len(off) - 1, _stream()))
 
 
 def war_index_evict(ix: Index, n_oldest: int) -> None:

@@ -24,7 +24,7 @@ struct MaxOp {
 // A token id outside [0, vocab) raises *bad (such ids would collide with separators or overflow the sort keys).
 __global__ void scatter_corpus_kernel(const int32_t* __restrict__ tokens, const int64_t* __restrict__ off, int T,
                                       int t0, int64_t dst_base, int32_t* __restrict__ corpus, int64_t n_out, int vocab,
-                                      int* __restrict__ bad) {
+                                      int* __restrict__ bad, int* __restrict__ status_word) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_out) return;
     // trajectory t covers output positions [off[t] + t, off[t+1] + t]; the last one is its separator
@@ -39,7 +39,12 @@ __global__ void scatter_corpus_kernel(const int32_t* __restrict__ tokens, const 
     int32_t v = -(t0 + t + 1);
     if (local < len) {
         v = tokens[off[t] + local];
-        if (v < 0 || v >= vocab) *bad = 1;
+        if (v < 0 || v >= vocab) {
+            if (bad) *bad = 1;
+            // stream-ordered append: nobody reads a flag back, so the token becomes an end-of-trajectory mark (it
+            // matches nothing and nothing continues into it) and the problem goes to the device status word
+            if (status_word) { war_set_device_status(status_word, WAR_ERR_INVALID_ARG); v = -(t0 + t + 1); }
+        }
     }
     corpus[dst_base + i] = v;
 }
@@ -365,7 +370,7 @@ war_status_t add_trajectories(war_index* ix, const int32_t* d_tokens, const int6
     if (e == cudaSuccess) e = cudaMemsetAsync(d_bad, 0, sizeof(int), s);
     if (e == cudaSuccess) {
         scatter_corpus_kernel<<<grid_for(n_out), kThreads, 0, s>>>(d_tokens + h_offsets[0], (const int64_t*)off.p, T, ix->T,
-                                                                  ix->M, ix->corpus, n_out, ix->vocab, d_bad);
+                                                                  ix->M, ix->corpus, n_out, ix->vocab, d_bad, nullptr);
         e = cudaGetLastError();
     }
     if (e == cudaSuccess) e = cudaMemcpyAsync(&bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost, s);
@@ -440,7 +445,208 @@ war_status_t evict_oldest(war_index* ix, int32_t n, cudaStream_t s) {
     return finish_index(ix, s);
 }
 
+// ---- stream-ordered append ----------------------------------------------------------------------------
+// The same result as war_index_append, enqueued on the caller's stream without a single host synchronisation: scratch
+// comes from the stream-ordered allocator, sized from what the host knows (token and trajectory counts); the prefix
+// doubling runs its fixed number of rounds over all new suffixes instead of shrinking the active set by counts read
+// back from the device; the publication is a one-word kernel behind everything that built the set.
+
+__global__ void set_u32_kernel(unsigned int* p, unsigned int v) { *p = v; }
+
+__global__ void full_keys_kernel(const int32_t* __restrict__ sa, const uint32_t* __restrict__ rank, int64_t n, int64_t h,
+                                 uint64_t* __restrict__ key, int32_t* __restrict__ val) {
+    const int64_t a = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (a >= n) return;
+    const int64_t s = sa[a];
+    const uint64_t hi = rank[s];
+    const uint64_t lo = (s + h < n) ? (uint64_t)rank[s + h] + 1u : 0u;
+    key[a] = (hi << 32) | lo;
+    val[a] = (int32_t)s;
+}
+
+// head[a] = a if slot a starts a new group, else 0 (the inclusive max scan turns it into the group's first slot)
+__global__ void full_heads_kernel(const uint64_t* __restrict__ key, int64_t n, uint32_t* __restrict__ head) {
+    const int64_t a = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (a >= n) return;
+    head[a] = (a > 0 && key[a] != key[a - 1]) ? (uint32_t)a : 0u;
+}
+
+size_t sort_full_scratch_bytes(int64_t n64, size_t* temp_bytes_out) {
+    const int n = (int)n64;
+    size_t t_sort64 = 0, t_sort32 = 0, t_scan = 0;
+    cub::DoubleBuffer<uint64_t> k64(nullptr, nullptr);
+    cub::DoubleBuffer<uint32_t> k32(nullptr, nullptr);
+    cub::DoubleBuffer<int32_t> v(nullptr, nullptr);
+    cub::DeviceRadixSort::SortPairs(nullptr, t_sort64, k64, v, n, 0, 64, (cudaStream_t)0);
+    cub::DeviceRadixSort::SortPairs(nullptr, t_sort32, k32, v, n, 0, 32, (cudaStream_t)0);
+    cub::DeviceScan::InclusiveScan(nullptr, t_scan, (uint32_t*)nullptr, (uint32_t*)nullptr, MaxOp(), n, (cudaStream_t)0);
+    size_t temp = t_sort64 > t_sort32 ? t_sort64 : t_sort32;
+    if (t_scan > temp) temp = t_scan;
+    auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    *temp_bytes_out = align(temp);
+    return 2 * align(sizeof(uint64_t) * n64) + 4 * align(sizeof(int32_t) * n64) + align(temp);
+}
+
+// sort_suffixes without host round trips: every round sorts all n (rank, rank at +h) keys.  `scratch` holds
+// sort_full_scratch_bytes(n) bytes.  Ties beyond max_depth keep the order of the start positions, as in sort_suffixes.
+war_status_t sort_suffixes_full(const int32_t* corpus, int64_t n64, int T_total, int vocab, int max_depth, int32_t* out_sa,
+                                void* scratch, cudaStream_t s) {
+    const int n = (int)n64;
+    size_t temp_bytes = 0;
+    (void)sort_full_scratch_bytes(n64, &temp_bytes);
+    auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t b_key = align(sizeof(uint64_t) * n64), b_i32 = align(sizeof(int32_t) * n64);
+    char* at = (char*)scratch;
+    uint64_t* key_a = (uint64_t*)at; at += b_key;
+    uint64_t* key_b = (uint64_t*)at; at += b_key;
+    int32_t* val_a = (int32_t*)at; at += b_i32;
+    int32_t* val_b = (int32_t*)at; at += b_i32;
+    uint32_t* rank = (uint32_t*)at; at += b_i32;
+    uint32_t* head = (uint32_t*)at; at += b_i32;
+    void* temp = at;
+    int sym_bits = 1;
+    while (((int64_t)1 << sym_bits) < (int64_t)vocab + T_total) ++sym_bits;
+    int pos_bits = 1;
+    while (((int64_t)1 << pos_bits) < n64 + 1) ++pos_bits;
+    {
+        cub::DoubleBuffer<uint32_t> k32((uint32_t*)key_a, (uint32_t*)key_b);
+        cub::DoubleBuffer<int32_t> val(val_a, val_b);
+        init_keys_kernel<<<grid_for(n64), kThreads, 0, s>>>(corpus, n64, T_total, k32.Current(), val.Current());
+        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(temp, temp_bytes, k32, val, n, 0, sym_bits, s));
+        WAR_CUDA_TRY(cudaMemcpyAsync(out_sa, val.Current(), sizeof(int32_t) * n64, cudaMemcpyDeviceToDevice, s));
+        flag32_kernel<<<grid_for(n64), kThreads, 0, s>>>(k32.Current(), n64, head);
+        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, head, head, MaxOp(), n, s));
+        scatter_rank_kernel<<<grid_for(n64), kThreads, 0, s>>>(out_sa, head, n64, rank);
+    }
+    for (int64_t h = 1; h < max_depth; h <<= 1) {
+        cub::DoubleBuffer<uint64_t> k64(key_a, key_b);
+        cub::DoubleBuffer<int32_t> val(val_a, val_b);
+        full_keys_kernel<<<grid_for(n64), kThreads, 0, s>>>(out_sa, rank, n64, h, k64.Current(), val.Current());
+        WAR_CUDA_TRY(cub::DeviceRadixSort::SortPairs(temp, temp_bytes, k64, val, n, 0, 32 + pos_bits, s));
+        WAR_CUDA_TRY(cudaMemcpyAsync(out_sa, val.Current(), sizeof(int32_t) * n64, cudaMemcpyDeviceToDevice, s));
+        full_heads_kernel<<<grid_for(n64), kThreads, 0, s>>>(k64.Current(), n64, head);
+        WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, temp_bytes, head, head, MaxOp(), n, s));
+        scatter_rank_kernel<<<grid_for(n64), kThreads, 0, s>>>(out_sa, head, n64, rank);
+    }
+    WAR_LAUNCH_CHECK();
+    return WAR_OK;
+}
+
+struct AsyncScratch {
+    void* p = nullptr;
+    cudaStream_t s = nullptr;
+    ~AsyncScratch() { if (p) cudaFreeAsync(p, s); }
+};
+
+// Memory freed to the stream-ordered allocator stays in its pool, so that the next update finds it without a trip to
+// the driver (once per device).
+void keep_pool_memory(int device) {
+    static std::once_flag once[64];
+    if (device < 0 || device >= 64) return;
+    std::call_once(once[device], [device]() {
+        cudaMemPool_t pool;
+        if (cudaDeviceGetDefaultMemPool(&pool, device) == cudaSuccess) {
+            unsigned long long keep = ~0ull;
+            cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+        }
+        (void)cudaGetLastError();
+    });
+}
+
+war_status_t append_async(war_index* ix, const int32_t* d_tokens, const int64_t* h_offsets, int32_t T, cudaStream_t s) {
+    const int64_t n_tok = h_offsets[T] - h_offsets[0];
+    const int64_t m = n_tok + T, M_old = ix->M, M = M_old + m;
+    const int32_t T_old = ix->T;
+    if (M > ix->capacity || M >= ((int64_t)1 << 31) - 256 || (int64_t)T_old + T >= ((int64_t)1 << 30)) return WAR_ERR_CAPACITY;
+    if (n_tok > 0 && !d_tokens) return WAR_ERR_INVALID_ARG;
+    if ((size_t)T + 1 > war_index::kStageEntries) return WAR_ERR_UNSUPPORTED;
+    int* status_word = war_status_word();
+    if (!status_word) return WAR_ERR_CUDA;
+    keep_pool_memory(ix->device);
+    const bool merge = M_old > 0 && m < M_old;
+    // ---- scratch, one stream-ordered allocation ----
+    auto align = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const int64_t n_sort = merge ? m : M;
+    size_t sort_temp = 0, temp_scan = 0, temp_scan2 = 0;
+    const size_t b_sort = sort_full_scratch_bytes(n_sort, &sort_temp);
+    WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(nullptr, temp_scan, (uint32_t*)nullptr, (uint32_t*)nullptr, MaxOp(), (int)m, s));
+    WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(nullptr, temp_scan2, (uint32_t*)nullptr, (uint32_t*)nullptr, SumOp(), (int)(M_old + 1), s));
+    size_t b_scan = align(temp_scan > temp_scan2 ? temp_scan : temp_scan2);
+    const size_t b_off = align(sizeof(int64_t) * ((size_t)T + 1)), b_new = align(sizeof(int32_t) * m), b_pos = align(sizeof(uint32_t) * m),
+                 b_add = align(sizeof(uint32_t) * (M_old + 1));
+    AsyncScratch scratch;
+    scratch.s = s;
+    WAR_CUDA_TRY(cudaMallocAsync(&scratch.p, b_off + b_sort + (merge ? b_new + b_pos + b_add + b_scan : 0), s));
+    char* at = (char*)scratch.p;
+    int64_t* d_off = (int64_t*)at; at += b_off;
+    void* sort_scratch = at; at += b_sort;
+    int32_t* new_sa = (int32_t*)at; at += merge ? b_new : 0;
+    uint32_t* pos = (uint32_t*)at; at += merge ? b_pos : 0;
+    uint32_t* add = (uint32_t*)at; at += merge ? b_add : 0;
+    void* scan_temp = at;
+    // ---- the trajectories' bounds go through pinned staging memory (its previous use has long been consumed) ----
+    WAR_CUDA_TRY(cudaEventSynchronize(ix->stage_free));
+    for (int t = 0; t <= T; ++t) ix->h_stage[t] = h_offsets[t] - h_offsets[0];
+    WAR_CUDA_TRY(cudaMemcpyAsync(d_off, ix->h_stage, sizeof(int64_t) * ((size_t)T + 1), cudaMemcpyHostToDevice, s));
+    WAR_CUDA_TRY(cudaEventRecord(ix->stage_free, s));
+    scatter_corpus_kernel<<<grid_for(m), kThreads, 0, s>>>(d_tokens + h_offsets[0], d_off, T, T_old, M_old, ix->corpus, m, ix->vocab,
+                                                          nullptr, status_word);
+    WAR_LAUNCH_CHECK();
+    // ---- host bookkeeping as of this point of the stream (undone below if anything fails to enqueue) ----
+    try {
+        for (int t = 1; t <= T; ++t) ix->bounds.push_back(M_old + (h_offsets[t] - h_offsets[0]) + t);
+    } catch (...) {
+        ix->bounds.resize((size_t)T_old + 1);
+        return WAR_ERR_OOM;
+    }
+    ix->M = M;
+    ix->T = T_old + T;
+    const war_index_arrays old = ix->published();
+    war_index_arrays& sh = ix->shadow();
+    auto enqueue = [&]() -> war_status_t {
+        if (merge) {
+            const war_status_t st = sort_suffixes_full(ix->corpus + M_old, m, ix->T, ix->vocab, ix->max_depth, new_sa, sort_scratch, s);
+            if (st != WAR_OK) return st;
+            insert_pos_kernel<<<grid_for(m), kThreads, 0, s>>>(ix->corpus, old.sa, old.bucket, new_sa, m, M_old, ix->vocab, ix->max_depth, pos);
+            WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(scan_temp, b_scan, pos, pos, MaxOp(), (int)m, s));
+            WAR_CUDA_TRY(cudaMemsetAsync(add, 0, b_add, s));
+            count_pos_kernel<<<grid_for(m), kThreads, 0, s>>>(pos, m, add);
+            WAR_CUDA_TRY(cub::DeviceScan::InclusiveScan(scan_temp, b_scan, add, add, SumOp(), (int)(M_old + 1), s));
+            scatter_old_kernel<<<grid_for(M_old), kThreads, 0, s>>>(old.sa, add, M_old, sh.sa);
+            scatter_new_kernel<<<grid_for(m), kThreads, 0, s>>>(new_sa, pos, m, M_old, sh.sa);
+        } else {
+            const war_status_t st = sort_suffixes_full(ix->corpus, M, ix->T, ix->vocab, ix->max_depth, sh.sa, sort_scratch, s);
+            if (st != WAR_OK) return st;
+        }
+        lcp_kernel<<<grid_for(M), kThreads, 0, s>>>(ix->corpus, sh.sa, M, ix->max_depth, sh.lcp);
+        bucket_from_sa_kernel<<<grid_for(M + 1), kThreads, 0, s>>>(ix->corpus, sh.sa, M, ix->vocab, sh.bucket);
+        WAR_LAUNCH_CHECK();
+        WAR_CUDA_TRY(cudaMemsetAsync(sh.memo, 0, sizeof(int32_t) * kMemoEntries * kMemoInts, s));
+        set_u32_kernel<<<1, 1, 0, s>>>(&ix->d_view->cur, (unsigned int)(ix->cur ^ 1));
+        WAR_LAUNCH_CHECK();
+        return WAR_OK;
+    };
+    const war_status_t st = enqueue();
+    if (st != WAR_OK) {                                      // nothing was published: forget the addition
+        ix->M = M_old;
+        ix->T = T_old;
+        ix->bounds.resize((size_t)T_old + 1);
+        return st;
+    }
+    { std::lock_guard<std::mutex> g(ix->lock); ix->cur ^= 1; }
+    return WAR_OK;
+}
+
 }  // namespace
+
+extern "C" war_status_t war_index_append_async(war_index_t* ix, const int32_t* d_tokens, const int64_t* h_offsets, int32_t T,
+                                               war_stream_t stream) {
+    if (!ix) return WAR_ERR_INVALID_ARG;
+    const war_status_t st = check_offsets(h_offsets, T);
+    if (st != WAR_OK) return st;
+    if (T == 0) return WAR_OK;
+    return append_async(ix, d_tokens, h_offsets, T, stream);
+}
 
 extern "C" war_status_t war_index_build(const int32_t* d_tokens, const int64_t* h_offsets, int32_t T, int32_t vocab,
                                         int32_t max_depth, int64_t capacity_tokens, war_stream_t stream,
@@ -470,6 +676,8 @@ extern "C" war_status_t war_index_build(const int32_t* d_tokens, const int64_t* 
     }
     if (e == cudaSuccess) e = cudaMemsetAsync(ix->corpus, 0xff, sizeof(int32_t) * (cap + 128), stream);
     if (e == cudaSuccess) e = cudaMalloc((void**)&ix->d_view, sizeof(war_index_view));
+    if (e == cudaSuccess) e = cudaMallocHost((void**)&ix->h_stage, sizeof(int64_t) * war_index::kStageEntries);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ix->stage_free, cudaEventDisableTiming);
     if (e == cudaSuccess) {
         war_index_view v;
         v.set[0] = ix->set[0]; v.set[1] = ix->set[1]; v.cur = (unsigned int)ix->cur;
@@ -617,6 +825,8 @@ extern "C" war_status_t war_index_destroy(war_index_t* ix) {
     if (!ix) return WAR_OK;
     if (ix->corpus) cudaFree(ix->corpus);
     if (ix->d_view) cudaFree(ix->d_view);
+    if (ix->h_stage) cudaFreeHost(ix->h_stage);
+    if (ix->stage_free) cudaEventDestroy(ix->stage_free);
     for (int k = 0; k < 2; ++k) {
         if (ix->set[k].sa) cudaFree(ix->set[k].sa);
         if (ix->set[k].lcp) cudaFree(ix->set[k].lcp);

@@ -34,6 +34,10 @@ struct war_index {
     int32_t* corpus = nullptr;   // [capacity + slack] trajectories joined by unique negative separators
     war_index_arrays set[2];
     war_index_view* d_view = nullptr;   // device copy of (set, cur)
+    // stream-ordered append: pinned staging memory for a batch's trajectory bounds, and the event after which it is free again
+    static constexpr size_t kStageEntries = 1 << 16;
+    int64_t* h_stage = nullptr;
+    cudaEvent_t stage_free = nullptr;
     int cur = 0;                 // published set (host copy); guarded by `lock` together with the pointers handed to queries
     std::mutex lock;
     int64_t M = 0;               // corpus entries in use

@@ -404,6 +404,84 @@ def test_drafts_keep_running_while_the_index_is_updated(war):
     ix.destroy()
 
 
+def test_stream_ordered_append_from_one_thread(war):
+    """war_index_append_async only enqueues the update: ONE host thread starts it on a side stream and goes on
+    drafting on its main stream.  Every draft enqueued meanwhile equals the checker's answer on the corpus before or
+    after the update (never anything else), drafts ordered behind the update see the grown corpus, two updates
+    enqueued back to back on one stream land in order, a full re-sort (the addition larger than what is stored) and a
+    merge both come out as a fresh build would, and a token outside the vocabulary becomes an end-of-trajectory mark
+    with WAR_ERR_INVALID_ARG in the device status."""
+    cfg = W.CONFIGS["tiny"]
+    tok, off = W.make_corpus(cfg)
+    tails, tl = W.make_request_tails(W.scaled(cfg, B=32))
+    T = cfg.n_traj
+    cuts = [6, 20, 44, T]                                             # 6 -> 20 is a full re-sort, the others merge
+    dev = U.dev()
+    d_tok = torch.from_numpy(tok).to(dev)
+    N, k = cfg.N, cfg.topk
+    ix = U.build_index(war, tok[:off[cuts[0]]], off[:cuts[0] + 1], cfg.vocab, max_depth=cfg.P + N, capacity=len(tok) + T + 64)
+    wants = [D.draft_batch(D.Corpus(tok[:off[c]], off[:c + 1]), tails, tl, N, k) for c in cuts]
+    same = lambda got, want: all(np.array_equal(g, w) for g, w in zip(got, want))
+    side = torch.cuda.Stream()
+    main = torch.cuda.current_stream()
+    i32 = dict(dtype=torch.int32, device=dev)
+    d_tails, d_tl = torch.from_numpy(tails).to(dev), torch.from_numpy(tl).to(dev)
+
+    def enqueue_draft():
+        bufs = [torch.full((32,), -7, **i32), torch.full((32,), -7, **i32)] + [torch.full((32, N), -7, **i32) for _ in range(3)]
+        war.war_draft(ix, d_tails, d_tl, N, k, 1, *bufs)
+        return bufs
+
+    for step in range(1, 4):
+        side.wait_stream(main)
+        with torch.cuda.stream(side):
+            war.war_index_append_async(ix, d_tok[off[cuts[step - 1]]:off[cuts[step]]], off[cuts[step - 1]:cuts[step] + 1] - off[cuts[step - 1]])
+        assert war.war_index_info(ix).T == cuts[step]                 # the handle's host side has advanced already
+        during = [enqueue_draft() for _ in range(6)]                  # not ordered against the update: old or new
+        main.wait_stream(side)
+        after = enqueue_draft()                                       # ordered behind it: new
+        torch.cuda.synchronize()
+        for bufs in during:
+            got = [b.cpu().numpy() for b in bufs]
+            assert same(got, wants[step - 1]) or same(got, wants[step])
+        assert same([b.cpu().numpy() for b in after], wants[step])
+    # the arrays themselves equal a fresh build's up to the order of suffixes that agree to the full depth: compare lcp and buckets
+    info = war.war_index_info(ix)
+    fresh = U.build_index(war, tok, off, cfg.vocab, max_depth=cfg.P + N)
+    f_info = war.war_index_info(fresh)
+    M = int(info.M)
+    assert M == int(f_info.M)
+    torch.cuda.synchronize()
+    lcp_a = _read_device(info.d_lcp, M); lcp_b = _read_device(f_info.d_lcp, M)
+    assert np.array_equal(lcp_a, lcp_b)
+    fresh.destroy()
+    # two updates back to back on one stream, then an eviction ordered behind them
+    ix2 = U.build_index(war, tok[:off[30]], off[:31], cfg.vocab, max_depth=cfg.P + N, capacity=len(tok) + T + 64)
+    with torch.cuda.stream(side):
+        war.war_index_append_async(ix2, d_tok[off[30]:off[40]], off[30:41] - off[30])
+        war.war_index_append_async(ix2, d_tok[off[40]:off[T]], off[40:T + 1] - off[40])
+        war.war_index_evict(ix2, 7)                                   # (synchronises the side stream itself)
+    got = U.run_draft(war, ix2, tails, tl, N, k)
+    want = D.draft_batch(D.Corpus(tok[off[7]:], off[7:] - off[7]), tails, tl, N, k)
+    assert same(got, want)
+    assert war.war_device_status() == 0
+    # a token outside the vocabulary: recorded, stored as an end-of-trajectory mark
+    bad = np.array([5, 9, cfg.vocab + 3, 9, 5, 9], np.int32)
+    with torch.cuda.stream(side):
+        war.war_index_append_async(ix2, torch.from_numpy(bad).to(dev), np.array([0, 6], np.int64))
+    side.synchronize()
+    assert war.war_device_status() == 1                               # WAR_ERR_INVALID_ARG
+    hist_tok = np.concatenate([tok[off[7]:], bad[:2], bad[3:]])
+    hist_off = np.concatenate([off[7:] - off[7], [off[T] - off[7] + 2, off[T] - off[7] + 5]])
+    got = U.run_draft(war, ix2, tails, tl, N, k)
+    want = D.draft_batch(D.Corpus(hist_tok, hist_off), tails, tl, N, k)
+    assert same(got, want)
+    with pytest.raises(war.WarError) as e:                            # over capacity: refused, nothing enqueued
+        war.war_index_append_async(ix2, d_tok, off)
+    assert e.value.code == 3
+    ix.destroy(); ix2.destroy()
+
+
 def test_memo_of_node_expansions_never_changes_an_answer(war):
     """The index caches the expansions of large nodes.  Same answers on an empty and on a filled memo, for different
     k on the same nodes, and after an append (which must drop the entries of the old suffix array)."""
