@@ -36,7 +36,7 @@ struct FusedPlan {                        // resident in shared memory for the w
     int mode;                             // 0 snake deal, 1 contiguous split
     int total;                            // snake deal: number of units
     int t_all, n_used;                    // contiguous split: tiles in the sequence, CTAs that get a range,
-    int cut_base, cut_rem;                //   t_all / n_used and t_all % n_used
+    int c0_first, c1_last;                //   the CTA where this CTA's first pair begins / where its last pair ends
     int lo, hi, r0, h0;                   // contiguous split: this CTA's range and the pair that holds its first tile
 };
 static_assert(sizeof(FusedPlan) <= 704, "the plan table shares 768 bytes of shared memory");
@@ -45,6 +45,8 @@ struct FusedPlanScratch {                 // only while the plan is made (lives 
     int keys[64];
     int weight[kFusedMaxB];               // units per chunk of a request: kv heads x row blocks (0: no work)
     int units_by_pos[kFusedMaxB];
+    int live_before[kFusedMaxB + 1];      // contiguous split: live requests before each request
+    int cut[kFusedMaxCtas + 2];           // contiguous split: first tile of every CTA's range
 };
 
 // Host-side rule for taking this path: few requests, and unit offsets that fit 16 bits (the snake deal creates at
@@ -133,16 +135,41 @@ __device__ __forceinline__ int chunk_search(const int* tiles, const int* weight,
 // unit wherever a pair ends inside it.  Measured on 4 to 64 requests of three recipes it wins from about 48 tiles per
 // CTA on (one row block per kv head); below that the searched chunk length does better.
 __host__ __device__ __forceinline__ bool contiguous_split_pays(int rows_max, long long t_all, int n_ctas) {
-    return rows_max <= kRowBlock && t_all >= 48ll * n_ctas && t_all < (1ll << 31);
+    return rows_max <= kRowBlock && t_all >= 48ll * n_ctas && t_all < (1ll << 30);
 }
 
 constexpr int kFusedMaxChunks = 192;      // chunks per request at most (what the merge of a row group can hold at once)
 __device__ __forceinline__ int chunk_floor(int t_max) { return max(4, (t_max + kFusedMaxChunks - 1) / kFusedMaxChunks); }
 
-// contiguous split: first tile of CTA c's range = floor(t_all * c / n_used), in 32-bit arithmetic
-// (t_all = cut_base * n_used + cut_rem, cut_rem * c < 2^20)
-__device__ __forceinline__ int cut_at(const FusedPlan* pl, int c) {
-    return pl->cut_base * c + (int)((unsigned)(pl->cut_rem * c) / (unsigned)pl->n_used);
+// Contiguous split with the cost of a unit in it.  A CTA pays for every unit it runs about as much as for
+// `unit_cost` tiles (its pipeline drains and fills again: epilogue, next Q tile, first loads; measured 12 to 21 us per
+// extra unit against 1.3 us per tile, more with more query rows), so equal TILE counts leave the CTAs that hold many
+// short pairs behind (finish times followed the unit count with correlation 0.9 to 0.99).  The sequence that is cut
+// into equal ranges therefore gives every pair `unit_cost` virtual tiles in front of its real ones; a cut that falls
+// among a pair's virtual tiles moves to the pair's first real tile.
+__host__ __device__ __forceinline__ int contiguous_unit_cost(int rows_max) { return 8 + rows_max / 16; }
+
+// First real tile (index in the sequence of all pairs' real tiles) of CTA x's range, x in [0, n_used].
+// start[r]: first real tile of request r's pairs; live_before[r]: live requests before r; weight[r] > 0: r is live.
+__device__ __forceinline__ int contiguous_cut(int x, int n_used, int t_all, int pairs, int unit_cost, const int* tiles,
+                                              const int* weight, const int* start, const int* live_before, int B, int Hkv) {
+    if (x >= n_used) return t_all;
+    // position in the weighted sequence, floor(w_all * x / n_used), in 32-bit arithmetic (w_all < 2^31, x < 2^10)
+    const unsigned w_all = (unsigned)t_all + (unsigned)(pairs * unit_cost);
+    const unsigned base = w_all / (unsigned)n_used, rem = w_all - base * (unsigned)n_used;
+    const unsigned p = base * (unsigned)x + rem * (unsigned)x / (unsigned)n_used;
+    // the request whose pairs hold weighted position p: the last live one that starts at or before it
+    int r = -1;
+#pragma unroll 1
+    for (int q = 0; q < B; ++q)
+        if (weight[q] > 0 && (unsigned)(start[q] + live_before[q] * Hkv * unit_cost) <= p) r = q;
+    if (r < 0) return 0;
+    const unsigned off = p - (unsigned)(start[r] + live_before[r] * Hkv * unit_cost);
+    const unsigned w = (unsigned)(tiles[r] + unit_cost);
+    const int h = (int)(off / w);
+    if (h >= Hkv) return start[r] + Hkv * tiles[r];              // (cannot happen: the next live request starts there)
+    const int o = (int)(off - (unsigned)h * w);
+    return start[r] + h * tiles[r] + max(0, o - unit_cost);
 }
 
 __device__ __forceinline__ void cursor_init(const FusedPlan* pl, Cursor& c) { c.k = 0; c.r = pl->r0; c.h = pl->h0; }
@@ -181,13 +208,8 @@ __device__ __forceinline__ bool next_unit(const FusedPlan* pl, Cursor& c, int B,
     const int t = pl->tiles[c.r];
     const int ps = pl->u.start[c.r] + c.h * t;
     if (ps >= hi) return false;
-    auto cta_of = [&](int x) -> int {                 // the CTA whose range [cut(c), cut(c+1)) holds tile x
-        int cc = min(pl->n_used - 1, (int)((unsigned)x / (unsigned)max(1, pl->cut_base)));
-        while (cc + 1 < pl->n_used && cut_at(pl, cc + 1) <= x) ++cc;
-        while (cc > 0 && cut_at(pl, cc) > x) --cc;
-        return cc;
-    };
-    const int c0 = ps >= lo ? cta : cta_of(ps), c1 = ps + t <= hi ? cta : cta_of(ps + t - 1);
+    // only a CTA's first unit can have begun in an earlier CTA, only its last one can go on into a later one
+    const int c0 = ps >= lo ? cta : pl->c0_first, c1 = ps + t <= hi ? cta : pl->c1_last;
     un.req = c.r; un.kvh = c.h; un.rb = 0; un.n_nodes = pl->n[c.r];
     un.tile_begin = max(lo, ps) - ps; un.tile_end = min(hi, ps + t) - ps;
     un.n_chunks = c1 - c0 + 1; un.chunk = cta - c0;
@@ -245,36 +267,61 @@ __device__ __noinline__ static void make(const int32_t* __restrict__ prefix_len,
     const bool contiguous = contiguous_split_pays(rows_max, t_all_ll, n_ctas);
 
     if (contiguous) {
-        // The tiles of all (request, kv head) pairs form one sequence; CTA c takes [cut(c), cut(c+1)), cut(c) = t_all * c / n_used.
+        // The tiles of all (request, kv head) pairs form one sequence; CTA c takes [cut(c), cut(c+1)) (contiguous_cut).
         if (warp == 0) {
             const int a0 = 2 * lane, a1 = 2 * lane + 1;
-            const int m0 = sc->weight[a0] > 0 ? pl->tiles[a0] * Hkv : 0, m1 = sc->weight[a1] > 0 ? pl->tiles[a1] * Hkv : 0;
-            int incl = m0 + m1;
+            const int l0 = sc->weight[a0] > 0, l1 = sc->weight[a1] > 0;
+            const int m0 = l0 ? pl->tiles[a0] * Hkv : 0, m1 = l1 ? pl->tiles[a1] * Hkv : 0;
+            int incl = m0 + m1, live = l0 + l1;
 #pragma unroll 1
-            for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+            for (int o = 1; o < 32; o <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, incl, o), z = __shfl_up_sync(0xffffffffu, live, o);
+                if (lane >= o) { incl += y; live += z; }
+            }
             pl->u.start[a0] = incl - m0 - m1;
             pl->u.start[a1] = incl - m1;
-            if (lane == 31) pl->u.start[64] = incl;
-            __syncwarp();
-            const int t_all = __shfl_sync(0xffffffffu, incl, 31);
-            const int n_used = min(n_ctas, max(1, t_all / 4));
-            if (lane == 0) {
-                pl->mode = 1; pl->total = 0; pl->t_all = t_all; pl->n_used = n_used;
-                pl->cut_base = (int)((unsigned)t_all / (unsigned)n_used); pl->cut_rem = t_all - pl->cut_base * n_used;
+            sc->live_before[a0] = live - l0 - l1;
+            sc->live_before[a1] = live - l1;
+            if (lane == 31) {
+                pl->u.start[64] = incl;
+                pl->mode = 1; pl->total = 0; pl->t_all = incl; pl->n_used = min(n_ctas, max(1, incl / 4));
             }
-            __syncwarp();
-            // this CTA's range and the pair that holds its first tile (lanes look at requests lane and lane + 32)
+        }
+        __syncthreads();
+        const int t_all = pl->t_all, n_used = pl->n_used;
+        const int unit_cost = contiguous_unit_cost(rows_max);
+        for (int x = tid; x <= n_used; x += kFusedThreads)
+            sc->cut[x] = contiguous_cut(x, n_used, t_all, pairs, unit_cost, pl->tiles, sc->weight, pl->u.start, sc->live_before, B, Hkv);
+        __syncthreads();
+        if (warp == 0) {
+            // this CTA's range, the pair that holds its first tile (lanes look at requests lane and lane + 32), and the
+            // CTAs where its first pair begins and its last pair ends (lanes look at cuts lane, lane + 32, ...)
             int lo = 0, hi = 0;
-            if (cta < n_used) { lo = cut_at(pl, cta); hi = cut_at(pl, cta + 1); }
+            if (cta < n_used) { lo = sc->cut[cta]; hi = sc->cut[cta + 1]; }
             int best = -1;
             for (int q = lane; q < B; q += 32)
                 if (sc->weight[q] > 0 && pl->u.start[q] <= lo) best = max(best, q);
             best = __reduce_max_sync(0xffffffffu, best);
-            if (lane == 0) {
-                pl->lo = lo; pl->hi = hi;
-                if (hi > lo && best >= 0) { pl->r0 = best; pl->h0 = (int)((unsigned)(lo - pl->u.start[best]) / (unsigned)pl->tiles[best]); }
-                else { pl->r0 = B; pl->h0 = 0; }
+            int r0 = B, h0 = 0, c0_first = cta, c1_last = cta;
+            if (hi > lo && best >= 0) {
+                r0 = best; h0 = (int)((unsigned)(lo - pl->u.start[best]) / (unsigned)pl->tiles[best]);
+                const int ps0 = pl->u.start[r0] + h0 * pl->tiles[r0];        // first tile of the pair that holds lo
+                int last = -1;                                               // the pair that holds hi - 1, and its last tile
+                for (int q = lane; q < B; q += 32)
+                    if (sc->weight[q] > 0 && pl->u.start[q] <= hi - 1) last = max(last, q);
+                last = __reduce_max_sync(0xffffffffu, last);
+                const int hl = (int)((unsigned)(hi - 1 - pl->u.start[last]) / (unsigned)pl->tiles[last]);
+                const int pe = pl->u.start[last] + (hl + 1) * pl->tiles[last] - 1;
+                // the CTA whose non-empty range holds a tile: the largest x with cut[x] <= tile and cut[x + 1] > tile
+                int f = -1, l = -1;
+                for (int x = lane; x < n_used; x += 32) {
+                    if (sc->cut[x] <= ps0 && sc->cut[x + 1] > ps0) f = x;
+                    if (sc->cut[x] <= pe && sc->cut[x + 1] > pe) l = x;
+                }
+                c0_first = __reduce_max_sync(0xffffffffu, f);
+                c1_last = __reduce_max_sync(0xffffffffu, l);
             }
+            if (lane == 0) { pl->lo = lo; pl->hi = hi; pl->r0 = r0; pl->h0 = h0; pl->c0_first = c0_first; pl->c1_last = c1_last; }
         }
         __syncthreads();
         return;
@@ -308,7 +355,7 @@ __device__ __noinline__ static void make(const int32_t* __restrict__ prefix_len,
         for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
         pl->u.s.pos_base[a0] = (uint16_t)(incl - m0 - m1);
         pl->u.s.pos_base[a1] = (uint16_t)(incl - m1);
-        if (lane == 31) { pl->mode = 0; pl->total = incl; pl->r0 = 0; pl->h0 = 0; pl->lo = 0; pl->hi = 0; pl->t_all = 0; pl->n_used = 0; }
+        if (lane == 31) { pl->mode = 0; pl->total = incl; pl->r0 = 0; pl->h0 = 0; pl->lo = 0; pl->hi = 0; pl->t_all = 0; pl->n_used = 0; pl->c0_first = 0; pl->c1_last = 0; }
     }
     __syncthreads();
 }

@@ -25,30 +25,41 @@ __device__ __forceinline__ uint64_t shfl64(uint64_t v, int src) {
 // (the caller checked that the sequence has fewer than 2^31 tiles) and the cuts are worked out once, one 64-bit division
 // per CTA in parallel: everything after that is additions, comparisons and 32-bit divisions.
 __device__ __noinline__ void plan_contiguous(const int* s_tiles, const uint8_t* s_n, int* s_start, int* s_cnt, int* s_cut, int B,
-                                             int Hkv, int n_ctas, AttnWorkspace w) {
+                                             int Hkv, int n_ctas, int rows_max, int pairs, AttnWorkspace w) {
+    __shared__ int s_live_before[65], s_weight[64];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (warp == 0) {                                             // first tile of every request's pairs in the sequence
         const int q0 = 2 * lane, q1 = 2 * lane + 1;              // two requests per lane: B <= 64
-        const int m0 = q0 < B && s_n[q0] > 0 ? s_tiles[q0] * Hkv : 0, m1 = q1 < B && s_n[q1] > 0 ? s_tiles[q1] * Hkv : 0;
-        int incl = m0 + m1;
+        const int l0 = q0 < B && s_n[q0] > 0 && s_tiles[q0] > 0, l1 = q1 < B && s_n[q1] > 0 && s_tiles[q1] > 0;
+        const int m0 = l0 ? s_tiles[q0] * Hkv : 0, m1 = l1 ? s_tiles[q1] * Hkv : 0;
+        int incl = m0 + m1, live = l0 + l1;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, incl, o), z = __shfl_up_sync(0xffffffffu, live, o);
+            if (lane >= o) { incl += y; live += z; }
+        }
         s_start[q0] = incl - m0 - m1;
         s_start[q1] = incl - m1;
+        s_live_before[q0] = live - l0 - l1;
+        s_live_before[q1] = live - l1;
+        s_weight[q0] = l0; s_weight[q1] = l1;
         if (lane == 31) s_start[64] = incl;
     }
     __syncthreads();
     const int t_all = s_start[64];
     const int n_used = min(n_ctas, max(1, t_all / 4));           // at least four tiles per CTA
-    for (int c = tid; c <= n_used; c += 1024) s_cut[c] = (int)((long long)t_all * c / n_used);
+    // the cuts of the one-launch path (a pair costs its tiles plus the cost of a unit)
+    const int unit_cost = fused_plan::contiguous_unit_cost(rows_max);
+    for (int c = tid; c <= n_used; c += 1024)
+        s_cut[c] = fused_plan::contiguous_cut(c, n_used, t_all, pairs, unit_cost, s_tiles, s_weight, s_start, s_live_before, B, Hkv);
     __syncthreads();
     auto req_of = [&](int x) -> int {                            // request whose pairs hold tile x of the sequence
         int r = 0;
         for (int q = 1; q < B; ++q) if (s_start[q] <= x && s_n[q] > 0 && s_tiles[q] > 0) r = q;
         return r;
     };
-    auto cta_of = [&](int x) -> int {                            // the CTA whose range holds tile x (ranges are equal within one)
-        int c = min(n_used - 1, x / max(1, t_all / n_used));       // a guess in 32 bits, then at most a few steps
+    auto cta_of = [&](int x) -> int {                            // the CTA whose (non-empty) range holds tile x
+        int c = min(n_used - 1, x / max(1, t_all / n_used));       // a guess, then steps along the cuts
         while (c + 1 < n_used && s_cut[c + 1] <= x) ++c;
         while (c > 0 && s_cut[c] > x) --c;
         return c;
@@ -218,10 +229,10 @@ attn_plan_kernel(const int32_t* __restrict__ prefix_len, const int32_t* __restri
         const int t_max = __reduce_max_sync(0xffffffffu, t_mx);
         const int t_sum = __reduce_add_sync(0xffffffffu, t_sm);               // < 2^31: at most 64 requests of < 2^24 tiles
         const long long t_all = (long long)t_sum * Hkv;
-        (void)pairs; (void)t_max;
+        (void)t_max;
         if (fused_plan::contiguous_split_pays(rows_max, t_all, n_ctas)) {
             __shared__ int s_start[65];
-            plan_contiguous(s_tiles, s_n, s_start, s_units, s_units + kMaxPlanCtas + 8, B, Hkv, n_ctas, w);   // (the snake deal's s_units is free here)
+            plan_contiguous(s_tiles, s_n, s_start, s_units, s_units + kMaxPlanCtas + 8, B, Hkv, n_ctas, rows_max, pairs, w);   // (the snake deal's s_units is free here)
             return;
         }
     }
