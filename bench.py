@@ -267,17 +267,17 @@ class Workload:
         self.index_stats["index_tokens"] = int(len(tok))
         # the same amount once more as a stream-ordered update (the oldest trajectories leave first to make room): how
         # long the host is held (enqueue) and how long the stream is busy with it
-        for _ in range(2):                                     # (the first call grows the allocator's pool; the second is what an engine sees)
-            war.war_index_evict(ix, k_new)
+        for j in range(2):                                     # (the first call grows the allocator's pool; the second is what an engine sees)
+            war.war_index_evict(ix, k_new)                     # trajectories [j * k_new, (j + 1) * k_new) leave ... and come back below
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize()
             t0 = time.perf_counter()
             e0.record()
-            war.war_index_append_async(ix, d_tok, off[:k_new + 1])
+            war.war_index_append_async(ix, d_tok, off[j * k_new:(j + 1) * k_new + 1])
             e1.record()
             host_s = time.perf_counter() - t0
             torch.cuda.synchronize()
-        self.index_stats["index_append_async"] = {"trajectories": k_new, "tokens": int(off[k_new]), "host_seconds": host_s,
+        self.index_stats["index_append_async"] = {"trajectories": k_new, "tokens": int(off[2 * k_new] - off[k_new]), "host_seconds": host_s,
                                                   "stream_seconds": 1e-3 * e0.elapsed_time(e1)}
         return ix
 
