@@ -3,7 +3,8 @@
 //
 // Match.  Four lanes own each candidate length 1..32 (warps 0-3 the lower end of the pattern's suffix-array interval,
 // warps 4-7 the upper end): a binary search inside the first token's bucket, pipelined two probes deep.  The longest
-// occurring length wins (occurrence is monotone in the length).
+// occurring length wins (occurrence is monotone in the length), and a length's search stops as soon as it is known not
+// to matter (a shorter length does not occur, or a sufficiently longer one does).
 //
 // Tree.  A node is a suffix-array interval [lo, lo+cnt) whose suffixes share the first `depth` tokens.  Its
 // children are the maximal runs between positions with lcp <= depth; a run's token is the suffix's token at
@@ -227,6 +228,7 @@ struct Shared {
     int mode, cur, lo, cnt, depth, n_nodes, thr_shared, long_runs_only, full_lo, full_cnt;
     int n_running, n_cap;
     int m_lo[32], m_hi[32], m_occ[32];          // per candidate length: interval [lo, hi) of its pattern, occurs
+    int min_fail, max_ok;                       // smallest length known not to occur, largest length known to occur
     int memo_slot;                              // >= 0: the node being expanded goes into this memo entry when it is done
     // a batch of small nodes created in one round (equal counts), expanded by one warp each
     int it_slot[kWarps], it_lo[kWarps], it_cnt[kWarps], it_depth[kWarps], n_items;
@@ -260,6 +262,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const war_index_view* __res
     int32_t* o_cnt = count ? count + row * N : nullptr;
 
     if (tid < P) sh.pat[tid] = tail[(size_t)b * P + tid];
+    if (tid == 0) { sh.min_fail = kMaxP + 1; sh.max_ok = 0; }
     // Workload-aware switch: a request with tail_len < 0 is not running; when more requests run than the limit,
     // nothing is looked up and every running request gets the root alone (a plain decode step through the same
     // calls).  Every CTA counts the running requests itself: no extra launch, no state between calls.
@@ -375,6 +378,12 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const war_index_view* __res
     // lanes per length (thread t: length (t % 128) / 4 + 1, every fourth token from t % 4 on behind the known common
     // prefix), so one probe of a binary search compares up to 32 tokens in a single memory latency whatever the depth of
     // the match.  The four lanes of a group hold the same search state.
+    // Occurrence is monotone in the length, and only the longest occurring length (and, when several lengths are
+    // scored, the few below it) is drafted from.  So a search is given up as soon as it cannot matter: every group
+    // posts its verdict the moment it has one (largest length seen to occur, smallest seen not to), and a group whose
+    // length lies above the latter or too far below the former stops probing.  The searches take as many steps as
+    // their buckets are deep (up to 22 on a frequent token against 10 on an average one), one memory latency each,
+    // so this ends the phase with the deepest bucket among the lengths that count instead of among all 32.
     const int tl = min(max(my_tl, 0), P);
     if (warp < 8) {
         const bool upper = warp >= 4;                             // first suffix above every suffix that starts with the pattern
@@ -392,6 +401,11 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const war_index_view* __res
                 searching = len > 1 && occurs;
             }
         }
+        const int keep_below = (int)gridDim.y - 1;                // lengths this far below the longest match are still drafted from
+        if (!upper && part == 0 && !searching) {                  // decided without a search
+            if (occurs) atomicMax(&sh.max_ok, len); else atomicMin(&sh.min_fail, len);
+        }
+        bool given_up = false;
         // bound by binary search; it remembers how many tokens the pattern shares with the suffixes at its
         // current ends, so comparisons restart there (all bucket members share token 0).  The search is pipelined two
         // probes deep so that a step costs one memory latency instead of two or three: while the current probe is
@@ -409,7 +423,12 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const war_index_view* __res
             c0 = at < len ? corpus[(int64_t)s_mid + at] : 0;
             c1 = at + 4 < len ? corpus[(int64_t)s_mid + at + 4] : 0;
         }
+        int seen_fail = kMaxP + 1, seen_ok = 0;                   // the two verdict words as read during the previous step
         while (__any_sync(0xffffffffu, a < z)) {                  // first suffix >= pattern (upper: > every match)
+            if (a < z && (len > seen_fail || len < seen_ok - keep_below)) {
+                z = a;                                            // this length no longer matters
+                given_up = true;
+            }
             const bool active = a < z;
             const int mid_l = a + ((mid - a) >> 1), mid_r = mid + 1 + ((z - mid - 1) >> 1);
             const bool has_l = active && a < mid, has_r = active && mid + 1 < z;
@@ -422,6 +441,10 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const war_index_view* __res
             const int from = min(ma, mz), nt = from + part;
             const int l0 = has_l && nt < len ? corpus[(int64_t)s_l + nt] : 0, l1 = has_l && nt + 4 < len ? corpus[(int64_t)s_l + nt + 4] : 0;
             const int r0 = has_r && nt < len ? corpus[(int64_t)s_r + nt] : 0, r1 = has_r && nt + 4 < len ? corpus[(int64_t)s_r + nt + 4] : 0;
+            // the verdicts so far ride along with this step's loads and are looked at when the next step begins, where
+            // the step waits for those loads anyway (a wait of their own anywhere else costs the step a second latency)
+            seen_fail = *(volatile int*)&sh.min_fail;
+            seen_ok = *(volatile int*)&sh.max_ok;
             // first differing position of the group (position * 2 + "corpus token smaller"); 2 * len = none differs.
             // Eight tokens first: most probes differ there; the rest (up to 24 more) only for the groups that need them.
             int key;
@@ -456,14 +479,18 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const war_index_view* __res
                 if (m < len ? (key & 1) != 0 : upper) { a = mid + 1; ma = m; mid = mid_r; s_mid = s_r; c0 = r0; c1 = r1; s_l = s_rl; s_r = s_rr; }
                 else { z = mid; mz = m; mid = mid_l; s_mid = s_l; c0 = l0; c1 = l1; s_l = s_ll; s_r = s_lr; }
                 at = nt;
+                if (a >= z && !upper && part == 0) {               // this search has just ended: post its verdict
+                    if (a < bucket_hi && mz == len) atomicMax(&sh.max_ok, len); else atomicMin(&sh.min_fail, len);
+                }
             }
         }
         if (!upper) {
             if (searching) {
                 lo = a;
                 // the pattern occurs iff the suffix there starts with it: that suffix was the last probe that was not
-                // below the pattern, and mz tokens of it agreed
-                occurs = lo < bucket_hi && mz == len;
+                // below the pattern, and mz tokens of it agreed (a search that was given up reports nothing: its
+                // length is either above the longest match or below every length that is drafted from)
+                occurs = !given_up && lo < bucket_hi && mz == len;
             }
             if (part == 0) { sh.m_lo[len - 1] = lo; sh.m_occ[len - 1] = occurs; }
         } else if (part == 0) {

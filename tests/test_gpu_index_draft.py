@@ -628,6 +628,41 @@ def test_scored_lengths_on_the_tiny_workload(war):
     ix.destroy()
 
 
+def test_searches_that_stop_early_never_change_an_answer(war):
+    """The match gives up the suffix lengths that cannot matter (above a length that does not occur, or too far below
+    one that does).  Here the lengths differ as much as they can in how long their searches take: one token makes up
+    half of the corpus (a bucket many steps deep), the others are rare (shallow buckets), and the tails put the frequent
+    token at every position while their longest matches run from nothing to the whole tail."""
+    rng = np.random.default_rng(77)
+    vocab, F = 400, 7
+    trajs = []
+    for _ in range(6):
+        t = rng.integers(0, vocab, size=3000)
+        t[rng.random(3000) < 0.5] = F
+        trajs.append(t.tolist())
+    tok, off = _flat(trajs)
+    P, B = 32, 64
+    tails = np.empty((B, P), np.int32)
+    for i in range(B):
+        at = int(rng.integers(P, len(tok)))
+        tails[i] = tok[at - P:at]                                         # occurs as a whole ...
+        cut = P if i == 1 else int(rng.integers(0, P + 1))                # ... then only its last `cut` tokens do
+        if cut < P:
+            tails[i, :P - cut] = rng.integers(0, vocab, size=P - cut)
+            tails[i, P - cut - 1] = vocab - 1 - (tails[i, P - cut - 1] % 2)
+        if i % 3 == 0:
+            tails[i, int(rng.integers(0, P))] = F
+    tl = np.full(B, P, np.int32)
+    tl[5], tl[6] = 3, 0
+    ix = U.build_index(war, tok, off, vocab, max_depth=P + 16)
+    corpus = D.Corpus(tok, off)
+    got = _compare_with_oracle(war, tok, off, vocab, tails, tl, 16, 4, ix=ix)
+    assert got[0].min() == 0 and got[0].max() == P and len(np.unique(got[0])) > 8
+    for nl in (2, 5, 32):
+        _compare_scored(war, ix, corpus, tails, tl, 16, 4, nl)
+    ix.destroy()
+
+
 def test_scored_lengths_argument_checks(war):
     tok, off = _flat([[1, 2, 3, 1, 2, 3]])
     ix = U.build_index(war, tok, off, vocab=4)
