@@ -92,18 +92,22 @@ class ClockSampler:
                 pass
 
     def summary(self, first: int = 0, last=None):
-        sm, mx, reasons = [], [], set()
+        sm, mx, watts, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows[first:last]:
             try:
                 sm.append(float(r[0])); mx.append(float(r[1]))
             except Exception:
                 continue
+            try:
+                watts.append(float(r[2]))
+            except Exception:
+                pass
             for name, v in zip(names, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "power_w": float(np.median(watts)) if watts else None, "reasons": sorted(reasons), "samples": len(sm)}
 
 
 def oracle_sample(cfg, corpus, tails, tail_len, attn, ctx, targets_fn, requests, budget_s=None, keep=False):
