@@ -2,7 +2,8 @@
 // interval into a frequency-ranked token tree.  One CTA per request.
 //
 // Match.  Four lanes own each candidate length 1..32 (warps 0-3 the lower end of the pattern's suffix-array interval,
-// warps 4-7 the upper end): a binary search inside the first token's bucket, pipelined two probes deep.  The longest
+// warps 4-7 the upper end): a binary search inside the first token's bucket, pipelined two probes deep; lengths 2-5 are
+// searched 33-way instead, by a warp each (warps 8-15).  The longest
 // occurring length wins (occurrence is monotone in the length), and a length's search stops as soon as it is known not
 // to matter (a shorter length does not occur, or a sufficiently longer one does).
 //
@@ -31,6 +32,7 @@ constexpr int kPoolCap = kMaxN * kMaxK;
 constexpr int kMemoMinCount = 33;        // nodes with at least this many occurrences go through the index's memo
 constexpr int kBlockScanMin = 1024;          // intervals at least this long are scanned by every warp (measured: 1024-2048 best)
 constexpr int kLongRunFirstMin = 1024;       // intervals at least this long first look for runs of 16 or more only
+constexpr int kWideFirst = 2, kWideLast = 5;  // candidate lengths searched 33-way by a warp of their own (warps 8-15)
 
 struct TopK {                                 // warp-uniform, sorted by (cnt desc, start asc)
     int cnt[kMaxK];
@@ -391,7 +393,8 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const war_index_view* __res
         const int* pat = sh.pat + (P - len);
         int lo = 0, bucket_hi = 0;
         bool occurs = false, searching = false;
-        if (len <= tl) {
+        const bool wide = len >= kWideFirst && len <= kWideLast && len <= tl;    // a warp of its own searches this length
+        if (len <= tl && !wide) {
             bool valid = true;
             for (int t = 0; t < len; ++t) valid = valid && pat[t] >= 0 && pat[t] < vocab;
             if (valid) {
@@ -402,7 +405,7 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const war_index_view* __res
             }
         }
         const int keep_below = (int)gridDim.y - 1;                // lengths this far below the longest match are still drafted from
-        if (!upper && part == 0 && !searching) {                  // decided without a search
+        if (!upper && part == 0 && !searching && !wide) {         // decided without a search
             if (occurs) atomicMax(&sh.max_ok, len); else atomicMin(&sh.min_fail, len);
         }
         bool given_up = false;
@@ -492,9 +495,66 @@ war_draft_kernel(const int32_t* __restrict__ corpus, const war_index_view* __res
                 // length is either above the longest match or below every length that is drafted from)
                 occurs = !given_up && lo < bucket_hi && mz == len;
             }
-            if (part == 0) { sh.m_lo[len - 1] = lo; sh.m_occ[len - 1] = occurs; }
-        } else if (part == 0) {
+            if (part == 0 && !wide) { sh.m_lo[len - 1] = lo; sh.m_occ[len - 1] = occurs; }
+        } else if (part == 0 && !wide) {
             sh.m_hi[len - 1] = searching ? a : bucket_hi;         // a one-token pattern's interval is its bucket
+        }
+    } else {
+        // Warps 8-15: the short candidate lengths, the ones that nearly always decide the match (the typical longest
+        // match is two to four tokens, and the search of the first length that fails is what releases all longer
+        // ones).  A warp per length and interval end narrows the bucket 33-way: every lane probes one suffix (its
+        // suffix-array entry, then the pattern's few tokens, all in flight together: two memory latencies per step)
+        // and the ballot of "sorts below the end that is looked for" picks the sub-interval.  A bucket of 2^21
+        // suffixes takes 5 steps = 10 latencies instead of the binary search's 21.
+        const int len = kWideFirst + ((warp - 8) & 3);
+        const bool upper = warp >= 12;
+        if (len <= tl) {
+            const int* pat = sh.pat + (P - len);
+            bool valid = true;
+            for (int t = 0; t < len; ++t) valid = valid && pat[t] >= 0 && pat[t] < vocab;
+            int a = 0, z = 0, bucket_hi = 0;
+            if (valid) { a = bucket[pat[0]]; bucket_hi = z = bucket[pat[0] + 1]; }
+            bool z_starts = false, given_up = false;              // z_starts: the suffix at z starts with the pattern
+            int q[kWideLast];
+            for (int t = 1; t < kWideLast; ++t) q[t] = t < len ? pat[t] : 0;
+            while (a < z) {
+                if (len > *(volatile int*)&sh.min_fail) { given_up = true; break; }
+                const int n = z - a;
+                const bool last = n <= 32;
+                const int pos = last ? a + lane : a + (int)(((unsigned long long)(lane + 1) * (unsigned)n) / 33u);
+                const bool live = !last || lane < n;
+                int cmp = 0;                                      // -1 the suffix sorts below the pattern, 0 starts with it, 1 above
+                if (live) {
+                    const int64_t sfx = sa[pos];
+                    int c[kWideLast];
+#pragma unroll
+                    for (int t = 1; t < kWideLast; ++t) c[t] = t < len ? corpus[sfx + t] : 0;
+#pragma unroll
+                    for (int t = 1; t < kWideLast; ++t)
+                        if (t < len && cmp == 0 && c[t] != q[t]) cmp = c[t] < q[t] ? -1 : 1;
+                }
+                const unsigned below = __ballot_sync(0xffffffffu, live && (upper ? cmp <= 0 : cmp < 0));
+                const unsigned starts = __ballot_sync(0xffffffffu, live && cmp == 0);
+                const int cnt = __popc(below);                    // the suffixes are sorted: the lanes below form a prefix
+                const int pos_prev = __shfl_sync(0xffffffffu, pos, max(cnt - 1, 0));
+                const int pos_next = __shfl_sync(0xffffffffu, pos, min(cnt, 31));
+                if (last) {
+                    if (cnt < n) z_starts = (starts >> cnt) & 1u;
+                    a = z = a + cnt;
+                } else {
+                    if (cnt < 32) { z = pos_next; z_starts = (starts >> cnt) & 1u; }
+                    if (cnt > 0) a = pos_prev + 1;
+                }
+            }
+            if (lane == 0) {
+                if (!upper) {
+                    const bool occurs = valid && !given_up && a < bucket_hi && z_starts;
+                    sh.m_lo[len - 1] = a; sh.m_occ[len - 1] = occurs;
+                    if (!given_up) { if (occurs) atomicMax(&sh.max_ok, len); else atomicMin(&sh.min_fail, len); }
+                } else {
+                    sh.m_hi[len - 1] = a;
+                }
+            }
         }
     }
     __syncthreads();
