@@ -62,6 +62,18 @@ __device__ __forceinline__ void tma_load_block(uint32_t dst, const CUtensorMap* 
         ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(block) : "memory");
 }
 
+// The same copy with an L2 eviction policy for the lines it brings in.
+__device__ __forceinline__ void tma_load_block_hint(uint32_t dst, const CUtensorMap* map, int block, uint64_t* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %3, %3, %3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(block), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
 // plain (untiled) bulk copy global -> shared: both addresses 16-byte aligned, size a multiple of 16 bytes
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

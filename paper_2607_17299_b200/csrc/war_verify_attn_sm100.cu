@@ -364,6 +364,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     if (warp == 8) {
         // ------------------------------------------------------------------ producer
+        // One-launch variant (64 requests or fewer), one row block per kv head: every K/V line is read once per call,
+        // by one CTA, and is marked to leave L2 first, so that the stream does not push out what the step reads again
+        // (the index the draft kernel probes, page tables, the kernels' own code).  With several row blocks the
+        // siblings share K/V through L2 and the lines keep the default policy; so do the large batches of the
+        // three-launch variant, where the mark bought nothing and cost 2-3 %.
+        const bool stream_once = kFused && a.w.row_blocks == 1;
+        const uint64_t evict_first = kFused ? l2_policy_evict_first() : 0ull;
         uint32_t ld = 0;
         bool ok = true;
         fused_plan::Cursor cur{0, 0, 0};
@@ -395,7 +402,8 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                     if (pg < 0 || pg >= a.num_pages) { war_set_device_status(a.status_word, WAR_ERR_BAD_PAGE); pg = 0; }
                     const CUtensorMap* map = is_v ? &v_map : &k_map;
                     if (!kTokenMajor) {
-                        tma_load_block(sRing + slot * kSlotBytes + lane * page_bytes, map, (int)(pg * a.Hkv + un.kvh), &bars->full[slot]);
+                        if (stream_once) tma_load_block_hint(sRing + slot * kSlotBytes + lane * page_bytes, map, (int)(pg * a.Hkv + un.kvh), &bars->full[slot], evict_first);
+                        else tma_load_block(sRing + slot * kSlotBytes + lane * page_bytes, map, (int)(pg * a.Hkv + un.kvh), &bars->full[slot]);
                     } else {
                         const uint32_t dst = sRing + slot * kSlotBytes + lane * (page_bytes >> 1);
                         tma_load_half_page(dst, map, 0, un.kvh, (int)pg, &bars->full[slot]);
