@@ -345,6 +345,7 @@ __device__ __noinline__ static void make(const int32_t* __restrict__ prefix_len,
         pl->u.s.nc[tid] = (uint16_t)nc;
         pl->pos_req[pos] = (uint8_t)tid;
         sc->units_by_pos[pos] = nc * sc->weight[tid];
+        sc->live_before[pos] = nc > 1 ? sc->weight[tid] : 0;      // (idle in this mode) split triples of the request
     }
     __syncthreads();
     if (warp == 0) {                                             // exclusive scan over the sorted positions, two per lane
@@ -355,7 +356,10 @@ __device__ __noinline__ static void make(const int32_t* __restrict__ prefix_len,
         for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
         pl->u.s.pos_base[a0] = (uint16_t)(incl - m0 - m1);
         pl->u.s.pos_base[a1] = (uint16_t)(incl - m1);
-        if (lane == 31) { pl->mode = 0; pl->total = incl; pl->r0 = 0; pl->h0 = 0; pl->lo = 0; pl->hi = 0; pl->t_all = 0; pl->n_used = 0; pl->c0_first = 0; pl->c1_last = 0; }
+        const int split = __reduce_add_sync(0xffffffffu, (a0 < B ? sc->live_before[a0] : 0) + (a1 < B ? sc->live_before[a1] : 0));
+        // (in this mode n_used holds the number of split (request, kv head, row block) triples and t_all the largest
+        // number of rows of a row block, for the deal of the merges)
+        if (lane == 31) { pl->mode = 0; pl->total = incl; pl->r0 = 0; pl->h0 = 0; pl->lo = 0; pl->hi = 0; pl->t_all = min(rows_max, kRowBlock); pl->n_used = split; pl->c0_first = 0; pl->c1_last = 0; }
     }
     __syncthreads();
 }

@@ -36,6 +36,8 @@ struct AttnWorkspace {
     int* pair_chunks;    // [B, Hkv]             and the number of chunks
     unsigned long long* pair_count;   // [B, Hkv, row_blocks]  one-launch path: (call number << 16) | units of a split
                                       // triple that have left their partial result
+    unsigned long long* pair_seen;    // [B, Hkv, row_blocks]  the same for the CTAs that share the triple's merge and have
+                                      // seen all of its partials
     AttnReq* req;        // [B]
     uint64_t* anc;       // [B, N] bit a of anc[b, j]: slot a is j or an ancestor of j
     AttnUnit* units;     // [max_units]
@@ -78,6 +80,7 @@ inline AttnWorkspace war_attn_workspace_layout(const war_attn_params_t* p, void*
     w.units = (AttnUnit*)(b + at); at += align(sizeof(AttnUnit) * (size_t)w.max_units);
     w.part_ml = (float*)(b + at); at += align(sizeof(float) * 2 * (size_t)w.max_units * w.rows);
     w.part_o = (float*)(b + at); at += align(sizeof(float) * (size_t)w.max_units * w.rows * p->D);
+    w.pair_seen = (unsigned long long*)(b + at); at += align(sizeof(unsigned long long) * (size_t)p->B * p->Hkv * w.row_blocks);
     w.bytes = at;
     return w;
 }

@@ -163,9 +163,23 @@ __device__ __forceinline__ void count_arrival(unsigned long long* p, unsigned lo
         cur = prev;
     }
 }
-// Bounded wait (one thread) until `target` arrivals of this call have been counted in *p; then the word is cleared.
+// The same count that also says how many of this call's arrivals there are now, this one included.
+__device__ __noinline__ int count_arrival_ranked(unsigned long long* p, unsigned long long call) {
+    const unsigned long long old = atomicAdd(p, 1ull);
+    if ((old >> 16) == call) return (int)(old & 0xffffull) + 1;
+    unsigned long long cur = old + 1ull;
+    while (true) {
+        if ((cur >> 16) == call) return (int)(atomicAdd(p, 1ull) & 0xffffull) + 1;
+        const unsigned long long prev = atomicCAS(p, cur, (call << 16) | 1ull);
+        if (prev == cur) return 1;
+        cur = prev;
+    }
+}
+// Bounded wait (one thread) until `target` arrivals of this call have been counted in p[0]; then the word is cleared.
+// When `parts` CTAs merge the triple, each a share of its rows, every one of them waits here; they count themselves
+// in *seen once they have seen the arrivals, and the last one to do so clears both words.
 template <class BarsT>
-__device__ __forceinline__ bool wait_arrivals(unsigned long long* p, unsigned long long call, int target, BarsT* bars, int* status_word) {
+__device__ __forceinline__ bool wait_arrivals(unsigned long long* p, unsigned long long* seen, unsigned long long call, int target, int parts, BarsT* bars, int* status_word) {
     auto there = [&]() -> bool {
         unsigned long long v;
         asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
@@ -186,6 +200,10 @@ __device__ __forceinline__ bool wait_arrivals(unsigned long long* p, unsigned lo
         }
     }
     __threadfence();
+    if (parts > 1) {
+        if (count_arrival_ranked(seen, call) < parts) return true;
+        *(volatile unsigned long long*)seen = 0ull;
+    }
     *(volatile unsigned long long*)p = 0ull;
     return true;
 }
@@ -203,7 +221,8 @@ struct MergeArgs {
     __nv_bfloat16* out; float* lse; int* status_word;
     int rows, G, N, Hq;
     int req, kvh, rb, n_nodes, n_chunks, slot_base, slot_stride, bump;
-    unsigned long long* arrivals; unsigned long long call;
+    int part, parts, share;              // this CTA merges share `part` of `parts`: rows [part * share, + share), share even
+    unsigned long long* arrivals; unsigned long long* seen; unsigned long long call;
 };
 template <class BarsT>
 __device__ __noinline__ bool merge_partials(const MergeArgs m, uint8_t* smem, BarsT* bars, uint32_t* phase_io) {
@@ -215,11 +234,19 @@ __device__ __noinline__ bool merge_partials(const MergeArgs m, uint8_t* smem, Ba
     const int rows_g = min(kRowBlock, ((kSlots * kSlotBytes) / (nch * 512)) & ~1);     // even, >= 2 (nch <= kFusedMaxChunks)
     const float* s_o = (const float*)(smem + kOffRing);
     const float2* s_ml = (const float2*)(smem + kOffQ);
-    for (int row0 = 0; row0 < rows_valid; row0 += rows_g, ++phase) {
-        const int rg = min(rows_g, (rows_valid - row0 + 1) & ~1);                     // rows copied (even; the workspace has them)
+    int r_lo = 0, r_hi = rows_valid;
+    if (m.parts > 1) {
+        r_lo = m.part * m.share; r_hi = min(rows_valid, r_lo + m.share);
+        if (r_lo >= r_hi) {                   // nothing falls to this share; it still takes part in clearing the counter
+            if (tid == 0 && !wait_arrivals(m.arrivals, m.seen, m.call, nch, m.parts, bars, m.status_word)) return false;
+            return true;
+        }
+    }
+    for (int row0 = r_lo; row0 < r_hi; row0 += rows_g, ++phase) {
+        const int rg = min(rows_g, (r_hi - row0 + 1) & ~1);                           // rows copied (even; the workspace has them)
         if (tid == 0) {
             // every chunk has left its partial
-            if (row0 == 0 && !wait_arrivals(m.arrivals, m.call, nch, bars, m.status_word)) { *phase_io = phase; return false; }
+            if (row0 == r_lo && !wait_arrivals(m.arrivals, m.seen, m.call, nch, m.parts, bars, m.status_word)) { *phase_io = phase; return false; }
             // the previous group's readers are done with the buffers
             if (phase > 0 && !mbar_wait(&bars->merge_free, (phase - 1) & 1u, bars, m.status_word)) { *phase_io = phase; return false; }
             mbar_arrive_expect_tx(&bars->merge_full, (uint32_t)(nch * rg * (512 + 8)));
@@ -236,7 +263,7 @@ __device__ __noinline__ bool merge_partials(const MergeArgs m, uint8_t* smem, Ba
         const int sub = lane & 7;
         for (int rbase = w8 * 4; rbase < rg; rbase += 32) {
             const int r = rbase + (lane >> 3);
-            const bool live = r < rg && row0 + r < rows_valid;
+            const bool live = r < rg && row0 + r < r_hi;
             const int rr = live ? r : 0;
             float M = -CUDART_INF_F;
 #pragma unroll 1
@@ -768,13 +795,16 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
             // requests are dealt to the CTAs in turn, so the work at the end of the kernel is spread over all SMs.
             // Nothing waits for this CTA any more (its own partials are out), so waiting here cannot close a cycle. ----
             uint32_t merge_phase = 0;
-            auto merge_one = [&](const UnitView& un) -> bool {
+            int share = kRowBlock;
+            auto merge_one = [&](const UnitView& un, int part, int parts) -> bool {
                 MergeArgs m;
+                m.part = part; m.parts = parts; m.share = share;
                 m.part_o = a.w.part_o; m.part_ml = a.w.part_ml; m.out = a.out; m.lse = a.lse; m.status_word = a.status_word;
                 m.rows = a.w.rows; m.G = a.G; m.N = a.N; m.Hq = a.Hq;
                 m.req = un.req; m.kvh = un.kvh; m.rb = un.rb; m.n_nodes = un.n_nodes; m.n_chunks = un.n_chunks;
                 m.slot_base = un.slot_base; m.slot_stride = un.slot_stride; m.bump = un.bump;
                 m.arrivals = &a.w.pair_count[(un.req * a.Hkv + un.kvh) * a.w.row_blocks + un.rb]; m.call = a.call;
+                m.seen = &a.w.pair_seen[(un.req * a.Hkv + un.kvh) * a.w.row_blocks + un.rb];
                 const bool done = merge_partials(m, smem, bars, &merge_phase);
                 return done;
             };
@@ -789,27 +819,37 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                     UnitView un;
                     if (!fetch(cur, un)) break;
                     if (un.n_chunks == 1 || un.chunk != 0 || tree_bad(un.req, un.n_nodes)) continue;
-                    ok = merge_one(un);
+                    ok = merge_one(un, 0, 1);
                 }
             } else {
-                int dealt = 0;                                         // triples of split requests before this one
+                // With few split triples every one is merged by two, four or eight CTAs, a share of its rows each: a
+                // triple of many chunks is up to a megabyte that one SM would bring in and walk through in several
+                // rounds.  Shares of at least 16 rows, on at most half of the CTAs (measured: 1 and 2 requests
+                // with 128-row trees 74 -> 47 and 75 -> 64 us per call, 2 and 3 requests with 32-row trees 64 -> 60
+                // and 71 -> 68; more shares than that bought nothing or cost a microsecond).
+                const int n_split = plan->n_used, rows_blk = plan->t_all;
+                int parts = 1, lg = 0;
+                while (parts < 8 && 4 * parts * n_split <= (int)gridDim.x && rows_blk >= 32 * parts) { parts *= 2; ++lg; }
+                share = (((rows_blk + parts - 1) >> lg) + 1) & ~1;
+                int dealt = 0;                                         // shares of split requests before this one
 #pragma unroll 1
                 for (int p = 0; p < a.B && ok; ++p) {
                     const int i = plan->pos_req[p];
                     const int nc = plan->u.s.nc[i], n = plan->n[i];
                     if (nc <= 1 || n == 0) continue;
-                    const int rbs = (a.G * n + kRowBlock - 1) / kRowBlock, per = a.Hkv * rbs;
+                    const int rbs = (a.G * n + kRowBlock - 1) / kRowBlock, per = a.Hkv * rbs, shares = per * parts;
                     int k = ((int)blockIdx.x - dealt) % (int)gridDim.x;
                     if (k < 0) k += gridDim.x;
-                    dealt += per;
-                    if (k >= per || tree_bad(i, n)) continue;
+                    dealt += shares;
+                    if (k >= shares || tree_bad(i, n)) continue;
 #pragma unroll 1
-                    for (; k < per && ok; k += gridDim.x) {
+                    for (; k < shares && ok; k += gridDim.x) {
+                        const int part = k / per, tr = k - part * per;       // the shares of a triple sit `per` CTAs apart
                         UnitView un;
-                        un.req = i; un.kvh = k / rbs; un.rb = k - un.kvh * rbs; un.n_nodes = n; un.n_chunks = nc; un.chunk = 0;
+                        un.req = i; un.kvh = tr / rbs; un.rb = tr - un.kvh * rbs; un.n_nodes = n; un.n_chunks = nc; un.chunk = 0;
                         un.tile_begin = un.tile_end = 0; un.slot = 0;
-                        un.slot_base = (int)plan->u.s.pos_base[p] + k; un.slot_stride = per; un.bump = 0;
-                        ok = merge_one(un);
+                        un.slot_base = (int)plan->u.s.pos_base[p] + tr; un.slot_stride = per; un.bump = 0;
+                        ok = merge_one(un, part, parts);
                     }
                 }
             }

@@ -358,6 +358,63 @@ def test_mid_size_batches_through_every_plan(war, seed):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("B,N,G", [(1, 32, 4), (2, 32, 4), (3, 24, 4), (2, 8, 4), (1, 64, 8), (4, 16, 4)])
+def test_few_requests_whose_merges_are_shared_out(war, B, N, G):
+    """With a handful of long requests every (request, kv head, row block) is cut into many chunks and its merge is
+    shared out to two, four or eight CTAs, a share of the rows each, which count themselves on a second counter word
+    before the last one clears both.  Checked against the fp64 checker, bit for bit against the three-launch path, and
+    on repeated calls and graph replays with one and the same workspace (the counters must come back to a state in which
+    the next call, or the replay with its frozen call number, starts from nothing)."""
+    rng = np.random.default_rng(4100 + 10 * B + N)
+    Hkv = 8
+    ctx = rng.integers(14000, 26000, B)
+    cfg = W.scaled(W.CONFIGS["low"], B=B, N=N, Hkv=Hkv, Hq=Hkv * G, page_size=16)
+    a = W.make_attention_inputs(cfg, np.asarray(ctx), device=U.dev())
+    nn = np.full(B, N, np.int32)
+    nn[-1] = max(1, N - 3)
+    par = np.full((B, N), -1, np.int32)
+    for i in range(B):
+        for j in range(1, nn[i]):
+            par[i, j] = int(rng.integers(0, j))
+    scale = 1.0 / np.sqrt(cfg.D)
+    d = U.dev()
+    params = war.attn_params(a.q, a.k_pool, a.v_pool, a.page_table, scale, 0)
+    ws = torch.full((war.war_verify_attn_workspace_bytes(params),), 0xa5, dtype=torch.uint8, device=d)
+    d_nn, d_par = torch.from_numpy(nn).to(d), torch.from_numpy(par).to(d)
+    outs = []
+    for _ in range(3):
+        out = torch.full(a.q.shape, 7.0, dtype=torch.bfloat16, device=d)
+        lse = torch.full(a.q.shape[:3], 7.0, dtype=torch.float32, device=d)
+        war.war_verify_attn(a.q, a.k_pool, a.v_pool, a.page_table, a.prefix_len, d_nn, d_par, params, ws, out, lse)
+        torch.cuda.synchronize()
+        outs.append((out, lse))
+    g_out = torch.full(a.q.shape, 7.0, dtype=torch.bfloat16, device=d)
+    g_lse = torch.full(a.q.shape[:3], 7.0, dtype=torch.float32, device=d)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            war.war_verify_attn(a.q, a.k_pool, a.v_pool, a.page_table, a.prefix_len, d_nn, d_par, params, ws, g_out, g_lse)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        g_out.fill_(7.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(g_out, outs[0][0]) and torch.equal(g_lse, outs[0][1])
+    assert all(torch.equal(o, outs[0][0]) and torch.equal(l, outs[0][1]) for o, l in outs[1:])
+    got3, got3_lse, raw3 = U.run_attn(war, a, nn, par, scale, 2)
+    live = torch.arange(N, device=d)[None, :] < d_nn[:, None]
+    assert torch.equal(outs[0][0][live], raw3[live]) and torch.equal(outs[0][1][live], torch.from_numpy(got3_lse).to(d)[live])
+    want = A.verify_attention(a.q, a.k_pool, a.v_pool, a.page_table.cpu().numpy(), a.prefix_len.cpu().numpy(), nn, par, scale)
+    got, got_lse = outs[0][0].float().cpu().numpy(), outs[0][1].cpu().numpy()
+    for i in range(B):
+        U.assert_attention_close(got[i], got_lse[i], want[i][0], want[i][1], int(nn[i]))
+    assert war.war_device_status() == 0
+    del a
+    torch.cuda.empty_cache()
+
+
 def test_a_wait_that_runs_out_ends_with_an_error_not_a_hang(war):
     """Every wait inside the tensor-core kernel has a time budget.  The library's self-test runs the same wait routine
     on a barrier that nobody completes: the waiter gives up after its budget (here 1 ms instead of the kernel's 2 s),
