@@ -635,9 +635,20 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                     for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, r + c * 32);
                     tmem_wait_ld();
                     if (need_mask) {
+                        // Which of the tile's 128 keys this row sees, as a bit mask built once: the first d keys are
+                        // prefix (all visible), key d + a is tree slot a (visible when a is the row's slot or an ancestor;
+                        // the ancestor mask has no bit at or above num_nodes, so keys past the request's end are out).
+                        // Two instructions per element afterwards: this path runs once per (request, kv head) and its
+                        // code, fetched cold, competes with the main loop for the instruction cache.
+                        const int d = pl - key0;                                  // < 128 here
+                        unsigned long long lo, hi;
+                        if (d >= 64) { lo = ~0ull; hi = ((1ull << (d - 64)) - 1ull) | (anc << (d - 64)); }
+                        else if (d > 0) { lo = ((1ull << d) - 1ull) | (anc << d); hi = anc >> (64 - d); }
+                        else { lo = d > -64 ? anc >> (-d) : 0ull; hi = 0ull; }
+                        const uint32_t w[4] = {(uint32_t)lo, (uint32_t)(lo >> 32), (uint32_t)hi, (uint32_t)(hi >> 32)};
 #pragma unroll
                         for (int e = 0; e < 128; ++e)
-                            if (!key_visible(key0 + e, pl, L, anc)) r[e] = 0xff800000u;     // -inf
+                            if (!((w[e >> 5] >> (e & 31)) & 1u)) r[e] = 0xff800000u;     // -inf
                     }
                     float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
