@@ -690,7 +690,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                         if (ok) {
                             tc_fence_after();
                             const float f = rescale ? corr : 1.f;
-#pragma unroll
+#pragma unroll 1                                                    // (rare: kept small, see the mask path above)
                             for (int c = 0; c < 4; ++c) {
                                 uint32_t o[32];
                                 tmem_ld32(tO + c * 32, o);
@@ -750,7 +750,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                     const bool split = un.n_chunks != 1;
                     const float f0 = split ? w0 : (lsum > 0.f ? w0 / lsum : 0.f), f1 = split ? w1 : (lsum > 0.f ? w1 / lsum : 0.f);
                     const bool use1 = theirs > 0;                  // uniform: O of group 1 is stale when it had no tile
-#pragma unroll
+#pragma unroll 1                                                    // (once per unit: kept small, see the mask path above)
                     for (int c = 0; c < 8; ++c) {
                         uint32_t o0[16], o1[16];
                         tmem_ld16(tO + c * 16, o0);
