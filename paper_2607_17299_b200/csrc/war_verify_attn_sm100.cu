@@ -120,15 +120,16 @@ __device__ __forceinline__ uint64_t warp_ancestor_mask(int q0, int q1, int n, in
     int p0 = (j0 > 0 && j0 < n) ? q0 : 0;
     int p1 = (j1 < n) ? q1 : 0;
     uint64_t a0 = 1ull << j0, a1 = 1ull << j1;
+    // (rolled loops: this runs once per unit, from code that is usually not in the instruction cache)
     if (n <= 32) {
-#pragma unroll
+#pragma unroll 1
         for (int r = 0; r < 5; ++r) {
             const uint64_t b = shfl_u64(a0, p0);
             const int q = __shfl_sync(0xffffffffu, p0, p0);
             a0 |= b; p0 = q;
         }
     } else {
-#pragma unroll
+#pragma unroll 1
         for (int r = 0; r < 6; ++r) {
             const uint64_t b00 = shfl_u64(a0, p0 & 31), b01 = shfl_u64(a1, p0 & 31);
             const uint64_t b10 = shfl_u64(a0, p1 & 31), b11 = shfl_u64(a1, p1 & 31);
