@@ -132,10 +132,10 @@ __device__ __forceinline__ int chunk_search(const int* tiles, const int* weight,
 
 // The contiguous split (the tiles of all (request, kv head) pairs as one sequence, cut into equal ranges, a CTA each)
 // balances the CTAs to within one tile and gives every CTA at most two split units, but a range pays for an extra
-// unit wherever a pair ends inside it.  Measured on 4 to 64 requests of three recipes it wins from about 48 tiles per
+// unit wherever a pair ends inside it.  Measured on 3 to 64 requests of three recipes it wins from 36-40 tiles per
 // CTA on (one row block per kv head); below that the searched chunk length does better.
 __host__ __device__ __forceinline__ bool contiguous_split_pays(int rows_max, long long t_all, int n_ctas) {
-    return rows_max <= kRowBlock && t_all >= 48ll * n_ctas && t_all < (1ll << 30);
+    return rows_max <= kRowBlock && t_all >= 36ll * n_ctas && t_all < (1ll << 30);
 }
 
 constexpr int kFusedMaxChunks = 192;      // chunks per request at most (what the merge of a row group can hold at once)
