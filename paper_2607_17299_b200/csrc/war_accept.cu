@@ -17,24 +17,43 @@ __global__ void war_accept_kernel(const int32_t* __restrict__ ids, const int32_t
     if (b >= B) return;
     __shared__ int s_parent[4][kMaxSlots];
     __shared__ int s_depth[4][kMaxSlots];        // -1 = some slot on the root path does not match
+    __shared__ int s_target[4][kMaxSlots];
     int* par = s_parent[threadIdx.x / 32];
     int* dep = s_depth[threadIdx.x / 32];
+    int* tgt = s_target[threadIdx.x / 32];
 
+    // The whole rows are requested at once, whatever num_nodes says (rows are N long; entries at or beyond num_nodes
+    // are read and ignored): one memory latency instead of the chain num_nodes -> parent -> target[parent].
     int n = num_nodes[b];
+    int p_in[2], id_in[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int j = lane + 32 * h;
+        p_in[h] = -1; id_in[h] = 0;
+        if (j < N) {
+            p_in[h] = parent[(size_t)b * N + j];
+            id_in[h] = ids[(size_t)b * N + j];
+            tgt[j] = target[(size_t)b * N + j];
+        }
+    }
     bool bad = n < 0 || n > N;
     if (bad) n = 0;
+    __syncwarp();
     // matched[j] per lane-owned slot; parents validated here
-    for (int j = lane; j < N; j += 32) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int j = lane + 32 * h;
+        if (j >= N) continue;
         int p = -1, m = 0;
         if (j < n) {
-            p = parent[(size_t)b * N + j];
+            p = p_in[h];
             if (j == 0) {
                 m = 1;
             } else if (p < 0 || p >= j) {
                 bad = true;
             } else {
-                const int want = mode == 0 ? target[(size_t)b * N + p] : target[(size_t)b * N + j];
-                m = ids[(size_t)b * N + j] == want;
+                const int want = mode == 0 ? tgt[p] : tgt[j];
+                m = id_in[h] == want;
             }
         }
         par[j] = p;
@@ -67,7 +86,7 @@ __global__ void war_accept_kernel(const int32_t* __restrict__ ids, const int32_t
         int a = best_slot;
         for (int d = best_depth - 1; d >= 0; --d) { accept_path[(size_t)b * N + d] = a; a = par[a]; }
         accept_len[b] = best_depth;
-        bonus[b] = (mode == 0 && n > 0) ? target[(size_t)b * N + best_slot] : -1;
+        bonus[b] = (mode == 0 && n > 0) ? tgt[best_slot] : -1;
     }
 }
 
