@@ -160,12 +160,23 @@ __device__ __forceinline__ int contiguous_cut(int x, int n_used, int t_all, int 
     const unsigned w_all = (unsigned)t_all + (unsigned)(pairs * unit_cost);
     const unsigned base = w_all / (unsigned)n_used, rem = w_all - base * (unsigned)n_used;
     const unsigned p = base * (unsigned)x + rem * (unsigned)x / (unsigned)n_used;
-    // the request whose pairs hold weighted position p: the last live one that starts at or before it
-    int r = -1;
+    // The request whose pairs hold weighted position p: the last live one that starts at or before it.  Weighted starts
+    // do not decrease with the request index (a request that is not live starts where the next live one does), the
+    // first is 0 and p lies below the end of the sequence, so the last index that starts at or before p is a live
+    // request: a binary search (this runs in every CTA of the one-launch path, for every cut, before the first copy).
+    int r = 0, top = B - 1;
 #pragma unroll 1
-    for (int q = 0; q < B; ++q)
-        if (weight[q] > 0 && (unsigned)(start[q] + live_before[q] * Hkv * unit_cost) <= p) r = q;
-    if (r < 0) return 0;
+    while (r < top) {
+        const int mid = (r + top + 1) >> 1;
+        if ((unsigned)(start[mid] + live_before[mid] * Hkv * unit_cost) <= p) r = mid; else top = mid - 1;
+    }
+    if (weight[r] <= 0) {                                            // (not reached: see above)
+        r = -1;
+#pragma unroll 1
+        for (int q = 0; q < B; ++q)
+            if (weight[q] > 0 && (unsigned)(start[q] + live_before[q] * Hkv * unit_cost) <= p) r = q;
+        if (r < 0) return 0;
+    }
     const unsigned off = p - (unsigned)(start[r] + live_before[r] * Hkv * unit_cost);
     const unsigned w = (unsigned)(tiles[r] + unit_cost);
     const int h = (int)(off / w);
