@@ -869,7 +869,9 @@ def main():
                 table[key] = {"skipped": str(e)}
                 continue
             n_steps = w2.steps_for(0.3, n_steps)                   # long enough for the clock sampler to see it
-            mark0 = clocks.mark()
+            torch.cuda.synchronize()
+            time.sleep(2.0)                                        # the set-up above (filling gigabytes of K/V) and the workloads
+            mark0 = clocks.mark()                                  # before it leave the board at its power cap: let it recover
             tt = w2.time_steps(n_steps, args.warmup, barrier, flush_l2=flush)
             entry = summarize(w2, tt, n_steps, "one launch" if w2.B <= FUSED_MAX_B else "three launches")
             entry["config"] = describe(W.CONFIGS[name], flush)
