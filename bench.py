@@ -723,6 +723,9 @@ def main():
 
     clocks = ClockSampler(local_rank)
     clocks.__enter__()
+    torch.cuda.synchronize()
+    time.sleep(2.0)                                        # the set-up (index build, gigabytes of K/V filled) leaves the board at its
+    # power cap: let it recover before the warm-up steps
     t = wl.time_steps(args.steps, args.warmup, barrier, flush_l2=args.flush_l2, cuda_graph=args.cuda_graph, clocks=clocks)
     time.sleep(0.06)                                       # let the sampler see the end of the timed region
     last_sample = clocks.mark()
